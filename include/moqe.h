@@ -1,0 +1,183 @@
+/*
+ * moqe.h -- C ABI of the routed, weight-only-quantized linear layer of MoQE
+ * (Mixture of Quantization Experts) for NVIDIA B200 (sm_100a).
+ *
+ * The method (paper, Section 3.1 "Mixture of Quantization Experts"): one
+ * full-precision model is quantized into several frozen variants, the
+ * "quantization experts"; a router scores the experts and every sample (one
+ * sequence or one image) is run by exactly ONE expert (Section 3.2 "Router
+ * Model"; Appendix "Convergence Observations", r(x) in [M]).  This library is
+ * the linear layer of such a model when a batch mixes samples routed to
+ * different experts that are all resident in device memory:
+ *
+ *     Y[m][:] = X[m][:] . dequant(W_e(m))^T ,   e(m) = expert of row m
+ *
+ * computed as  sort rows by expert -> grouped dequant-GEMM -> unsort.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name starts with h_.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All work is enqueued on it; no call synchronises except where stated.
+ *   - Matrices are dense row-major: W[N][K] (N output features, K input
+ *     features, K contiguous), X[M][K], Y[M][N]; bf16 = bfloat16 bit patterns.
+ *   - Every call returns a moqe_status.  Argument errors are detected on the
+ *     host before anything is launched and leave outputs untouched.  Errors
+ *     only a kernel can see (an expert id outside [0,E)) never trap: the
+ *     offending rows are written as zeros, a status word is set on the device
+ *     and moqe_async_status() reports it.
+ *   - The caller owns X, Y, ids, perm, offsets and workspaces.  The library
+ *     owns only what a moqe_expert* points at.
+ *   - Row pointers and row pitches must be 16-byte aligned (K % 8 == 0 for
+ *     bf16 rows), else MOQE_ERR_UNSUPPORTED.
+ */
+#ifndef MOQE_H_
+#define MOQE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MOQE_API __attribute__((visibility("default")))
+#else
+#define MOQE_API
+#endif
+
+typedef enum {
+    MOQE_OK = 0,
+    MOQE_ERR_NULL = 1,         /* a required pointer is NULL */
+    MOQE_ERR_SHAPE = 2,        /* a size is negative, zero where it may not be, or inconsistent */
+    MOQE_ERR_UNSUPPORTED = 3,  /* bits not in {3,4,8}; group not 0 or a multiple of 32 dividing K;
+                                  K % 8 != 0; E > MOQE_MAX_EXPERTS; misaligned pointer */
+    MOQE_ERR_ALLOC = 4,        /* device allocation failed */
+    MOQE_ERR_WORKSPACE = 5,    /* workspace NULL or smaller than the *_workspace() figure */
+    MOQE_ERR_MISMATCH = 6,     /* experts of one call disagree on N or K */
+    MOQE_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
+    MOQE_ERR_EXPERT_ID = 8,    /* asynchronous: an id outside [0,E) was seen by a kernel */
+    MOQE_ERR_TIMEOUT = 9       /* asynchronous: a bounded in-kernel wait ran out */
+} moqe_status;
+
+#define MOQE_MAX_EXPERTS 32
+
+/* One quantization expert of one linear layer: b-bit codes in the library's
+ * private packed layout plus fp16 scales and integer zero-points, on device. */
+typedef struct moqe_expert moqe_expert;
+
+/* ---------------------------------------------------------------------------
+ * Expert construction (Section 3.1: the experts are quantized variants of the
+ * same full-precision model, frozen afterwards).  The paper names no quantizer
+ * for this library's purpose; the one implemented is affine round-to-nearest:
+ * for every output channel n and every group of `group` consecutive k
+ * (group == 0: the whole row), in IEEE fp32 with round-half-to-even,
+ *   symmetric : a = max|w|, qmax = 2^(b-1)-1, s = fp16(a/qmax),
+ *               c = clamp(rint(w/s), -qmax, qmax) + 2^(b-1),  z = 2^(b-1)
+ *   asymmetric: lo = min(0,min w), hi = max(0,max w), s = fp16((hi-lo)/(2^b-1)),
+ *               z = clamp(rint(-lo/s), 0, 2^b-1), c = clamp(rint(w/s)+z, 0, 2^b-1)
+ *   s == 0 or non-finite after the fp16 rounding -> s = 1;   dequant = s*(c-z).
+ * W: device fp32 [N][K], finite.  bits in {3,4,8}; group 0 or a multiple of 32
+ * that divides K.  On success *out owns new device buffers (cudaMalloc'ed by
+ * this call; it is therefore not capturable in a CUDA graph) and must be
+ * released with moqe_expert_destroy.  The kernels run on `stream`.
+ * ------------------------------------------------------------------------- */
+MOQE_API moqe_status moqe_quantize_rtn(const float* W, int N, int K, int bits, int group, int sym,
+                              void* stream, moqe_expert** out);
+
+/* Canonical, layout-independent view of an expert, for checking and storage:
+ * codes [N][K] one code per byte, scales_f16 [N][K/g] and zeros_f16 [N][K/g]
+ * as IEEE binary16 bit patterns (zeros hold the integer zero-point; symmetric
+ * experts export 2^(b-1)).  g = K when group == 0.  Any output may be NULL. */
+MOQE_API moqe_status moqe_expert_export(const moqe_expert* e, uint8_t* codes, uint16_t* scales_f16,
+                               uint16_t* zeros_f16, void* stream);
+
+/* Inverse of export: build an expert from canonical device arrays.  For a
+ * symmetric expert zeros_f16 may be NULL. */
+MOQE_API moqe_status moqe_expert_import(int N, int K, int bits, int group, int sym, const uint8_t* codes,
+                               const uint16_t* scales_f16, const uint16_t* zeros_f16, void* stream,
+                               moqe_expert** out);
+
+/* Host-side description.  code_bytes = N*K*bits/8 exactly (the paper's storage
+ * ratios FP16 : Int8 : Int4 = 1 : 1/2 : 1/4, Appendix "Peak VRAM and CPU RAM
+ * usage analysis"); meta_bytes = scales (+ zeros when asymmetric), 2 bytes each;
+ * alloc_bytes = what the packed buffers really occupy (padding included).
+ * Any output may be NULL. */
+MOQE_API moqe_status moqe_expert_info(const moqe_expert* e, int* N, int* K, int* bits, int* group, int* sym,
+                             size_t* code_bytes, size_t* meta_bytes, size_t* alloc_bytes);
+
+/* Frees the expert's device buffers (cudaFree: synchronises the device). */
+MOQE_API moqe_status moqe_expert_destroy(moqe_expert* e);
+
+/* ---------------------------------------------------------------------------
+ * Hard routing (Section 3.2; Appendix: the router's decision r(x) is one expert
+ * index per sample, and the expert's output is not weighted by the score).
+ * ids[s] = smallest index attaining the maximum of logits[s][0..E); NaN never
+ * wins; an all-NaN row gives 0.  logits fp32 [S][E]; ids int32 [S].
+ * ------------------------------------------------------------------------- */
+MOQE_API moqe_status moqe_route(const float* logits, int S, int E, int32_t* ids, void* stream);
+
+/* Per-sample ids -> per-row ids: rows [row_offsets[s], row_offsets[s+1]) take
+ * ids[s].  row_offsets int32 [S+1], non-decreasing, row_offsets[0] == 0,
+ * row_offsets[S] == M.  row_ids int32 [M]. */
+MOQE_API moqe_status moqe_expand_ids(const int32_t* ids, const int32_t* row_offsets, int S, int M,
+                            int32_t* row_ids, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Stable counting sort of rows by expert id, and the row gather / scatter.
+ * (The batching glue between "one expert per sample" and a grouped GEMM; the
+ * per-expert counts are the n_i of the load statistic F_i = n_i / B of
+ * Section 3.3 "Router Fine-Tuning".)
+ *   offsets[e] = number of rows with id < e            (int32 [E+1])
+ *   perm[offsets[e] + r] = the r-th row, in increasing row index, with id e
+ *   Xp[j][:] = X[perm[j]][:]                            (rows of C bf16, C % 8 == 0)
+ * moqe_permute: X and Xp may both be NULL (indices only).  Rows whose id is
+ * outside [0,E) are sorted behind all valid rows (offsets[E] then counts only
+ * the valid ones), their Xp rows are zero, and MOQE_ERR_EXPERT_ID is latched.
+ * workspace: moqe_permute_workspace(M, E) bytes, contents irrelevant on entry.
+ * moqe_unpermute: Y[perm[j]][:] = Yp[j][:].
+ * ------------------------------------------------------------------------- */
+MOQE_API size_t moqe_permute_workspace(int M, int E);
+MOQE_API moqe_status moqe_permute(const void* X_bf16, const int32_t* row_ids, int M, int C, int E, void* Xp_bf16,
+                         int32_t* perm, int32_t* offsets, void* workspace, size_t workspace_bytes,
+                         void* stream);
+MOQE_API moqe_status moqe_unpermute(const void* Yp_bf16, const int32_t* perm, int M, int C, void* Y_bf16,
+                           void* stream);
+
+/* ---------------------------------------------------------------------------
+ * The routed dequant-GEMM (Section 3.1: "the activated quantization expert
+ * performs the inference on this sample" -- here for a whole mixed batch):
+ *   Y[m][n] = bf16( sum_k X[m][k] * s_e[n][k/g] * (c_e[n][k] - z_e[n][k/g]) ),
+ *   e = row_ids[m], accumulated in fp32.
+ * X bf16 [M][K]; row_ids int32 [M]; h_experts: HOST array of E expert handles
+ * that agree on N and K; Y bf16 [M][N] (every row is written; rows with an
+ * invalid id are written as zeros).  M == 0 is valid.  workspace:
+ * moqe_routed_qgemm_workspace(M, N, K, E) bytes, contents irrelevant on entry;
+ * calls that share a workspace must not overlap on the device.
+ * Small batches stream each touched expert's packed weights once (split-K
+ * dequant-MMA kernel); large batches run the persistent tcgen05 grouped GEMM.
+ * ------------------------------------------------------------------------- */
+MOQE_API size_t moqe_routed_qgemm_workspace(int M, int N, int K, int E);
+MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_ids, int M,
+                              const moqe_expert* const* h_experts, int E, void* Y_bf16,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same, with the kernel chosen by the caller (testing / measurement):
+ * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM. */
+MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
+                                   const moqe_expert* const* h_experts, int E, void* Y_bf16,
+                                   void* workspace, size_t workspace_bytes, void* stream, int path);
+
+/* Synchronises `stream`, then returns and clears the first error latched by a
+ * kernel on the current device (MOQE_OK if none). */
+MOQE_API moqe_status moqe_async_status(void* stream);
+
+MOQE_API const char* moqe_status_str(moqe_status s);
+
+/* Number of kernels this library has launched so far in this process. */
+MOQE_API unsigned long long moqe_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOQE_H_ */

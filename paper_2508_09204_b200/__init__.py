@@ -1,0 +1,244 @@
+"""Python binding of ``libmoqe.so`` (the routed quantized-linear library for B200).
+
+Argument marshalling only: every function takes torch CUDA tensors, passes
+their device pointers and the current CUDA stream to the C-ABI call of the
+same name (``include/moqe.h``), and returns torch tensors.  No arithmetic of
+the method happens in Python, and there is no CPU fallback: if the shared
+library is missing, loading fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoqe.so")
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_WORKSPACE, ERR_MISMATCH, ERR_CUDA, ERR_EXPERT_ID, ERR_TIMEOUT = range(1, 10)
+MAX_EXPERTS = 32
+PATH_AUTO, PATH_STREAM, PATH_TCGEN05 = 0, 1, 2
+
+EXPORTED = (
+    "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",
+    "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_unpermute",
+    "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_async_status",
+    "moqe_status_str", "moqe_launch_count",
+)
+
+
+class MoqeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_str(code)} (moqe_status {code})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2508_09204_b200.build` "
+                "(there is no fallback implementation)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
+        L.moqe_quantize_rtn.argtypes = [vp, i32, i32, i32, i32, i32, vp, C.POINTER(vp)]
+        L.moqe_expert_export.argtypes = [vp, vp, vp, vp, vp]
+        L.moqe_expert_import.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, C.POINTER(vp)]
+        L.moqe_expert_info.argtypes = [vp] + [C.POINTER(i32)] * 5 + [C.POINTER(sz)] * 3
+        L.moqe_expert_destroy.argtypes = [vp]
+        L.moqe_route.argtypes = [vp, i32, i32, vp, vp]
+        L.moqe_expand_ids.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.moqe_permute_workspace.argtypes = [i32, i32]
+        L.moqe_permute_workspace.restype = sz
+        L.moqe_permute.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.moqe_unpermute.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.moqe_routed_qgemm_workspace.argtypes = [i32, i32, i32, i32]
+        L.moqe_routed_qgemm_workspace.restype = sz
+        L.moqe_routed_qgemm.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp]
+        L.moqe_routed_qgemm_path.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
+        L.moqe_async_status.argtypes = [vp]
+        L.moqe_status_str.argtypes = [i32]
+        L.moqe_status_str.restype = C.c_char_p
+        L.moqe_launch_count.argtypes = []
+        L.moqe_launch_count.restype = C.c_ulonglong
+        _lib = L
+    return _lib
+
+
+def status_str(code: int) -> str:
+    return lib().moqe_status_str(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise MoqeError(code, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}")
+    return t.contiguous()
+
+
+class Expert:
+    """Owner of one ``moqe_expert*`` (destroyed with the Python object)."""
+
+    def __init__(self, handle: int):
+        self.handle = C.c_void_p(handle)
+        N, K, bits, group, sym = (C.c_int() for _ in range(5))
+        cb, mb, ab = (C.c_size_t() for _ in range(3))
+        _check(lib().moqe_expert_info(self.handle, N, K, bits, group, sym, cb, mb, ab), "moqe_expert_info")
+        self.N, self.K, self.bits, self.group, self.sym = N.value, K.value, bits.value, group.value, bool(sym.value)
+        self.code_bytes, self.meta_bytes, self.alloc_bytes = cb.value, mb.value, ab.value
+
+    @property
+    def groups_per_row(self) -> int:
+        return 1 if self.group == 0 else self.K // self.group
+
+    def close(self):
+        if self.handle is not None and self.handle.value:
+            lib().moqe_expert_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def moqe_quantize_rtn(W: torch.Tensor, bits: int, group: int, sym: bool) -> Expert:
+    """RTN-quantize the fp32 device matrix ``W[N][K]`` into a packed expert."""
+    W = _dev(W, torch.float32, "W")
+    N, K = W.shape
+    out = C.c_void_p()
+    _check(lib().moqe_quantize_rtn(_ptr(W), N, K, int(bits), int(group), int(bool(sym)), _stream(), C.byref(out)),
+           "moqe_quantize_rtn")
+    return Expert(out.value)
+
+
+def moqe_expert_export(e: Expert) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """-> (codes uint8 [N][K], scales fp16 [N][K/g], zeros fp16 [N][K/g])."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    codes = torch.empty((e.N, e.K), dtype=torch.uint8, device=dev)
+    scales = torch.empty((e.N, e.groups_per_row), dtype=torch.float16, device=dev)
+    zeros = torch.empty((e.N, e.groups_per_row), dtype=torch.float16, device=dev)
+    _check(lib().moqe_expert_export(e.handle, _ptr(codes), _ptr(scales), _ptr(zeros), _stream()), "moqe_expert_export")
+    return codes, scales, zeros
+
+
+def moqe_expert_import(bits: int, group: int, sym: bool, codes: torch.Tensor, scales: torch.Tensor,
+                       zeros: Optional[torch.Tensor]) -> Expert:
+    codes = _dev(codes, torch.uint8, "codes")
+    scales = _dev(scales, torch.float16, "scales")
+    zeros = None if zeros is None else _dev(zeros, torch.float16, "zeros")
+    N, K = codes.shape
+    out = C.c_void_p()
+    _check(lib().moqe_expert_import(N, K, int(bits), int(group), int(bool(sym)), _ptr(codes), _ptr(scales), _ptr(zeros),
+                                    _stream(), C.byref(out)), "moqe_expert_import")
+    return Expert(out.value)
+
+
+def moqe_route(logits: torch.Tensor) -> torch.Tensor:
+    """First-max arg-max over each row of fp32 ``logits[S][E]`` -> int32 ids."""
+    logits = _dev(logits, torch.float32, "logits")
+    S, E = logits.shape
+    ids = torch.empty(S, dtype=torch.int32, device=logits.device)
+    _check(lib().moqe_route(_ptr(logits), S, E, _ptr(ids), _stream()), "moqe_route")
+    return ids
+
+
+def moqe_expand_ids(ids: torch.Tensor, row_offsets: torch.Tensor, M: int) -> torch.Tensor:
+    ids = _dev(ids, torch.int32, "ids")
+    row_offsets = _dev(row_offsets, torch.int32, "row_offsets")
+    row_ids = torch.empty(M, dtype=torch.int32, device=ids.device)
+    _check(lib().moqe_expand_ids(_ptr(ids), _ptr(row_offsets), ids.numel(), int(M), _ptr(row_ids), _stream()),
+           "moqe_expand_ids")
+    return row_ids
+
+
+def moqe_permute(X: Optional[torch.Tensor], row_ids: torch.Tensor, E: int):
+    """-> (Xp or None, perm int32 [M], offsets int32 [E+1])."""
+    row_ids = _dev(row_ids, torch.int32, "row_ids")
+    M = row_ids.numel()
+    dev = row_ids.device
+    Cc = 0
+    Xp = None
+    if X is not None:
+        X = _dev(X, torch.bfloat16, "X")
+        Cc = X.shape[1]
+        Xp = torch.empty_like(X)
+    perm = torch.empty(M, dtype=torch.int32, device=dev)
+    offsets = torch.empty(E + 1, dtype=torch.int32, device=dev)
+    wsb = lib().moqe_permute_workspace(M, E)
+    ws = torch.empty(max(wsb, 1), dtype=torch.uint8, device=dev)
+    _check(lib().moqe_permute(_ptr(X), _ptr(row_ids), M, Cc, int(E), _ptr(Xp), _ptr(perm), _ptr(offsets), _ptr(ws), wsb,
+                              _stream()), "moqe_permute")
+    return Xp, perm, offsets
+
+
+def moqe_unpermute(Yp: torch.Tensor, perm: torch.Tensor) -> torch.Tensor:
+    Yp = _dev(Yp, torch.bfloat16, "Yp")
+    perm = _dev(perm, torch.int32, "perm")
+    M, Cc = Yp.shape
+    Y = torch.empty_like(Yp)
+    _check(lib().moqe_unpermute(_ptr(Yp), _ptr(perm), M, Cc, _ptr(Y), _stream()), "moqe_unpermute")
+    return Y
+
+
+def moqe_routed_qgemm_workspace(M: int, N: int, K: int, E: int) -> int:
+    return int(lib().moqe_routed_qgemm_workspace(int(M), int(N), int(K), int(E)))
+
+
+def alloc_workspace(nbytes: int, device=None) -> torch.Tensor:
+    """Device scratch of at least ``nbytes`` (256-byte aligned: torch's allocator returns 512-byte aligned blocks)."""
+    dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
+
+
+def moqe_routed_qgemm(X: torch.Tensor, row_ids: torch.Tensor, experts: Sequence[Expert],
+                      Y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      path: int = PATH_AUTO) -> torch.Tensor:
+    """``Y[m] = X[m] . dequant(W_{row_ids[m]})^T`` for bf16 ``X[M][K]`` -> bf16 ``Y[M][N]``."""
+    X = _dev(X, torch.bfloat16, "X")
+    row_ids = _dev(row_ids, torch.int32, "row_ids")
+    M, K = X.shape
+    E = len(experts)
+    if E == 0:
+        raise MoqeError(ERR_SHAPE, "moqe_routed_qgemm")
+    N = experts[0].N
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(moqe_routed_qgemm_workspace(M, N, K, E), X.device)
+    arr = (C.c_void_p * E)(*[e.handle for e in experts])
+    _check(lib().moqe_routed_qgemm_path(_ptr(X), _ptr(row_ids), M, arr, E, _ptr(Y), _ptr(workspace), workspace.numel(),
+                                        _stream(), int(path)), "moqe_routed_qgemm")
+    return Y
+
+
+def moqe_async_status() -> int:
+    """Synchronises the current stream and returns (and clears) the latched device error."""
+    return int(lib().moqe_async_status(_stream()))
+
+
+def moqe_launch_count() -> int:
+    return int(lib().moqe_launch_count())

@@ -1,0 +1,130 @@
+// C-ABI entry points that tie the kernels together: the routed dequant-GEMM
+// call, the device status word, status strings and the launch counter.
+#include <atomic>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace moqe {
+
+namespace {
+std::atomic<unsigned long long> g_launches{0};
+std::mutex g_status_mutex;
+int* g_status_words[64] = {nullptr};
+}  // namespace
+
+void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int* device_status_word() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    if (!g_status_words[dev]) {
+        int* p = nullptr;
+        if (cudaMalloc(&p, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) { cudaFree(p); return nullptr; }
+        g_status_words[dev] = p;
+    }
+    return g_status_words[dev];
+}
+
+namespace {
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+struct WsLayout {
+    size_t perm, offsets, sort, body, total;
+};
+
+WsLayout ws_layout(int M, int Np, int K, int E) {
+    WsLayout w;
+    size_t off = 0;
+    w.perm = off;    off += align256((size_t)M * sizeof(int32_t) + 16);
+    w.offsets = off; off += align256((MOQE_MAX_EXPERTS + 2) * sizeof(int32_t));
+    w.sort = off;    off += align256(sort_workspace_bytes(M, E));
+    w.body = off;
+    size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np);
+    off += align256(a > b ? a : b);
+    w.total = off;
+    return w;
+}
+
+constexpr int AUTO_STREAM_MAX_ROWS = 128;
+
+}  // namespace
+}  // namespace moqe
+
+using namespace moqe;
+
+extern "C" size_t moqe_routed_qgemm_workspace(int M, int N, int K, int E) {
+    if (M < 0 || N <= 0 || K <= 0 || E <= 0) return 0;
+    int Np = (N + 127) / 128 * 128;
+    return ws_layout(M, Np, K, E).total;
+}
+
+extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
+                                              const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
+                                              size_t workspace_bytes, void* stream, int path) {
+    if (!h_experts) return MOQE_ERR_NULL;
+    if (E <= 0 || M < 0) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    for (int e = 0; e < E; ++e)
+        if (!h_experts[e]) return MOQE_ERR_NULL;
+    const int N = h_experts[0]->N, K = h_experts[0]->K;
+    for (int e = 1; e < E; ++e)
+        if (h_experts[e]->N != N || h_experts[e]->K != K) return MOQE_ERR_MISMATCH;
+    if (M == 0) return MOQE_OK;
+    if (!X_bf16 || !row_ids || !Y_bf16) return MOQE_ERR_NULL;
+    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
+    if (path < 0 || path > 2) return MOQE_ERR_SHAPE;
+    const int Np = h_experts[0]->Np;
+    WsLayout w = ws_layout(M, Np, K, E);
+    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)workspace;
+    int32_t* perm = (int32_t*)(base + w.perm);
+    int32_t* offsets = (int32_t*)(base + w.offsets);
+    const bool use_stream = path == 1 || (path == 0 && M <= AUTO_STREAM_MAX_ROWS);
+    size_t zero_bytes = use_stream ? stream_zero_bytes(M, Np) : 0;
+    moqe_status s = launch_sort(row_ids, M, E, perm, offsets, base + w.sort, w.body - w.sort, base + w.body, zero_bytes,
+                                Y_bf16, N, st);
+    if (s != MOQE_OK) return s;
+    if (use_stream)
+        return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
+                                   w.total - w.body, st);
+    return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+}
+
+extern "C" moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_ids, int M,
+                                         const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+    return moqe_routed_qgemm_path(X_bf16, row_ids, M, h_experts, E, Y_bf16, workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" moqe_status moqe_async_status(void* stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MOQE_ERR_CUDA;
+    int* w = device_status_word();
+    if (!w) return MOQE_ERR_ALLOC;
+    int v = 0;
+    if (cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MOQE_ERR_CUDA;
+    if (v != 0 && cudaMemset(w, 0, sizeof(int)) != cudaSuccess) return MOQE_ERR_CUDA;
+    return (moqe_status)v;
+}
+
+extern "C" const char* moqe_status_str(moqe_status s) {
+    switch (s) {
+        case MOQE_OK: return "ok";
+        case MOQE_ERR_NULL: return "a required pointer is NULL";
+        case MOQE_ERR_SHAPE: return "bad or inconsistent size";
+        case MOQE_ERR_UNSUPPORTED: return "unsupported format, size or alignment";
+        case MOQE_ERR_ALLOC: return "device allocation failed";
+        case MOQE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case MOQE_ERR_MISMATCH: return "experts disagree on N or K";
+        case MOQE_ERR_CUDA: return "a CUDA call failed";
+        case MOQE_ERR_EXPERT_ID: return "an expert id outside [0,E) was seen on the device";
+        case MOQE_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
+    }
+    return "unknown status";
+}
+
+extern "C" unsigned long long moqe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

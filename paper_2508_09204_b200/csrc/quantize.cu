@@ -1,0 +1,420 @@
+// Expert construction: RTN quantizer, packer, canonical import / export.
+//
+// Section 3.1 of the paper: the experts are quantized variants of one
+// full-precision model, built once and frozen.  The quantizer is affine
+// round-to-nearest per (output channel, group of input features); see moqe.h
+// for the exact arithmetic.  Every fp32 operation below is a single IEEE
+// operation (explicit __f*_rn intrinsics, no fused multiply-add, no fast
+// math), so codes, scales and zero-points are reproducible bit for bit.
+#include <new>
+
+#include "common.cuh"
+
+namespace moqe {
+namespace {
+
+// ---------------------------------------------------------------------------
+// piece <-> packed words
+// ---------------------------------------------------------------------------
+// code index i = 8*G + t  (chunk G, position t)  <->  k = 128*kb + 32*G + 8*q + t
+template <int BITS>
+struct PieceWords;   // number of 32-bit words per piece
+template <> struct PieceWords<4> { static constexpr int n = 4; };
+template <> struct PieceWords<8> { static constexpr int n = 8; };
+template <> struct PieceWords<3> { static constexpr int n = 3; };
+
+template <int BITS>
+__device__ __forceinline__ void encode_piece(const uint32_t (&c)[32], uint32_t (&w)[PieceWords<BITS>::n]) {
+    if constexpr (BITS == 4) {
+#pragma unroll
+        for (int G = 0; G < 4; ++G) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                int nib = (t & 1) ? 4 + (t >> 1) : (t >> 1);
+                v |= (c[8 * G + t] & 0xFu) << (4 * nib);
+            }
+            w[G] = v;
+        }
+    } else if constexpr (BITS == 8) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            w[j] = (c[4 * j] & 0xFFu) | ((c[4 * j + 1] & 0xFFu) << 8) | ((c[4 * j + 2] & 0xFFu) << 16) |
+                   ((c[4 * j + 3] & 0xFFu) << 24);
+    } else {
+        w[0] = w[1] = w[2] = 0;
+#pragma unroll
+        for (int i = 0; i < 30; ++i) {
+            int p = i >> 1;
+            w[p / 5] |= (c[i] & 7u) << (3 * (p % 5) + 16 * (i & 1));
+        }
+#pragma unroll
+        for (int b = 0; b < 3; ++b) {
+            w[b] |= ((c[30] >> b) & 1u) << 15;
+            w[b] |= ((c[31] >> b) & 1u) << 31;
+        }
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void decode_piece(const uint32_t (&w)[PieceWords<BITS>::n], uint32_t (&c)[32]) {
+    if constexpr (BITS == 4) {
+#pragma unroll
+        for (int G = 0; G < 4; ++G)
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                int nib = (t & 1) ? 4 + (t >> 1) : (t >> 1);
+                c[8 * G + t] = (w[G] >> (4 * nib)) & 0xFu;
+            }
+    } else if constexpr (BITS == 8) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) c[i] = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 30; ++i) {
+            int p = i >> 1;
+            c[i] = (w[p / 5] >> (3 * (p % 5) + 16 * (i & 1))) & 7u;
+        }
+        c[30] = c[31] = 0;
+#pragma unroll
+        for (int b = 0; b < 3; ++b) {
+            c[30] |= ((w[b] >> 15) & 1u) << b;
+            c[31] |= ((w[b] >> 31) & 1u) << b;
+        }
+    }
+}
+
+// address of the words of piece (half, slot) inside a blob
+template <int BITS>
+__device__ __forceinline__ void store_piece(uint8_t* blob, int half, int slot, const uint32_t (&w)[PieceWords<BITS>::n]) {
+    if constexpr (BITS == 4) {
+        *reinterpret_cast<uint4*>(blob + half * 512 + slot * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else if constexpr (BITS == 8) {
+        *reinterpret_cast<uint4*>(blob + half * 1024 + slot * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(blob + half * 1024 + 512 + slot * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+    } else {
+        uint32_t* a = reinterpret_cast<uint32_t*>(blob + slot * 16);
+        uint32_t* b = reinterpret_cast<uint32_t*>(blob + 512 + slot * 8);
+        if (half == 0) { a[0] = w[0]; a[1] = w[1]; a[2] = w[2]; }
+        else           { a[3] = w[0]; b[0] = w[1]; b[1] = w[2]; }
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void load_piece(const uint8_t* blob, int half, int slot, uint32_t (&w)[PieceWords<BITS>::n]) {
+    if constexpr (BITS == 4) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if constexpr (BITS == 8) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 1024 + slot * 16);
+        uint4 u = *reinterpret_cast<const uint4*>(blob + half * 1024 + 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; w[4] = u.x; w[5] = u.y; w[6] = u.z; w[7] = u.w;
+    } else {
+        const uint32_t* a = reinterpret_cast<const uint32_t*>(blob + slot * 16);
+        const uint32_t* b = reinterpret_cast<const uint32_t*>(blob + 512 + slot * 8);
+        if (half == 0) { w[0] = a[0]; w[1] = a[1]; w[2] = a[2]; }
+        else           { w[0] = a[3]; w[1] = b[0]; w[2] = b[1]; }
+    }
+}
+
+// piece id -> coordinates.  Pieces are numbered so that consecutive threads own
+// consecutive slots of one half of one blob (coalesced packed accesses).
+struct PieceCoord { int nt, kb, nb, half, slot, q, r, n; size_t blob_index; };
+__device__ __forceinline__ PieceCoord piece_coord(long long pid, int KB) {
+    PieceCoord pc;
+    pc.slot = (int)(pid & 31);
+    pc.half = (int)((pid >> 5) & 1);
+    pc.nb = (int)((pid >> 6) & 7);
+    long long tile = pid >> 9;
+    pc.kb = (int)(tile % KB);
+    pc.nt = (int)(tile / KB);
+    pc.q = pc.slot >> 3;
+    pc.r = pc.slot & 7;
+    pc.n = pc.nt * 128 + pc.nb * 16 + pc.half * 8 + pc.r;
+    pc.blob_index = (size_t)tile * 8 + pc.nb;
+    return pc;
+}
+
+// ---------------------------------------------------------------------------
+// K1a: per (channel, group) scale and zero-point.  One warp per group.
+// ---------------------------------------------------------------------------
+__global__ void rtn_scales_kernel(const float* __restrict__ W, int N, int K, int bits, int g, int G, int sym, int Np,
+                                  __half* __restrict__ scales_t, __nv_bfloat16* __restrict__ zeros_t) {
+    long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (warp >= (long long)N * G) return;
+    int n = (int)(warp / G), gi = (int)(warp % G);
+    const float* w = W + (size_t)n * K + (size_t)gi * g;
+    float lo = 0.f, hi = 0.f, a = 0.f;
+    for (int k = lane; k < g; k += 32) {
+        float v = w[k];
+        lo = fminf(lo, v);
+        hi = fmaxf(hi, v);
+        a = fmaxf(a, fabsf(v));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+    }
+    if (lane != 0) return;
+    const int L = (1 << bits) - 1;
+    const int qmax = (1 << (bits - 1)) - 1;
+    float s32 = sym ? __fdiv_rn(a, (float)qmax) : __fdiv_rn(__fsub_rn(hi, lo), (float)L);
+    __half sh = __float2half_rn(s32);
+    float s = __half2float(sh);
+    if (!(s > 0.f) || isinf(s)) { sh = __float2half_rn(1.0f); s = 1.0f; }
+    scales_t[(size_t)gi * Np + n] = sh;
+    if (!sym) {
+        int z = (int)rintf(__fdiv_rn(-lo, s));
+        z = max(0, min(L, z));
+        zeros_t[(size_t)gi * Np + n] = __float2bfloat16_rn((float)z);   // exact: z <= 255
+    }
+}
+
+// ---------------------------------------------------------------------------
+// K1b: codes + packing (FROM_CODES: canonical codes are given, only pack)
+// ---------------------------------------------------------------------------
+template <int BITS, bool FROM_CODES>
+__global__ void encode_pack_kernel(const float* __restrict__ W, const uint8_t* __restrict__ canon, int N, int K,
+                                   int g /*0 = per channel*/, int sym, int Np, int KB,
+                                   const __half* __restrict__ scales_t, const __nv_bfloat16* __restrict__ zeros_t,
+                                   uint8_t* __restrict__ packed, long long npieces) {
+    long long pid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pid >= npieces) return;
+    PieceCoord pc = piece_coord(pid, KB);
+    constexpr int L = (1 << BITS) - 1;
+    constexpr int half_code = 1 << (BITS - 1);
+    constexpr int qmax = half_code - 1;
+    uint32_t c[32];
+#pragma unroll
+    for (int G = 0; G < 4; ++G) {
+        int k0 = pc.kb * 128 + 32 * G + 8 * pc.q;
+        bool live = (pc.n < N) && (k0 < K);            // K % 8 == 0: a chunk is wholly inside or outside
+        if (!live) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t) c[8 * G + t] = 0;
+            continue;
+        }
+        if constexpr (FROM_CODES) {
+            uint2 v = *reinterpret_cast<const uint2*>(canon + (size_t)pc.n * K + k0);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                c[8 * G + t] = (v.x >> (8 * t)) & 0xFFu;
+                c[8 * G + 4 + t] = (v.y >> (8 * t)) & 0xFFu;
+            }
+        } else {
+            int gi = g ? k0 / g : 0;
+            float s = __half2float(scales_t[(size_t)gi * Np + pc.n]);
+            int z = sym ? half_code : (int)__bfloat162float(zeros_t[(size_t)gi * Np + pc.n]);
+            const float4* src = reinterpret_cast<const float4*>(W + (size_t)pc.n * K + k0);
+            float4 v0 = src[0], v1 = src[1];
+            float wv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                int q = (int)rintf(__fdiv_rn(wv[t], s));
+                if (sym) q = max(-qmax, min(qmax, q)) + half_code;
+                else     q = max(0, min(L, q + z));
+                c[8 * G + t] = (uint32_t)q;
+            }
+        }
+    }
+    uint32_t w[PieceWords<BITS>::n];
+    encode_piece<BITS>(c, w);
+    store_piece<BITS>(packed + pc.blob_index * (size_t)moqe_blob_bytes(BITS), pc.half, pc.slot, w);
+}
+
+template <int BITS>
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, int N, int K, int KB, uint8_t* __restrict__ canon,
+                              long long npieces) {
+    long long pid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pid >= npieces) return;
+    PieceCoord pc = piece_coord(pid, KB);
+    if (pc.n >= N) return;
+    uint32_t w[PieceWords<BITS>::n];
+    load_piece<BITS>(packed + pc.blob_index * (size_t)moqe_blob_bytes(BITS), pc.half, pc.slot, w);
+    uint32_t c[32];
+    decode_piece<BITS>(w, c);
+#pragma unroll
+    for (int G = 0; G < 4; ++G) {
+        int k0 = pc.kb * 128 + 32 * G + 8 * pc.q;
+        if (k0 >= K) continue;
+        uint2 v;
+        v.x = c[8 * G] | (c[8 * G + 1] << 8) | (c[8 * G + 2] << 16) | (c[8 * G + 3] << 24);
+        v.y = c[8 * G + 4] | (c[8 * G + 5] << 8) | (c[8 * G + 6] << 16) | (c[8 * G + 7] << 24);
+        *reinterpret_cast<uint2*>(canon + (size_t)pc.n * K + k0) = v;
+    }
+}
+
+// canonical [N][G] fp16 scales / zero-points  <->  transposed padded device arrays
+__global__ void meta_export_kernel(const __half* __restrict__ scales_t, const __nv_bfloat16* __restrict__ zeros_t, int N,
+                                   int G, int Np, int bits, uint16_t* __restrict__ scales_out,
+                                   uint16_t* __restrict__ zeros_out) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)N * G) return;
+    int n = (int)(i / G), gi = (int)(i % G);
+    if (scales_out) scales_out[i] = __half_as_ushort(scales_t[(size_t)gi * Np + n]);
+    if (zeros_out) {
+        float z = zeros_t ? __bfloat162float(zeros_t[(size_t)gi * Np + n]) : (float)(1 << (bits - 1));
+        zeros_out[i] = __half_as_ushort(__float2half_rn(z));
+    }
+}
+
+__global__ void meta_import_kernel(const uint16_t* __restrict__ scales_in, const uint16_t* __restrict__ zeros_in, int N,
+                                   int G, int Np, __half* __restrict__ scales_t, __nv_bfloat16* __restrict__ zeros_t) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)N * G) return;
+    int n = (int)(i / G), gi = (int)(i % G);
+    scales_t[(size_t)gi * Np + n] = __ushort_as_half(scales_in[i]);
+    if (zeros_t) zeros_t[(size_t)gi * Np + n] = __float2bfloat16_rn(__half2float(__ushort_as_half(zeros_in[i])));
+}
+
+moqe_status check_format(int N, int K, int bits, int group) {
+    if (N <= 0 || K <= 0) return MOQE_ERR_SHAPE;
+    if (bits != 3 && bits != 4 && bits != 8) return MOQE_ERR_UNSUPPORTED;
+    if (K % 8 != 0) return MOQE_ERR_UNSUPPORTED;
+    if (group < 0) return MOQE_ERR_SHAPE;
+    if (group != 0) {
+        if (K % group != 0) return MOQE_ERR_SHAPE;
+        if (!(group == 32 || group == 64 || group % 128 == 0)) return MOQE_ERR_UNSUPPORTED;
+    }
+    return MOQE_OK;
+}
+
+moqe_status alloc_expert(int N, int K, int bits, int group, int sym, cudaStream_t st, moqe_expert** out) {
+    moqe_expert* e = new (std::nothrow) moqe_expert();
+    if (!e) return MOQE_ERR_ALLOC;
+    e->N = N; e->K = K; e->bits = bits; e->group = group; e->sym = sym ? 1 : 0;
+    e->Np = (N + 127) / 128 * 128;
+    e->Kp = (K + 127) / 128 * 128;
+    e->G = group ? K / group : 1;
+    e->Gp = group ? e->Kp / group : 1;
+    e->codes = nullptr; e->scales_t = nullptr; e->zeros_t = nullptr;
+    if (cudaGetDevice(&e->device) != cudaSuccess) { delete e; return MOQE_ERR_CUDA; }
+    e->codes_alloc = (size_t)e->Np * e->Kp * bits / 8;
+    e->meta_alloc = (size_t)e->Gp * e->Np * 2;
+    bool ok = cudaMalloc(&e->codes, e->codes_alloc) == cudaSuccess &&
+              cudaMalloc(&e->scales_t, e->meta_alloc) == cudaSuccess &&
+              (e->sym || cudaMalloc(&e->zeros_t, e->meta_alloc) == cudaSuccess);
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(e->codes); cudaFree(e->scales_t); cudaFree(e->zeros_t);
+        delete e;
+        return MOQE_ERR_ALLOC;
+    }
+    cudaMemsetAsync(e->scales_t, 0, e->meta_alloc, st);
+    if (e->zeros_t) cudaMemsetAsync(e->zeros_t, 0, e->meta_alloc, st);
+    *out = e;
+    return MOQE_OK;
+}
+
+template <bool FROM_CODES>
+moqe_status launch_encode(const moqe_expert* e, const float* W, const uint8_t* canon, cudaStream_t st) {
+    int KB = e->Kp / 128;
+    long long npieces = (long long)(e->Np / 128) * KB * 512;
+    unsigned blocks = (unsigned)((npieces + 127) / 128);
+#define MOQE_ENC(B)                                                                                                  \
+    encode_pack_kernel<B, FROM_CODES><<<blocks, 128, 0, st>>>(W, canon, e->N, e->K, e->group, e->sym, e->Np, KB,      \
+                                                              e->scales_t, e->zeros_t, e->codes, npieces)
+    if (e->bits == 4) MOQE_ENC(4);
+    else if (e->bits == 8) MOQE_ENC(8);
+    else MOQE_ENC(3);
+#undef MOQE_ENC
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace
+}  // namespace moqe
+
+using namespace moqe;
+
+extern "C" moqe_status moqe_quantize_rtn(const float* W, int N, int K, int bits, int group, int sym, void* stream,
+                                         moqe_expert** out) {
+    if (!W || !out) return MOQE_ERR_NULL;
+    moqe_status s = check_format(N, K, bits, group);
+    if (s != MOQE_OK) return s;
+    if (reinterpret_cast<uintptr_t>(W) % 16 != 0) return MOQE_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    moqe_expert* e = nullptr;
+    s = alloc_expert(N, K, bits, group, sym, st, &e);
+    if (s != MOQE_OK) return s;
+    int g = group ? group : K;
+    long long warps = (long long)N * e->G;
+    unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
+    rtn_scales_kernel<<<blocks, 256, 0, st>>>(W, N, K, bits, g, e->G, e->sym, e->Np, e->scales_t, e->zeros_t);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) { moqe_expert_destroy(e); return MOQE_ERR_CUDA; }
+    s = launch_encode<false>(e, W, nullptr, st);
+    if (s != MOQE_OK) { moqe_expert_destroy(e); return s; }
+    *out = e;
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_import(int N, int K, int bits, int group, int sym, const uint8_t* codes,
+                                          const uint16_t* scales_f16, const uint16_t* zeros_f16, void* stream,
+                                          moqe_expert** out) {
+    if (!codes || !scales_f16 || !out) return MOQE_ERR_NULL;
+    if (!sym && !zeros_f16) return MOQE_ERR_NULL;
+    moqe_status s = check_format(N, K, bits, group);
+    if (s != MOQE_OK) return s;
+    if (reinterpret_cast<uintptr_t>(codes) % 8 != 0) return MOQE_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    moqe_expert* e = nullptr;
+    s = alloc_expert(N, K, bits, group, sym, st, &e);
+    if (s != MOQE_OK) return s;
+    long long n = (long long)N * e->G;
+    meta_import_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(scales_f16, zeros_f16, N, e->G, e->Np, e->scales_t,
+                                                                    e->zeros_t);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) { moqe_expert_destroy(e); return MOQE_ERR_CUDA; }
+    s = launch_encode<true>(e, nullptr, codes, st);
+    if (s != MOQE_OK) { moqe_expert_destroy(e); return s; }
+    *out = e;
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_export(const moqe_expert* e, uint8_t* codes, uint16_t* scales_f16,
+                                          uint16_t* zeros_f16, void* stream) {
+    if (!e) return MOQE_ERR_NULL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (codes) {
+        if (reinterpret_cast<uintptr_t>(codes) % 8 != 0) return MOQE_ERR_UNSUPPORTED;
+        int KB = e->Kp / 128;
+        long long npieces = (long long)(e->Np / 128) * KB * 512;
+        unsigned blocks = (unsigned)((npieces + 127) / 128);
+        if (e->bits == 4) unpack_kernel<4><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
+        else if (e->bits == 8) unpack_kernel<8><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
+        else unpack_kernel<3><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
+        count_launch();
+    }
+    if (scales_f16 || zeros_f16) {
+        long long n = (long long)e->N * e->G;
+        meta_export_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e->scales_t, e->zeros_t, e->N, e->G, e->Np,
+                                                                        e->bits, scales_f16, zeros_f16);
+        count_launch();
+    }
+    return cuda_ok(cudaGetLastError());
+}
+
+extern "C" moqe_status moqe_expert_info(const moqe_expert* e, int* N, int* K, int* bits, int* group, int* sym,
+                                        size_t* code_bytes, size_t* meta_bytes, size_t* alloc_bytes) {
+    if (!e) return MOQE_ERR_NULL;
+    if (N) *N = e->N;
+    if (K) *K = e->K;
+    if (bits) *bits = e->bits;
+    if (group) *group = e->group;
+    if (sym) *sym = e->sym;
+    if (code_bytes) *code_bytes = (size_t)e->N * e->K * e->bits / 8;
+    if (meta_bytes) *meta_bytes = (size_t)e->N * e->G * 2 * (e->sym ? 1 : 2);
+    if (alloc_bytes) *alloc_bytes = e->codes_alloc + e->meta_alloc * (e->sym ? 1 : 2);
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_destroy(moqe_expert* e) {
+    if (!e) return MOQE_ERR_NULL;
+    cudaError_t a = cudaFree(e->codes), b = cudaFree(e->scales_t), c = cudaFree(e->zeros_t);
+    delete e;
+    return (a == cudaSuccess && b == cudaSuccess && c == cudaSuccess) ? MOQE_OK : MOQE_ERR_CUDA;
+}

@@ -1,0 +1,278 @@
+// Hard routing (arg-max), stable counting sort of rows by expert id, and the
+// row gather / scatter around the grouped GEMM.
+//
+// Section 3.2 / Appendix of the paper: the router's decision is one expert
+// index per sample.  The sort is the batching glue that turns "one expert per
+// sample" into contiguous per-expert row segments; its per-expert counts are
+// the n_i of the load statistic F_i = n_i / B (Section 3.3).
+//
+// Sort: bucket = id for valid ids, bucket E for ids outside [0,E) (those rows
+// end up behind all valid rows and latch MOQE_ERR_EXPERT_ID).  Within a warp
+// the stable rank of a row among equal ids comes from __match_any_sync; warps
+// and blocks are combined with prefix sums, so perm is the unique stable order.
+#include "common.cuh"
+
+namespace moqe {
+namespace {
+
+constexpr int SORT_THREADS = 1024;
+constexpr int SORT_WARPS = SORT_THREADS / 32;
+constexpr int MAXB = MOQE_MAX_EXPERTS + 1;   // buckets incl. the invalid-id bucket
+
+__global__ void route_kernel(const float* __restrict__ logits, int S, int E, int32_t* __restrict__ ids) {
+    int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    const float* l = logits + (size_t)s * E;
+    int best = -1;
+    float bv = 0.f;
+    for (int e = 0; e < E; ++e) {
+        float v = l[e];
+        if (v != v) continue;                       // NaN never wins
+        if (best < 0 || v > bv) { best = e; bv = v; }
+    }
+    ids[s] = best < 0 ? 0 : best;
+}
+
+__global__ void expand_ids_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ row_offsets, int S, int M,
+                                  int32_t* __restrict__ row_ids) {
+    int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    // largest s with row_offsets[s] <= m  (row_offsets is non-decreasing, row_offsets[0] = 0)
+    int lo = 0, hi = S;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (row_offsets[mid] <= m) lo = mid; else hi = mid;
+    }
+    row_ids[m] = ids[lo];
+}
+
+// Per-block pieces of the sort --------------------------------------------------
+// Stable rank of each of this block's rows inside the block, and per-bucket block
+// totals.  Row m = base + threadIdx.x.  On return (after the trailing barrier)
+// s_warp[w][b] = number of rows of bucket b in warps < w of this block, and
+// s_tot[b] = rows of bucket b in the block.
+struct BlockRank { int bucket; int rank; bool live; };
+
+__device__ __forceinline__ BlockRank block_rank(const int32_t* __restrict__ row_ids, int M, int E, long long base,
+                                                int (*s_warp)[MAXB], int* s_tot, int* status) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    long long m = base + threadIdx.x;
+    BlockRank br;
+    br.live = m < M;
+    int id = br.live ? row_ids[m] : 0;
+    bool bad = br.live && (id < 0 || id >= E);
+    if (bad) latch_status(status, (int)MOQE_ERR_EXPERT_ID);
+    br.bucket = bad ? E : id;
+    for (int i = threadIdx.x; i < SORT_WARPS * MAXB; i += blockDim.x) (&s_warp[0][0])[i] = 0;
+    __syncthreads();
+    unsigned live_mask = __ballot_sync(0xffffffffu, br.live);
+    int rank_in_warp = 0;
+    if (br.live) {
+        unsigned peers = __match_any_sync(live_mask, br.bucket);
+        rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+        if (rank_in_warp == 0) s_warp[warp][br.bucket] = __popc(peers);
+    }
+    __syncthreads();
+    if (threadIdx.x <= E) {                         // exclusive scan over warps, one thread per bucket
+        int run = 0;
+        for (int w = 0; w < SORT_WARPS; ++w) { int c = s_warp[w][threadIdx.x]; s_warp[w][threadIdx.x] = run; run += c; }
+        s_tot[threadIdx.x] = run;
+    }
+    __syncthreads();
+    br.rank = rank_in_warp + (br.live ? s_warp[warp][br.bucket] : 0);
+    return br;
+}
+
+__device__ __forceinline__ void zero_row(void* Y, int N, long long row) {
+    // one thread zeroes a whole row: only rows with an invalid id take this path
+    uint4* y = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(Y) + (size_t)row * N);
+    for (int i = 0; i < N / 8; ++i) y[i] = make_uint4(0, 0, 0, 0);
+}
+
+// M <= 1024: the whole sort in one block; also clears `zero_region` (split-K arrival counters).
+__global__ void __launch_bounds__(SORT_THREADS) sort_small_kernel(const int32_t* __restrict__ row_ids, int M, int E,
+                                                                  int32_t* __restrict__ perm, int32_t* __restrict__ offsets,
+                                                                  uint32_t* __restrict__ zero_region, size_t zero_words,
+                                                                  void* Y, int N, int* status) {
+    __shared__ int s_warp[SORT_WARPS][MAXB];
+    __shared__ int s_tot[MAXB];
+    __shared__ int s_off[MAXB + 1];
+    for (size_t i = threadIdx.x; i < zero_words; i += blockDim.x) zero_region[i] = 0u;
+    BlockRank br = block_rank(row_ids, M, E, 0, s_warp, s_tot, status);
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int b = 0; b <= E; ++b) { s_off[b] = run; run += s_tot[b]; }
+        s_off[E + 1] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x <= E) offsets[threadIdx.x] = s_off[threadIdx.x];
+    if (br.live) {
+        perm[s_off[br.bucket] + br.rank] = threadIdx.x;
+        if (br.bucket == E && Y) zero_row(Y, N, threadIdx.x);
+    }
+}
+
+// M > 1024: three kernels.  (1) per-block bucket totals
+__global__ void __launch_bounds__(SORT_THREADS) sort_hist_kernel(const int32_t* __restrict__ row_ids, int M, int E,
+                                                                 int32_t* __restrict__ block_tot, int* status) {
+    __shared__ int s_warp[SORT_WARPS][MAXB];
+    __shared__ int s_tot[MAXB];
+    block_rank(row_ids, M, E, (long long)blockIdx.x * SORT_THREADS, s_warp, s_tot, status);
+    if (threadIdx.x <= E) block_tot[(size_t)blockIdx.x * MAXB + threadIdx.x] = s_tot[threadIdx.x];
+}
+
+// (2) exclusive scan in (bucket-major, block-minor) order; block_tot becomes the base slot of (block, bucket)
+__global__ void sort_scan_kernel(int32_t* __restrict__ block_tot, int nblk, int E, int32_t* __restrict__ offsets) {
+    __shared__ int s_sum[MAXB];
+    __shared__ int s_off[MAXB + 1];
+    int b = threadIdx.x;
+    if (b <= E) {
+        int run = 0;
+        for (int i = 0; i < nblk; ++i) { int c = block_tot[(size_t)i * MAXB + b]; block_tot[(size_t)i * MAXB + b] = run; run += c; }
+        s_sum[b] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int i = 0; i <= E; ++i) { s_off[i] = run; run += s_sum[i]; }
+    }
+    __syncthreads();
+    if (b <= E) {
+        offsets[b] = s_off[b];
+        for (int i = 0; i < nblk; ++i) block_tot[(size_t)i * MAXB + b] += s_off[b];
+    }
+}
+
+// (3) scatter row indices to their slots
+__global__ void __launch_bounds__(SORT_THREADS) sort_scatter_kernel(const int32_t* __restrict__ row_ids, int M, int E,
+                                                                    const int32_t* __restrict__ block_base,
+                                                                    int32_t* __restrict__ perm, void* Y, int N) {
+    __shared__ int s_warp[SORT_WARPS][MAXB];
+    __shared__ int s_tot[MAXB];
+    long long base = (long long)blockIdx.x * SORT_THREADS;
+    BlockRank br = block_rank(row_ids, M, E, base, s_warp, s_tot, nullptr);
+    if (br.live) {
+        long long m = base + threadIdx.x;
+        perm[block_base[(size_t)blockIdx.x * MAXB + br.bucket] + br.rank] = (int32_t)m;
+        if (br.bucket == E && Y) zero_row(Y, N, m);
+    }
+}
+
+// Row gather / scatter: 16 bytes per thread, a row is covered by consecutive threads.
+// GATHER : dst[j] = src[perm[j]]   (rows j >= n_valid, i.e. invalid ids, are zero-filled)
+// SCATTER: dst[perm[j]] = src[j]
+template <bool GATHER>
+__global__ void move_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ perm,
+                                 const int32_t* __restrict__ n_valid_ptr, long long M, int vec_per_row,
+                                 uint4* __restrict__ dst) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * vec_per_row) return;
+    long long j = i / vec_per_row;
+    int v = (int)(i % vec_per_row);
+    long long p = perm[j];
+    if (GATHER) {
+        bool valid = !n_valid_ptr || j < *n_valid_ptr;
+        dst[j * vec_per_row + v] = valid ? src[p * vec_per_row + v] : make_uint4(0, 0, 0, 0);
+    } else {
+        dst[p * vec_per_row + v] = src[j * vec_per_row + v];
+    }
+}
+
+}  // namespace
+
+size_t sort_workspace_bytes(int M, int E) {
+    (void)E;
+    if (M <= SORT_THREADS) return 256;
+    size_t nblk = ((size_t)M + SORT_THREADS - 1) / SORT_THREADS;
+    return (nblk * MAXB * sizeof(int32_t) + 255) / 256 * 256;
+}
+
+// Sort rows by id.  zero_region (optional, 4-byte multiple) is cleared on the way;
+// Y (optional) gets zero rows where the id is invalid.
+moqe_status launch_sort(const int32_t* row_ids, int M, int E, int32_t* perm, int32_t* offsets, void* ws, size_t ws_bytes,
+                        void* zero_region, size_t zero_bytes, void* Y_zero_invalid, int N, cudaStream_t st) {
+    int* status = device_status_word();
+    if (!status) return MOQE_ERR_ALLOC;
+    if (M <= SORT_THREADS) {
+        sort_small_kernel<<<1, SORT_THREADS, 0, st>>>(row_ids, M, E, perm, offsets, (uint32_t*)zero_region,
+                                                      zero_bytes / 4, Y_zero_invalid, N, status);
+        count_launch();
+        return cuda_ok(cudaGetLastError());
+    }
+    if (!ws || ws_bytes < sort_workspace_bytes(M, E)) return MOQE_ERR_WORKSPACE;
+    if (zero_region && zero_bytes) {
+        if (cudaMemsetAsync(zero_region, 0, zero_bytes, st) != cudaSuccess) return MOQE_ERR_CUDA;
+    }
+    int nblk = (M + SORT_THREADS - 1) / SORT_THREADS;
+    int32_t* block_tot = (int32_t*)ws;
+    sort_hist_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, block_tot, status);
+    sort_scan_kernel<<<1, 64, 0, st>>>(block_tot, nblk, E, offsets);
+    sort_scatter_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, block_tot, perm, Y_zero_invalid, N);
+    count_launch(3);
+    return cuda_ok(cudaGetLastError());
+}
+
+moqe_status launch_gather(const void* X, const int32_t* perm, const int32_t* n_valid_ptr, int M, int C, void* Xp,
+                          cudaStream_t st) {
+    if (M == 0) return MOQE_OK;
+    int vec = C / 8;
+    long long total = (long long)M * vec;
+    move_rows_kernel<true><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint4*)X, perm, n_valid_ptr, M, vec,
+                                                                           (uint4*)Xp);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace moqe
+
+using namespace moqe;
+
+extern "C" moqe_status moqe_route(const float* logits, int S, int E, int32_t* ids, void* stream) {
+    if (!logits || !ids) return MOQE_ERR_NULL;
+    if (S < 0 || E <= 0) return MOQE_ERR_SHAPE;
+    if (S == 0) return MOQE_OK;
+    route_kernel<<<(S + 255) / 256, 256, 0, (cudaStream_t)stream>>>(logits, S, E, ids);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+extern "C" moqe_status moqe_expand_ids(const int32_t* ids, const int32_t* row_offsets, int S, int M, int32_t* row_ids,
+                                       void* stream) {
+    if (!ids || !row_offsets || !row_ids) return MOQE_ERR_NULL;
+    if (S < 0 || M < 0 || (S == 0 && M != 0)) return MOQE_ERR_SHAPE;
+    if (M == 0) return MOQE_OK;
+    expand_ids_kernel<<<(M + 255) / 256, 256, 0, (cudaStream_t)stream>>>(ids, row_offsets, S, M, row_ids);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+extern "C" size_t moqe_permute_workspace(int M, int E) { return sort_workspace_bytes(M < 0 ? 0 : M, E); }
+
+extern "C" moqe_status moqe_permute(const void* X_bf16, const int32_t* row_ids, int M, int C, int E, void* Xp_bf16,
+                                    int32_t* perm, int32_t* offsets, void* workspace, size_t workspace_bytes,
+                                    void* stream) {
+    if (!row_ids || !perm || !offsets) return MOQE_ERR_NULL;
+    if ((X_bf16 == nullptr) != (Xp_bf16 == nullptr)) return MOQE_ERR_NULL;
+    if (M < 0 || E <= 0 || (X_bf16 && C <= 0)) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    if (X_bf16 && (C % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Xp_bf16 % 16)) return MOQE_ERR_UNSUPPORTED;
+    if (M > SORT_THREADS && (!workspace || workspace_bytes < sort_workspace_bytes(M, E))) return MOQE_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    moqe_status s = launch_sort(row_ids, M, E, perm, offsets, workspace, workspace_bytes, nullptr, 0, nullptr, 0, st);
+    if (s != MOQE_OK || !X_bf16) return s;
+    return launch_gather(X_bf16, perm, offsets + E, M, C, Xp_bf16, st);
+}
+
+extern "C" moqe_status moqe_unpermute(const void* Yp_bf16, const int32_t* perm, int M, int C, void* Y_bf16,
+                                      void* stream) {
+    if (!Yp_bf16 || !perm || !Y_bf16) return MOQE_ERR_NULL;
+    if (M < 0 || C <= 0) return MOQE_ERR_SHAPE;
+    if (C % 8 != 0 || (uintptr_t)Yp_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
+    if (M == 0) return MOQE_OK;
+    int vec = C / 8;
+    long long total = (long long)M * vec;
+    move_rows_kernel<false><<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+        (const uint4*)Yp_bf16, perm, nullptr, M, vec, (uint4*)Y_bf16);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}

@@ -1,0 +1,143 @@
+"""GPU parity: the routed dequant-GEMM against the oracle, element by element, on seeded inputs.
+
+Tolerance (stated by the target: bf16 output, fp32 accumulation): max relative error 1e-2
+(|d| / max(|ref|, rms(ref))) and mean absolute error <= 2e-3, both sides rounded to bf16.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import moqe_workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+ALL_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True), (3, 64, False), (4, 0, False),
+               (4, 32, False), (8, 128, False), (3, 32, True), (4, 256, False)]
+
+
+def _run(X, ids, gpu, path=0):
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import dev, bf16_to_torch, torch_to_bits
+    Y = moqe.moqe_routed_qgemm(bf16_to_torch(X), torch.from_numpy(ids).to(dev()), gpu, path=path)
+    st = moqe.moqe_async_status()
+    return torch_to_bits(Y), st
+
+
+def _paths():
+    import paper_2508_09204_b200 as moqe
+    return [moqe.PATH_STREAM, moqe.PATH_TCGEN05]
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_tiny_workload_full_compare(path):
+    """Config 'tiny': 1024x1024, W8 per-channel + W4 g128, 4 sequences x 16 tokens, every element compared."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close, assert_expert_matches
+    w = wl.get("tiny")
+    layer = w.layers[0]
+    W, X = wl.layer_inputs(w, layer)
+    gpu, What, canon = build_experts(W, w.experts)
+    for e, c in zip(gpu, canon):
+        assert_expert_matches(e, c)
+    ids = oracle.expand_ids(oracle.route(wl.router_logits(w)), w.row_offsets(layer))
+    Y, st = _run(X, ids, gpu, path)
+    assert st == moqe.OK
+    ref = oracle.routed_gemm(X, ids, What)
+    mx, mean = assert_close(Y, ref, "tiny")
+    assert mean < 2e-4            # in practice the two sides differ by a few bf16 roundings only
+
+
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (37, 136, 2304), (64, 1000, 640),
+                                   (150, 264, 1408)])
+def test_all_formats_small_shapes(path, M, N, K):
+    """Every supported format as its own expert; ragged N (not a multiple of 16/128), K not a multiple of 128,
+    several K blobs and splits, an expert that gets no rows."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close
+    specs = [f for f in ALL_FORMATS if f[1] == 0 or K % f[1] == 0]
+    W = wl.weights_f32(f"qg/{N}/{K}", N, K)
+    X = wl.activations_bf16(f"qg/{M}/{K}", M, K)
+    gpu, What, _ = build_experts(W, specs)
+    E = len(specs)
+    rs = np.random.default_rng(M + N + K)
+    ids = rs.integers(0, E, size=M).astype(np.int32)
+    if M > 4:
+        ids[ids == 2] = 0                                        # expert 2 idle
+    Y, st = _run(X, ids, gpu, path)
+    assert st == moqe.OK
+    assert_close(Y, oracle.routed_gemm(X, ids, What), f"M{M} N{N} K{K}")
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_exact_integer_case_on_gpu(path):
+    """On-grid W8 weights with power-of-two scale and small-integer activations: the exact int64 product."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts
+    rs = np.random.default_rng(55)
+    M, N, K = 24, 256, 512
+    q = rs.integers(-127, 128, size=(N, K))
+    q[:, 0], q[:, 1] = 127, -127
+    s0 = 2.0 ** -9
+    W = (q * s0).astype(np.float32)
+    Xi = rs.integers(-8, 9, size=(M, K))
+    X = wl.f32_to_bf16_bits(Xi.astype(np.float32))
+    gpu, _, _ = build_experts(W, [(8, 0, True)])
+    Y, st = _run(X, np.zeros(M, np.int32), gpu, path)
+    exact = (Xi.astype(np.int64) @ q.astype(np.int64).T).astype(np.float64) * s0
+    assert np.array_equal(Y, wl.f32_to_bf16_bits(exact.astype(np.float32)))
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_degenerate_batches(path):
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close, dev, bf16_to_torch
+    N, K = 256, 512
+    W = wl.weights_f32("deg", N, K)
+    specs = [(8, 0, True), (4, 128, False), (3, 128, False)]
+    gpu, What, _ = build_experts(W, specs)
+    # all rows to one expert == that expert alone (one expert per sample)
+    X = wl.activations_bf16("deg/X", 40, K)
+    for e in range(3):
+        ids = np.full(40, e, np.int32)
+        Y, st = _run(X, ids, gpu, path)
+        Y1, _ = _run(X, np.zeros(40, np.int32), [gpu[e]], path)
+        assert st == moqe.OK and np.array_equal(Y, Y1)
+        assert_close(Y, oracle.routed_gemm(X, ids, What), f"single expert {e}")
+    # batch shuffle: rows move with their inputs, bit for bit
+    rs = np.random.default_rng(3)
+    ids = rs.integers(0, 3, size=40).astype(np.int32)
+    Y, _ = _run(X, ids, gpu, path)
+    p = rs.permutation(40)
+    Yp, _ = _run(X[p], ids[p], gpu, path)
+    assert np.array_equal(Yp, Y[p])
+    # M = 0
+    Y0 = moqe.moqe_routed_qgemm(torch.empty((0, K), dtype=torch.bfloat16, device=dev()),
+                                torch.empty(0, dtype=torch.int32, device=dev()), gpu, path=path)
+    assert Y0.shape == (0, N)
+    # invalid ids: zero rows + latched status, other rows unaffected
+    bad = ids.copy()
+    bad[[3, 17]] = [7, -2]
+    Yb, st = _run(X, bad, gpu, path)
+    assert st == moqe.ERR_EXPERT_ID
+    assert np.all(Yb[[3, 17]] == 0)
+    keep = np.setdiff1d(np.arange(40), [3, 17])
+    assert np.array_equal(Yb[keep], Y[keep])
+
+
+def test_argument_errors():
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, dev
+    W1 = wl.weights_f32("err1", 128, 256)
+    W2 = wl.weights_f32("err2", 256, 256)
+    g1, _, _ = build_experts(W1, [(4, 128, False)])
+    g2, _, _ = build_experts(W2, [(4, 128, False)])
+    X = torch.zeros((8, 256), dtype=torch.bfloat16, device=dev())
+    ids = torch.zeros(8, dtype=torch.int32, device=dev())
+    with pytest.raises(moqe.MoqeError) as ei:
+        moqe.moqe_routed_qgemm(X, ids, [g1[0], g2[0]])
+    assert ei.value.code == moqe.ERR_MISMATCH
+    with pytest.raises(moqe.MoqeError) as ei:
+        moqe.moqe_routed_qgemm(X, ids, g1, workspace=torch.empty(256, dtype=torch.uint8, device=dev()))
+    assert ei.value.code == moqe.ERR_WORKSPACE
