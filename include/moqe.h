@@ -50,7 +50,7 @@ typedef enum {
     MOQE_OK = 0,
     MOQE_ERR_NULL = 1,         /* a required pointer is NULL */
     MOQE_ERR_SHAPE = 2,        /* a size is negative, zero where it may not be, or inconsistent */
-    MOQE_ERR_UNSUPPORTED = 3,  /* bits not in {3,4,8}; group not 0 or a multiple of 32 dividing K;
+    MOQE_ERR_UNSUPPORTED = 3,  /* bits not in {3,4,8}; group not 0, 32, 64 or a multiple of 128;
                                   K % 8 != 0; E > MOQE_MAX_EXPERTS; misaligned pointer */
     MOQE_ERR_ALLOC = 4,        /* device allocation failed */
     MOQE_ERR_WORKSPACE = 5,    /* workspace NULL or smaller than the *_workspace() figure */
@@ -77,8 +77,8 @@ typedef struct moqe_expert moqe_expert;
  *   asymmetric: lo = min(0,min w), hi = max(0,max w), s = fp16((hi-lo)/(2^b-1)),
  *               z = clamp(rint(-lo/s), 0, 2^b-1), c = clamp(rint(w/s)+z, 0, 2^b-1)
  *   s == 0 or non-finite after the fp16 rounding -> s = 1;   dequant = s*(c-z).
- * W: device fp32 [N][K], finite.  bits in {3,4,8}; group 0 or a multiple of 32
- * that divides K.  On success *out owns new device buffers (cudaMalloc'ed by
+ * W: device fp32 [N][K], finite.  bits in {3,4,8}; group 0, 32, 64 or a multiple
+ * of 128, dividing K.  On success *out owns new device buffers (cudaMalloc'ed by
  * this call; it is therefore not capturable in a CUDA graph) and must be
  * released with moqe_expert_destroy.  The kernels run on `stream`.
  * ------------------------------------------------------------------------- */
@@ -163,7 +163,8 @@ MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_id
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /* Same, with the kernel chosen by the caller (testing / measurement):
- * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM. */
+ * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM (automatic
+ * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles. */
 MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
                                    const moqe_expert* const* h_experts, int E, void* Y_bf16,
                                    void* workspace, size_t workspace_bytes, void* stream, int path);

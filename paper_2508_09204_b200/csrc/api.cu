@@ -76,7 +76,7 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     if (M == 0) return MOQE_OK;
     if (!X_bf16 || !row_ids || !Y_bf16) return MOQE_ERR_NULL;
     if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
-    if (path < 0 || path > 2) return MOQE_ERR_SHAPE;
+    if (path < 0 || path > 4) return MOQE_ERR_SHAPE;
     const int Np = h_experts[0]->Np;
     WsLayout w = ws_layout(M, Np, K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
@@ -92,6 +92,7 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     if (use_stream)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
+    tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
     return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
 

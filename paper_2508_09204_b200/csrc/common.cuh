@@ -85,6 +85,7 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
 size_t stream_zero_bytes(int M, int Np);
 
 // qgemm_tcgen05.cu
+void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)
 size_t tc_workspace_bytes(int M, int K, int E, int Np);
 moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
                             const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes,

@@ -1,0 +1,71 @@
+// Register-level unpacking of packed expert codes to exact bf16 integers (c - z).
+//
+// A "piece" is the 32 codes of one output channel that one lane owns inside a
+// 16-channel x 128-k blob (see common.cuh): four chunks G = 0..3 of 8
+// consecutive k.  unpack_chunk turns chunk G into four bf16x2 registers
+// (k offsets {0,1},{2,3},{4,5},{6,7}) whose values are the exact integers
+// c - z; the group scale is applied later in fp32, so the tensor cores only
+// see exactly representable operands.
+#pragma once
+#include "common.cuh"
+
+namespace moqe {
+
+template <int BITS> struct PieceWords;
+template <> struct PieceWords<4> { static constexpr int n = 4; };
+template <> struct PieceWords<8> { static constexpr int n = 8; };
+template <> struct PieceWords<3> { static constexpr int n = 3; };
+
+__device__ __forceinline__ uint32_t hsub2_bf16(uint32_t a, uint32_t b) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a), y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 r = __hsub2(x, y);
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// z: the integer zero-point of this channel and group, as a float.
+template <int BITS, int G>
+__device__ __forceinline__ void unpack_chunk(const uint32_t (&w)[PieceWords<BITS>::n], float z, uint32_t (&out)[4]) {
+    if constexpr (BITS == 4) {
+        // 0x4300 | c is the bf16 number 128 + c; subtracting 128 + z (<= 143, exact in bf16) is exact.
+        const uint32_t zz = pack_bf16x2(128.f + z, 128.f + z);
+        const uint32_t v = w[G];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = hsub2_bf16(((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zz);
+    } else if constexpr (BITS == 3) {
+        const uint32_t zz = pack_bf16x2(128.f + z, 128.f + z);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = 4 * G + i;                 // pair index inside the piece
+            uint32_t v;
+            if (p < 15) v = (w[p / 5] >> (3 * (p % 5))) & 0x00070007u;
+            else v = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u);
+            out[i] = hsub2_bf16(v | 0x43004300u, zz);
+        }
+    } else {
+        // 0x4B000000 | c is the fp32 number 2^23 + c; subtracting 2^23 + z is exact and |c - z| <= 255
+        // has at most 8 significant bits, so the conversion to bf16 is exact too.
+        const float f = 8388608.f + z;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t s = w[2 * G + (i >> 1)];
+            const uint32_t sel = 0x7540u + 2 * (i & 1);
+            float a = __uint_as_float(__byte_perm(s, 0x4B000000u, sel)) - f;
+            float b = __uint_as_float(__byte_perm(s, 0x4B000000u, sel + 1)) - f;
+            out[i] = pack_bf16x2(a, b);
+        }
+    }
+}
+
+// group index of chunk G of k-block kb:  per channel -> 0;  g = 32 -> 4*kb + G;  g = 64 -> 2*kb + G/2;
+// g >= 128 -> 128*kb / g
+__device__ __forceinline__ int group_of_chunk(int group, int kb, int G) {
+    if (group == 0) return 0;
+    if (group >= 128) return kb * 128 / group;
+    return (kb * 128 + 32 * G) / group;
+}
+
+}  // namespace moqe

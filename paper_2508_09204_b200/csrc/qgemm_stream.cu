@@ -20,7 +20,7 @@
 // inference on this sample") is the operation; the paper describes no kernel.
 #include <type_traits>
 
-#include "common.cuh"
+#include "dequant.cuh"
 
 namespace moqe {
 namespace {
@@ -65,95 +65,33 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint32_t hsub2_bf16(uint32_t a, uint32_t b) {
-    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a), y = *reinterpret_cast<__nv_bfloat162*>(&b);
-    __nv_bfloat162 r = __hsub2(x, y);
-    return *reinterpret_cast<uint32_t*>(&r);
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&r);
-}
-
 // The raw packed words one lane holds for one blob: the pieces of channel rows
-// gl and gl + 8 (gl = lane / 4) at k quarter q = lane % 4.
-template <int BITS> struct LaneBlob;
-template <> struct LaneBlob<4> { uint4 lo, hi; };
-template <> struct LaneBlob<8> { uint4 lo0, lo1, hi0, hi1; };
-template <> struct LaneBlob<3> { uint4 x; uint2 y; };
+// gl (lo) and gl + 8 (hi), gl = lane / 4, at k quarter q = lane % 4.
+template <int BITS>
+struct LaneBlob { uint32_t lo[PieceWords<BITS>::n], hi[PieceWords<BITS>::n]; };
 
 template <int BITS>
 __device__ __forceinline__ void load_blob(LaneBlob<BITS>& b, const uint8_t* blob, int slot) {
     if constexpr (BITS == 4) {
-        b.lo = ldg_stream16(blob + slot * 16);
-        b.hi = ldg_stream16(blob + 512 + slot * 16);
+        uint4 l = ldg_stream16(blob + slot * 16), h = ldg_stream16(blob + 512 + slot * 16);
+        b.lo[0] = l.x; b.lo[1] = l.y; b.lo[2] = l.z; b.lo[3] = l.w;
+        b.hi[0] = h.x; b.hi[1] = h.y; b.hi[2] = h.z; b.hi[3] = h.w;
     } else if constexpr (BITS == 8) {
-        b.lo0 = ldg_stream16(blob + slot * 16);
-        b.lo1 = ldg_stream16(blob + 512 + slot * 16);
-        b.hi0 = ldg_stream16(blob + 1024 + slot * 16);
-        b.hi1 = ldg_stream16(blob + 1536 + slot * 16);
+        uint4 l0 = ldg_stream16(blob + slot * 16), l1 = ldg_stream16(blob + 512 + slot * 16);
+        uint4 h0 = ldg_stream16(blob + 1024 + slot * 16), h1 = ldg_stream16(blob + 1536 + slot * 16);
+        b.lo[0] = l0.x; b.lo[1] = l0.y; b.lo[2] = l0.z; b.lo[3] = l0.w;
+        b.lo[4] = l1.x; b.lo[5] = l1.y; b.lo[6] = l1.z; b.lo[7] = l1.w;
+        b.hi[0] = h0.x; b.hi[1] = h0.y; b.hi[2] = h0.z; b.hi[3] = h0.w;
+        b.hi[4] = h1.x; b.hi[5] = h1.y; b.hi[6] = h1.z; b.hi[7] = h1.w;
     } else {
-        b.x = ldg_stream16(blob + slot * 16);
-        b.y = ldg_stream8(blob + 512 + slot * 8);
+        uint4 x = ldg_stream16(blob + slot * 16);
+        uint2 y = ldg_stream8(blob + 512 + slot * 8);
+        b.lo[0] = x.x; b.lo[1] = x.y; b.lo[2] = x.z;
+        b.hi[0] = x.w; b.hi[1] = y.x; b.hi[2] = y.y;
     }
 }
 
 __device__ __forceinline__ float pick4(const float (&a)[4], int j) { return j == 0 ? a[0] : j == 1 ? a[1] : j == 2 ? a[2] : a[3]; }
-__device__ __forceinline__ uint32_t word_of(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-
-// Chunk G of both rows -> four bf16x2 registers per row holding exact integers (c - z):
-// register i = (k offsets 2i, 2i+1) of the chunk's 8 consecutive k.
-// zlo / zhi: zero-points of rows gl and gl+8 for this chunk's group.
-template <int BITS, int G>
-__device__ __forceinline__ void unpack_chunk(const LaneBlob<BITS>& b, float zlo, float zhi, uint32_t (&lo)[4], uint32_t (&hi)[4]) {
-    if constexpr (BITS == 4) {
-        // 0x4300 | c  is the bf16 number 128 + c; subtracting 128 + z is exact
-        const uint32_t zl = pack_bf16x2(128.f + zlo, 128.f + zlo), zh = pack_bf16x2(128.f + zhi, 128.f + zhi);
-        const uint32_t wl = word_of(b.lo, G), wh = word_of(b.hi, G);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            lo[i] = hsub2_bf16(((wl >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zl);
-            hi[i] = hsub2_bf16(((wh >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zh);
-        }
-    } else if constexpr (BITS == 3) {
-        const uint32_t zl = pack_bf16x2(128.f + zlo, 128.f + zlo), zh = pack_bf16x2(128.f + zhi, 128.f + zhi);
-        const uint32_t wlo[3] = {b.x.x, b.x.y, b.x.z};
-        const uint32_t whi[3] = {b.x.w, b.y.x, b.y.y};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int p = 4 * G + i;
-            uint32_t vl, vh;
-            if (p < 15) {
-                vl = (wlo[p / 5] >> (3 * (p % 5))) & 0x00070007u;
-                vh = (whi[p / 5] >> (3 * (p % 5))) & 0x00070007u;
-            } else {
-                vl = ((wlo[0] >> 15) & 0x00010001u) | ((wlo[1] >> 14) & 0x00020002u) | ((wlo[2] >> 13) & 0x00040004u);
-                vh = ((whi[0] >> 15) & 0x00010001u) | ((whi[1] >> 14) & 0x00020002u) | ((whi[2] >> 13) & 0x00040004u);
-            }
-            lo[i] = hsub2_bf16(vl | 0x43004300u, zl);
-            hi[i] = hsub2_bf16(vh | 0x43004300u, zh);
-        }
-    } else {
-        // 0x4B000000 | c  is the fp32 number 2^23 + c; subtracting 2^23 + z is exact, and so is
-        // the conversion of the (<= 9-bit) difference to bf16 unless |c - z| = 255 needs 8 bits: fine.
-        const float fl = 8388608.f + zlo, fh = 8388608.f + zhi;
-        const uint4& vl = (G < 2) ? b.lo0 : b.lo1;
-        const uint4& vh = (G < 2) ? b.hi0 : b.hi1;
-        const uint32_t wl[2] = {word_of(vl, 2 * (G & 1)), word_of(vl, 2 * (G & 1) + 1)};
-        const uint32_t wh[2] = {word_of(vh, 2 * (G & 1)), word_of(vh, 2 * (G & 1) + 1)};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t sl = wl[i >> 1], sh = wh[i >> 1];
-            const uint32_t s0 = 0x7540u + 2 * (i & 1), s1 = s0 + 1;
-            float l0 = __uint_as_float(__byte_perm(sl, 0x4B000000u, s0)) - fl;
-            float l1 = __uint_as_float(__byte_perm(sl, 0x4B000000u, s1)) - fl;
-            float h0 = __uint_as_float(__byte_perm(sh, 0x4B000000u, s0)) - fh;
-            float h1 = __uint_as_float(__byte_perm(sh, 0x4B000000u, s1)) - fh;
-            lo[i] = pack_bf16x2(l0, l1);
-            hi[i] = pack_bf16x2(h0, h1);
-        }
-    }
-}
 
 // per-blob scale / zero-point values of the lane's two channel rows (up to 4 groups per blob)
 struct BlobMeta { float s_lo[4], s_hi[4], z_lo[4], z_hi[4]; };
@@ -236,7 +174,8 @@ __device__ __forceinline__ void run_task(const StreamParams& p, const ExpertDev&
                     constexpr int G = decltype(Gc)::value;
                     const int gj = per_channel ? 0 : (ngrp == 4 ? G : (ngrp == 2 ? (G >> 1) : 0));
                     uint32_t lo[4], hi[4];
-                    unpack_chunk<BITS, G>(cur, pick4(mcur.z_lo, gj), pick4(mcur.z_hi, gj), lo, hi);
+                    unpack_chunk<BITS, G>(cur.lo, pick4(mcur.z_lo, gj), lo);
+                    unpack_chunk<BITS, G>(cur.hi, pick4(mcur.z_hi, gj), hi);
 #pragma unroll
                     for (int t = 0; t < NT; ++t) {
                         uint4 xb = *reinterpret_cast<const uint4*>(xrow + t * 8 * XS_STRIDE + G * 64);

@@ -1,7 +1,561 @@
-// placeholder until the tcgen05 grouped GEMM lands
-#include "common.cuh"
+// Routed dequant-GEMM for large batches (prefill shapes): a persistent,
+// warp-specialised grouped GEMM on the 5th-generation tensor cores.
+//
+//   tile         : 128 output channels (UMMA M, the TMEM lanes) x TN tokens (UMMA N, TMEM columns)
+//   A operand    : the expert's weights.  Packed 128x128-code tiles arrive by bulk
+//                  async copy; four "dequant" warps unpack them in registers to the
+//                  exact integers (c - z) in bf16 and store them as a K-major,
+//                  128-byte-swizzled shared-memory operand (64 k per stage).
+//   B operand    : token rows, loaded by TMA (2-D tiled, 128-byte swizzle) from the
+//                  expert-sorted activation matrix.
+//   accumulation : tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) into one of two TMEM
+//                  buffers per quantization group; eight "epilogue" warps drain the
+//                  finished buffer, multiply by the group's fp32 scale and add into
+//                  register accumulators while the MMA fills the other buffer:
+//                      Y[m][n] = sum_G s[n][G] * (sum_{k in G} X[m][k] * (c[n][k] - z[n][G]))
+//                  so the tensor core only multiplies exactly representable numbers.
+//                  Per-channel experts need a single scale at the end of K.
+//   scheduling   : one CTA per SM walks the tile list (expert, token tile, channel
+//                  tile) derived on the device from the per-expert offset table;
+//                  rows are written straight to their original positions through
+//                  `perm` (fused un-permutation).
+//
+// Every mbarrier wait is bounded (2 s of %globaltimer); on expiry the CTA sets
+// an abort flag, latches MOQE_ERR_TIMEOUT, lets copies in flight land, frees
+// its TMEM and returns.
+//
+// The operation is Section 3.1 of the paper (the selected quantization expert
+// runs the sample); the paper describes no kernel.
+#include <cuda.h>
+
+#include <type_traits>
+
+#include "dequant.cuh"
+
 namespace moqe {
-size_t tc_workspace_bytes(int, int, int, int) { return 0; }
-moqe_status launch_qgemm_tc(const void*, int, int, int, const moqe_expert* const*, int, void*, const int32_t*,
-                            const int32_t*, void*, size_t, cudaStream_t) { return MOQE_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int TC_THREADS = 512;
+constexpr int NS = 3;                 // operand stages (A tile + X tile, 64 k each)
+constexpr int NWS = 3;                // packed-weight stages (128 k each)
+constexpr int A_STAGE_BYTES = 128 * 128;          // 128 channels x 64 bf16
+constexpr int W_STAGE_BYTES = 128 * 128;          // largest packed tile (W8)
+constexpr int XBOX_ROWS = 64;
+constexpr int XBOX_BYTES = XBOX_ROWS * 128;
+
+struct TcParams {
+    ExpertDev ex[MOQE_MAX_EXPERTS];
+    const int32_t* perm;
+    const int32_t* offsets;
+    uint16_t* Y;
+    int* status;
+    int M, N, K, Np, KB, E, n_tiles;
+};
+
+template <int TN>
+struct Smem {
+    static constexpr int a_off = 0;
+    static constexpr int x_off = a_off + NS * A_STAGE_BYTES;
+    static constexpr int w_off = x_off + NS * TN * 128;
+    static constexpr int bar_off = w_off + NWS * W_STAGE_BYTES;
+    // barriers: wfull[NWS] wempty[NWS] xfull[NS] afull[NS] empty[NS] accfull[2] accempty[2]
+    static constexpr int n_bars = 2 * NWS + 3 * NS + 4;
+    static constexpr int misc_off = bar_off + n_bars * 8;              // tmem addr, abort flag
+    static constexpr int off_off = misc_off + 16;                      // offsets[E+1]
+    static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;
+    static constexpr int total = perm_off + 8 * (TN / 2) * 4;          // per epilogue warp: its columns' target rows
+    static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
+};
+
+// ---------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+// Bounded wait.  Returns false if the CTA is aborting (someone's wait ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_test(bar, parity)) return true;
+    unsigned long long t0 = global_ns();
+    for (unsigned spin = 1;; ++spin) {
+        if (mbar_test(bar, parity)) return true;
+        if ((spin & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                latch_status(status, (int)MOQE_ERR_TIMEOUT);
+                return false;
+            }
+            __nanosleep(64);
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile, rows of 64 bf16 (128 bytes), 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------- tile list
+struct TileInfo { int e, nt, m0, rows; };
+
+template <int TN>
+__device__ __forceinline__ bool decode_tile(const int* s_off, int E, int n_tiles, int t, TileInfo& ti) {
+    for (int e = 0; e < E; ++e) {
+        int Me = s_off[e + 1] - s_off[e];
+        int cnt = ((Me + TN - 1) / TN) * n_tiles;
+        if (t < cnt) {
+            int mt = t / n_tiles;
+            ti.e = e;
+            ti.nt = t - mt * n_tiles;
+            ti.m0 = s_off[e] + mt * TN;
+            ti.rows = min(TN, Me - mt * TN);
+            return true;
+        }
+        t -= cnt;
+    }
+    return false;
+}
+
+struct Ring {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int n) { if (++stage == n) { stage = 0; phase ^= 1u; } }
+};
+
+// ---------------------------------------------------------------------------- dequant role
+template <int BITS>
+__device__ __forceinline__ void load_piece_smem(const unsigned char* blob, int half, int slot, uint32_t (&w)[PieceWords<BITS>::n]) {
+    if constexpr (BITS == 4) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if constexpr (BITS == 8) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 1024 + slot * 16);
+        uint4 u = *reinterpret_cast<const uint4*>(blob + half * 1024 + 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; w[4] = u.x; w[5] = u.y; w[6] = u.z; w[7] = u.w;
+    } else {
+        if (half == 0) {
+            uint4 v = *reinterpret_cast<const uint4*>(blob + slot * 16);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z;
+        } else {
+            w[0] = *reinterpret_cast<const uint32_t*>(blob + slot * 16 + 12);
+            uint2 u = *reinterpret_cast<const uint2*>(blob + 512 + slot * 8);
+            w[1] = u.x; w[2] = u.y;
+        }
+    }
+}
+
+// One k-block (128 k) of one tile: wait for the packed tile, pull this thread's four pieces into
+// registers, release the packed stage, then fill the two 64-k operand stages.
+template <int BITS>
+__device__ __forceinline__ bool dequant_kblock(const ExpertDev& ex, int Np, int nt, int kb, unsigned char* smem_w,
+                                               unsigned char* smem_a_base, uint32_t bar_wfull, uint32_t bar_wempty,
+                                               uint32_t wphase, uint32_t bar_empty0, uint32_t bar_afull0, Ring& ring,
+                                               volatile int* abort_flag, int* status) {
+    const int lane = threadIdx.x & 31, dw = (threadIdx.x >> 5) & 3;
+    const int q = lane >> 3, r = lane & 7;
+    constexpr int NWORDS = PieceWords<BITS>::n;
+    const float sym_z = (float)(1 << (BITS - 1));
+    // zero-points of the four pieces' channels, per chunk
+    float z[4][4];
+#pragma unroll
+    for (int pi = 0; pi < 4; ++pi) {
+        const int n = nt * 128 + (2 * dw + (pi >> 1)) * 16 + (pi & 1) * 8 + r;
+        if (!ex.zeros_t) {
+#pragma unroll
+            for (int G = 0; G < 4; ++G) z[pi][G] = sym_z;
+        } else if (ex.group == 32 || ex.group == 64) {
+#pragma unroll
+            for (int G = 0; G < 4; ++G)
+                z[pi][G] = __bfloat162float(ex.zeros_t[(size_t)group_of_chunk(ex.group, kb, G) * Np + n]);
+        } else {
+            float v = __bfloat162float(ex.zeros_t[(size_t)group_of_chunk(ex.group, kb, 0) * Np + n]);
+#pragma unroll
+            for (int G = 0; G < 4; ++G) z[pi][G] = v;
+        }
+    }
+    if (!mbar_wait(bar_wfull, wphase, abort_flag, status)) return false;
+    uint32_t w[4][NWORDS];
+#pragma unroll
+    for (int pi = 0; pi < 4; ++pi)
+        load_piece_smem<BITS>(smem_w + (2 * dw + (pi >> 1)) * moqe_blob_bytes(BITS), pi & 1, lane, w[pi]);
+    mbar_arrive(bar_wempty);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        if (!mbar_wait(bar_empty0 + 8 * ring.stage, ring.phase ^ 1u, abort_flag, status)) return false;
+        unsigned char* a_stage = smem_a_base + ring.stage * A_STAGE_BYTES;
+#pragma unroll
+        for (int pi = 0; pi < 4; ++pi) {
+            const int row = (2 * dw + (pi >> 1)) * 16 + (pi & 1) * 8 + r;
+            auto put = [&](auto Gc) {
+                constexpr int G = decltype(Gc)::value;
+                uint32_t out[4];
+                unpack_chunk<BITS, G>(w[pi], z[pi][G], out);
+                const int chunk = (G & 1) * 4 + q;
+                *reinterpret_cast<uint4*>(a_stage + row * 128 + ((chunk ^ (row & 7)) << 4)) =
+                    make_uint4(out[0], out[1], out[2], out[3]);
+            };
+            if (h == 0) { put(std::integral_constant<int, 0>{}); put(std::integral_constant<int, 1>{}); }
+            else        { put(std::integral_constant<int, 2>{}); put(std::integral_constant<int, 3>{}); }
+        }
+        fence_proxy_async();
+        mbar_arrive(bar_afull0 + 8 * ring.stage);
+        ring.advance(NS);
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------- the kernel
+template <int TN, bool REGSPLIT>
+__global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_constant__ TcParams p,
+                                                                const __grid_constant__ CUtensorMap tmap) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    using L = Smem<TN>;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::bar_off;
+    const uint32_t bar_wfull = bar0, bar_wempty = bar0 + 8 * NWS, bar_xfull = bar0 + 16 * NWS;
+    const uint32_t bar_afull = bar_xfull + 8 * NS, bar_empty = bar_afull + 8 * NS;
+    const uint32_t bar_accfull = bar_empty + 8 * NS, bar_accempty = bar_accfull + 16;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::misc_off);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
+    int* s_off = reinterpret_cast<int*>(smem + L::off_off);
+    int* s_perm = reinterpret_cast<int*>(smem + L::perm_off);
+
+    if (tid == 0) {
+        for (int i = 0; i < NWS; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, 128); }
+        for (int i = 0; i < NS; ++i) { mbar_init(bar_xfull + 8 * i, 1); mbar_init(bar_afull + 8 * i, 128); mbar_init(bar_empty + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accempty + 8 * i, 256); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i <= p.E; i += TC_THREADS) s_off[i] = p.offsets[i];
+    if (warp == 1) tmem_alloc(sbase + L::misc_off, 2 * TN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp < 4) {
+        if constexpr (REGSPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if (warp == 0 && lane == 0) {
+            // ---------------- X producer: TMA boxes of 64 token rows x 64 k ----------------
+            Ring ring;
+            TileInfo ti;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
+                const int nbox = (ti.rows + XBOX_ROWS - 1) / XBOX_ROWS;
+                for (int ks = 0; ks < 2 * p.KB; ++ks) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status))) break;
+                    const uint32_t full = bar_xfull + 8 * ring.stage;
+                    mbar_expect_tx(full, nbox * XBOX_BYTES);
+                    const uint32_t dst = sbase + L::x_off + ring.stage * (TN * 128);
+                    for (int b = 0; b < nbox; ++b) tma_load_2d(dst + b * XBOX_BYTES, &tmap, ks * 64, ti.m0 + b * XBOX_ROWS, full);
+                    ring.advance(NS);
+                }
+            }
+        } else if (warp == 2 && lane == 0) {
+            // ---------------- W producer: one packed 128x128-code tile per k-block ----------------
+            Ring ring;
+            TileInfo ti;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
+                const ExpertDev& ex = p.ex[ti.e];
+                const uint32_t bytes = (uint32_t)moqe_tile_bytes(ex.bits);
+                const uint8_t* src = ex.codes + (size_t)ti.nt * p.KB * bytes;
+                for (int kb = 0; kb < p.KB; ++kb) {
+                    if (!(ok = mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status))) break;
+                    const uint32_t full = bar_wfull + 8 * ring.stage;
+                    mbar_expect_tx(full, bytes);
+                    bulk_load(sbase + L::w_off + ring.stage * W_STAGE_BYTES, src + (size_t)kb * bytes, bytes, full);
+                    ring.advance(NWS);
+                }
+            }
+        } else if (warp == 1 && lane == 0) {
+            // ---------------- MMA issuer ----------------
+            Ring ring;
+            TileInfo ti;
+            bool ok = true;
+            uint32_t acc_use[2] = {0, 0};
+            int buf = 0;
+            for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
+                const ExpertDev& ex = p.ex[ti.e];
+                const int n_eff = (ti.rows + 15) & ~15;
+                const uint32_t idesc = umma_idesc(n_eff);
+                const int group_k = ex.group == 0 ? p.KB * 128 : min(ex.group, 128);
+                int kcount = 0;
+                for (int ks = 0; ok && ks < 2 * p.KB; ++ks) {
+                    if (!(ok = mbar_wait(bar_xfull + 8 * ring.stage, ring.phase, s_abort, p.status))) break;
+                    if (!(ok = mbar_wait(bar_afull + 8 * ring.stage, ring.phase, s_abort, p.status))) break;
+                    tc_fence_after();
+                    const uint64_t adesc = umma_desc_sw128(sbase + L::a_off + ring.stage * A_STAGE_BYTES);
+                    const uint64_t bdesc = umma_desc_sw128(sbase + L::x_off + ring.stage * (TN * 128));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (kcount == 0) {
+                            if (!(ok = mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status))) break;
+                            tc_fence_after();
+                        }
+                        umma_bf16(tmem_base + buf * TN, adesc + 2 * j, bdesc + 2 * j, idesc, kcount > 0 ? 1u : 0u);
+                        kcount += 16;
+                        if (kcount == group_k) {
+                            umma_commit(bar_accfull + 8 * buf);
+                            acc_use[buf]++;
+                            buf ^= 1;
+                            kcount = 0;
+                        }
+                    }
+                    umma_commit(bar_empty + 8 * ring.stage);
+                    ring.advance(NS);
+                }
+            }
+        }
+    } else if (warp < 8) {
+        if constexpr (REGSPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+        // ---------------- dequant warps ----------------
+        Ring wring, ring;
+        TileInfo ti;
+        bool ok = true;
+        for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
+            const ExpertDev& ex = p.ex[ti.e];
+            for (int kb = 0; ok && kb < p.KB; ++kb) {
+                unsigned char* sw = smem + L::w_off + wring.stage * W_STAGE_BYTES;
+                const uint32_t wf = bar_wfull + 8 * wring.stage, we = bar_wempty + 8 * wring.stage;
+                if (ex.bits == 4)
+                    ok = dequant_kblock<4>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                else if (ex.bits == 8)
+                    ok = dequant_kblock<8>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                else
+                    ok = dequant_kblock<3>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                wring.advance(NWS);
+            }
+        }
+    } else {
+        if constexpr (REGSPLIT) asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
+        // ---------------- epilogue warps: scale-and-accumulate, then store ----------------
+        constexpr int NCOL = TN / 2;                       // columns (tokens) per warp
+        const int ew = warp - 8, quarter = ew & 3, colhalf = ew >> 2;
+        const int col0 = colhalf * NCOL;
+        const int row = quarter * 32 + lane;               // channel inside the tile = TMEM lane
+        TileInfo ti;
+        bool ok = true;
+        uint32_t acc_use[2] = {0, 0};
+        int buf = 0;
+        for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
+            const ExpertDev& ex = p.ex[ti.e];
+            const int n = ti.nt * 128 + row;
+            const int n_eff = (ti.rows + 15) & ~15;
+            int* my_perm = s_perm + ew * NCOL;                     // private to this warp: no cross-warp barrier
+            __syncwarp();
+            for (int i = lane; i < NCOL; i += 32) my_perm[i] = (col0 + i < ti.rows) ? p.perm[ti.m0 + col0 + i] : -1;
+            __syncwarp();
+            float acc[NCOL];
+#pragma unroll
+            for (int i = 0; i < NCOL; ++i) acc[i] = 0.f;
+            const int group_k = ex.group == 0 ? p.KB * 128 : min(ex.group, 128);
+            const int ngroups = p.KB * 128 / group_k;
+            for (int gi = 0; ok && gi < ngroups; ++gi) {
+                const int sidx = ex.group == 0 ? 0 : (ex.group >= 128 ? gi * 128 / ex.group : gi);
+                const float s = __half2float(ex.scales_t[(size_t)sidx * p.Np + n]);
+                if (!(ok = mbar_wait(bar_accfull + 8 * buf, acc_use[buf] & 1u, s_abort, p.status))) break;
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < NCOL / 32; ++c) {
+                    if (col0 + c * 32 < n_eff) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * TN + col0 + c * 32, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(s, __uint_as_float(v[i]), acc[c * 32 + i]);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bar_accempty + 8 * buf);
+                acc_use[buf]++;
+                buf ^= 1;
+            }
+            if (ok && n < p.N) {
+#pragma unroll
+                for (int i = 0; i < NCOL; ++i) {
+                    const int col = col0 + i;
+                    if (col < ti.rows) p.Y[(size_t)my_perm[i] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[i]));
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        // let bulk copies that may still be in flight land before the shared memory is released
+        unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2 * TN);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)f;
+    }
+    return fn;
+}
+
+int g_tile_tokens_override = 0;
+
+}  // namespace
+
+void tc_set_tile_tokens(int tn) { g_tile_tokens_override = tn; }
+
+size_t tc_workspace_bytes(int M, int K, int E, int Np) {
+    (void)E; (void)Np;
+    return ((size_t)M * K * 2 + 255) / 256 * 256;
+}
+
+moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
+                            const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
+    if (M == 0) return MOQE_OK;
+    if (!ws || ws_bytes < tc_workspace_bytes(M, K, E, ex[0]->Np)) return MOQE_ERR_WORKSPACE;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return MOQE_ERR_CUDA;
+    // 1. expert-sorted copy of the activations (rows with an invalid id become zero rows at the end)
+    void* Xp = ws;
+    moqe_status s = launch_gather(X, perm, offsets + E, M, K, Xp, st);
+    if (s != MOQE_OK) return s;
+    // 2. tensor map over Xp[M][K] bf16: boxes of 64 k x 64 rows, 128-byte swizzle, zero fill outside
+    CUtensorMap tmap;
+    cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    cuuint64_t gstride[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)XBOX_ROWS};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Xp, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return MOQE_ERR_CUDA;
+    TcParams p;
+    for (int e = 0; e < E; ++e) {
+        p.ex[e].codes = ex[e]->codes;
+        p.ex[e].scales_t = ex[e]->scales_t;
+        p.ex[e].zeros_t = ex[e]->zeros_t;
+        p.ex[e].bits = ex[e]->bits;
+        p.ex[e].group = ex[e]->group;
+    }
+    p.perm = perm; p.offsets = offsets; p.Y = (uint16_t*)Y; p.status = device_status_word();
+    p.M = M; p.N = N; p.K = K; p.Np = ex[0]->Np; p.KB = ex[0]->Kp / 128; p.E = E; p.n_tiles = p.Np / 128;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int tn = g_tile_tokens_override ? g_tile_tokens_override : (M >= 2048 ? 256 : 128);
+    long long max_tiles = ((long long)(M + tn - 1) / tn + E) * p.n_tiles;
+    int grid = (int)(max_tiles < sms ? max_tiles : sms);
+    cudaError_t err;
+    if (tn == 256) {
+        static bool attr = false;
+        if (!attr) {
+            if (cudaFuncSetAttribute(qgemm_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<256>::dyn_bytes) != cudaSuccess)
+                return MOQE_ERR_CUDA;
+            attr = true;
+        }
+        qgemm_tc_kernel<256, true><<<grid, TC_THREADS, Smem<256>::dyn_bytes, st>>>(p, tmap);
+    } else {
+        static bool attr = false;
+        if (!attr) {
+            if (cudaFuncSetAttribute(qgemm_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::dyn_bytes) != cudaSuccess)
+                return MOQE_ERR_CUDA;
+            attr = true;
+        }
+        qgemm_tc_kernel<128, false><<<grid, TC_THREADS, Smem<128>::dyn_bytes, st>>>(p, tmap);
+    }
+    err = cudaGetLastError();
+    count_launch();
+    return cuda_ok(err);
+}
+
+}  // namespace moqe

@@ -8,7 +8,7 @@
 // math), so codes, scales and zero-points are reproducible bit for bit.
 #include <new>
 
-#include "common.cuh"
+#include "dequant.cuh"
 
 namespace moqe {
 namespace {
@@ -17,12 +17,6 @@ namespace {
 // piece <-> packed words
 // ---------------------------------------------------------------------------
 // code index i = 8*G + t  (chunk G, position t)  <->  k = 128*kb + 32*G + 8*q + t
-template <int BITS>
-struct PieceWords;   // number of 32-bit words per piece
-template <> struct PieceWords<4> { static constexpr int n = 4; };
-template <> struct PieceWords<8> { static constexpr int n = 8; };
-template <> struct PieceWords<3> { static constexpr int n = 3; };
-
 template <int BITS>
 __device__ __forceinline__ void encode_piece(const uint32_t (&c)[32], uint32_t (&w)[PieceWords<BITS>::n]) {
     if constexpr (BITS == 4) {

@@ -251,9 +251,12 @@ extern "C" size_t moqe_permute_workspace(int M, int E) { return sort_workspace_b
 extern "C" moqe_status moqe_permute(const void* X_bf16, const int32_t* row_ids, int M, int C, int E, void* Xp_bf16,
                                     int32_t* perm, int32_t* offsets, void* workspace, size_t workspace_bytes,
                                     void* stream) {
-    if (!row_ids || !perm || !offsets) return MOQE_ERR_NULL;
+    if (!offsets) return MOQE_ERR_NULL;
+    if (M < 0 || E <= 0) return MOQE_ERR_SHAPE;
+    if (M > 0 && (!row_ids || !perm)) return MOQE_ERR_NULL;           // an empty batch needs no row arrays
+    if (M == 0) X_bf16 = Xp_bf16 = nullptr;
     if ((X_bf16 == nullptr) != (Xp_bf16 == nullptr)) return MOQE_ERR_NULL;
-    if (M < 0 || E <= 0 || (X_bf16 && C <= 0)) return MOQE_ERR_SHAPE;
+    if (X_bf16 && C <= 0) return MOQE_ERR_SHAPE;
     if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
     if (X_bf16 && (C % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Xp_bf16 % 16)) return MOQE_ERR_UNSUPPORTED;
     if (M > SORT_THREADS && (!workspace || workspace_bytes < sort_workspace_bytes(M, E))) return MOQE_ERR_WORKSPACE;

@@ -29,7 +29,7 @@ def _paths():
     return [moqe.PATH_STREAM, moqe.PATH_TCGEN05]
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 3, 4])
 def test_tiny_workload_full_compare(path):
     """Config 'tiny': 1024x1024, W8 per-channel + W4 g128, 4 sequences x 16 tokens, every element compared."""
     import paper_2508_09204_b200 as moqe
@@ -48,7 +48,7 @@ def test_tiny_workload_full_compare(path):
     assert mean < 2e-4            # in practice the two sides differ by a few bf16 roundings only
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 3, 4])
 @pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (37, 136, 2304), (64, 1000, 640),
                                    (150, 264, 1408)])
 def test_all_formats_small_shapes(path, M, N, K):
@@ -70,7 +70,7 @@ def test_all_formats_small_shapes(path, M, N, K):
     assert_close(Y, oracle.routed_gemm(X, ids, What), f"M{M} N{N} K{K}")
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 3, 4])
 def test_exact_integer_case_on_gpu(path):
     """On-grid W8 weights with power-of-two scale and small-integer activations: the exact int64 product."""
     import paper_2508_09204_b200 as moqe
@@ -89,7 +89,7 @@ def test_exact_integer_case_on_gpu(path):
     assert np.array_equal(Y, wl.f32_to_bf16_bits(exact.astype(np.float32)))
 
 
-@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("path", [1, 3, 4])
 def test_degenerate_batches(path):
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, assert_close, dev, bf16_to_torch
