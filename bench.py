@@ -1,0 +1,446 @@
+#!/usr/bin/env python
+"""Benchmark of the routed quantized-linear path on B200.
+
+One *step* is one pass of the whole hot path over one synthetic batch of a
+workload: route (arg-max of resident logits) -> expand ids -> stable sort by
+expert -> the routed dequant-GEMM of every linear layer of the block, each fed
+its own resident activations, outputs written back in original row order.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is tokens/s over all N GPUs with inputs
+resident in HBM; `e2e` is the same metric with host buffers (pinned host ->
+device copies of logits and activations and device -> host copies of the outputs
+inside the timed region); `roofline` describes the dominant kernel; and
+`cpu_baseline` is the CPU oracle timed on this machine's cores on a bounded
+sample.  `--impl reference` times that oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import moqe_workloads as wl  # noqa: E402
+
+METRIC = "routed_qgemm_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# --------------------------------------------------------------------------- helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the GPU is under load."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if bit and (r & bit):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def workload_logits(w, seed, pooled_from=None):
+    if w.routing == "router_mlp":
+        layer = w.layers[0]
+        X = wl.activations_bf16(f"{w.name}/{layer.name}/X", w.M_of(layer), layer.K, w.relu_inputs, seed)
+        return wl.router_logits(w, seed, pooled=wl.mean_pool(X, w.row_offsets(layer)))
+    return wl.router_logits(w, seed)
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_plan(w):
+    """Distinct layer shapes with their multiplicity inside the block: timing one of each and
+    weighting by the multiplicity reproduces the block's work exactly."""
+    shapes = {}
+    for l in w.layers:
+        key = (l.N, l.K, l.rows_per_sample)
+        if key not in shapes:
+            shapes[key] = [l, 0]
+        shapes[key][1] += 1
+    return list(shapes.values())
+
+
+def run_oracle_once(w, prepared, rows_per_layer):
+    """-> seconds of oracle routed GEMM for the block (distinct shapes x multiplicity), rows sampled."""
+    import oracle
+    total = 0.0
+    for (layer, mult, X, row_ids, What, rows) in prepared:
+        t0 = time.perf_counter()
+        oracle.routed_gemm(X, row_ids, What, rows=rows)
+        dt = time.perf_counter() - t0
+        M = X.shape[0]
+        total += dt * mult * (M / float(len(rows)))          # linear in rows: extrapolated to all M rows
+    return total
+
+
+def prepare_oracle(w, seed, max_rows):
+    import oracle
+    ids = oracle.route(workload_logits(w, seed))
+    prepared, t_quant, t_deq = [], 0.0, 0.0
+    for layer, mult in oracle_sample_plan(w):
+        W, X = wl.layer_inputs(w, layer, seed)
+        row_ids = oracle.expand_ids(ids, w.row_offsets(layer))
+        What = []
+        for sp in w.experts:
+            t0 = time.perf_counter()
+            c, s, z = oracle.quantize_rtn(W, sp.bits, sp.group, sp.sym)
+            t1 = time.perf_counter()
+            What.append(oracle.dequantize(c, s, z, sp.group))
+            t2 = time.perf_counter()
+            t_quant += (t1 - t0) * mult
+            t_deq += (t2 - t1) * mult
+        M = X.shape[0]
+        _, offsets, perm, _ = oracle.permutation(row_ids, w.n_experts)
+        if M <= max_rows:
+            rows = np.arange(M, dtype=np.int32)
+        else:                                                 # first/last row of every expert + evenly spaced rows
+            per = max(1, max_rows // w.n_experts)
+            pick = []
+            for e in range(w.n_experts):
+                lo, hi = int(offsets[e]), int(offsets[e + 1])
+                if hi > lo:
+                    pick.extend(perm[np.unique(np.linspace(lo, hi - 1, num=min(per, hi - lo)).astype(np.int64))])
+            rows = np.array(sorted(set(int(v) for v in pick)), dtype=np.int32)
+        prepared.append((layer, mult, X, row_ids, What, rows))
+    return prepared, t_quant, t_deq
+
+
+def oracle_sample_text(w, prepared):
+    parts = [f"{layer.name} x{mult} ({len(rows)}/{X.shape[0]} rows, all N, full K)" for (layer, mult, X, _, _, rows) in prepared]
+    return "oracle routed GEMM on one layer of each distinct shape, weighted by its count in the block: " + "; ".join(parts)
+
+
+def reference_arm(args, w):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    tokens = sum(w.sample_rows) if w.layers[0].rows_per_sample is None else w.n_samples
+    budget_s = 150.0
+    max_rows = 16
+    prepared, t_quant, t_deq = prepare_oracle(w, args.seed, max_rows)
+    probe = 0.0
+    t0 = time.perf_counter()
+    run_oracle_once(w, prepared, None)
+    probe = time.perf_counter() - t0
+    if probe * (args.steps + args.warmup) > budget_s and max_rows > 3:
+        max_rows = max(3, int(max_rows * budget_s / (probe * (args.steps + args.warmup))))
+        prepared, t_quant, t_deq = prepare_oracle(w, args.seed, max_rows)
+    for _ in range(args.warmup):
+        run_oracle_once(w, prepared, None)
+    times = [run_oracle_once(w, prepared, None) for _ in range(args.steps)]
+    step_s = float(np.mean(times))
+    value = tokens / step_s
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "tokens_per_step": tokens, "note": "CPU oracle (plain C, fp32 sequential accumulation), extrapolated linearly to the block"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": oracle_sample_text(w, prepared), "dequant_s": t_deq, "quantize_s": t_quant},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- the CUDA arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_decode", choices=list(wl.WORKLOAD_ORDER))
+    ap.add_argument("--path", type=int, default=0, help="0 auto, 1 streaming kernel, 2-4 tcgen05 kernel")
+    ap.add_argument("--seed", type=int, default=wl.BASE_SEED)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    args = ap.parse_args()
+    w = wl.get(args.workload)
+    heavy = w.kind in ("prefill", "mixed", "conv")
+    if args.steps is None:
+        args.steps = 20 if heavy else 2000
+    if args.warmup is None:
+        args.warmup = 3 if heavy else 200
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2508_09204_b200 as moqe
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the routed path has no CPU fallback")
+    moqe.lib()                                              # fails loudly if the CUDA library is not built
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    seed = args.seed + 1000 * rank                          # every rank owns its own shard of samples (weak scaling)
+    E = w.n_experts
+
+    # ---- experts (replicated on every rank) and resident inputs ---------------------------------
+    layers = []
+    for layer in w.layers:
+        Wd = torch.from_numpy(wl.weights_f32(f"{w.name}/{layer.name}/W", layer.N, layer.K, 0.02, args.seed)).to(dev)
+        experts = [moqe.moqe_quantize_rtn(Wd, sp.bits, sp.group, sp.sym) for sp in w.experts]
+        del Wd
+        M = w.M_of(layer)
+        Xh = torch.from_numpy(wl.activations_bf16(f"{w.name}/{layer.name}/X", M, layer.K, w.relu_inputs, seed).view(np.int16)).view(torch.bfloat16).pin_memory()
+        X = Xh.to(dev)
+        Y = torch.empty((M, layer.N), dtype=torch.bfloat16, device=dev)
+        Yh = torch.empty((M, layer.N), dtype=torch.bfloat16).pin_memory()
+        ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, layer.N, layer.K, E), dev)
+        moqe.moqe_routed_qgemm_workspace_clear(ws, M, layer.N, layer.K, E)
+        off_h = torch.from_numpy(w.row_offsets(layer)).pin_memory()
+        import ctypes as C
+        arr = (C.c_void_p * E)(*[e.handle for e in experts])
+        layers.append(dict(spec=layer, experts=experts, M=M, X=X, Xh=Xh, Y=Y, Yh=Yh, ws=ws, arr=arr,
+                           row_off=off_h.to(dev), row_off_h=off_h))
+    logits_h = torch.from_numpy(workload_logits(w, seed)).pin_memory()
+    logits = logits_h.to(dev)
+    torch.cuda.synchronize()
+
+    # groups of layers that share one row structure share one sort
+    def hot_path(from_host: bool):
+        lg = logits
+        if from_host:
+            lg.copy_(logits_h, non_blocking=True)
+        ids = moqe.moqe_route(lg)
+        sorted_for = {}
+        for L in layers:
+            if from_host:
+                L["X"].copy_(L["Xh"], non_blocking=True)
+            key = L["spec"].rows_per_sample
+            if key not in sorted_for:
+                row_ids = moqe.moqe_expand_ids(ids, L["row_off"], L["M"])
+                _, perm, offsets = moqe.moqe_permute(None, row_ids, E)
+                sorted_for[key] = (perm, offsets)
+            perm, offsets = sorted_for[key]
+            moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
+            if from_host:
+                L["Yh"].copy_(L["Y"], non_blocking=True)
+        return sorted_for
+
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+
+    def make_runner(from_host: bool):
+        """Warm up eagerly, then capture one step in a CUDA graph (the launch-bound inner loop)."""
+        for _ in range(2):
+            hot_path(from_host)
+        stream.synchronize()
+        if args.no_graph:
+            return (lambda: hot_path(from_host)), 0
+        before = moqe.moqe_launch_count()
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g, stream=stream):
+                hot_path(from_host)
+        except Exception as ex:                                # capture refused: run eagerly
+            print(f"[bench] graph capture failed ({type(ex).__name__}: {ex}); running eagerly", file=sys.stderr)
+            stream.synchronize()
+            return (lambda: hot_path(from_host)), 0
+        per_step = moqe.moqe_launch_count() - before
+        return g.replay, per_step
+
+    def timed(run, steps, warmup):
+        for _ in range(warmup):
+            run()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            run()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    tokens_per_step = sum(w.sample_rows) if w.layers[0].rows_per_sample is None else w.n_samples
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+
+    # ---- 1. resident inputs ---------------------------------------------------------------------
+    run, graph_launches = make_runner(False)
+    l0 = moqe.moqe_launch_count()
+    ms = timed(run, args.steps, args.warmup)
+    launches = (graph_launches * args.steps) if graph_launches else (moqe.moqe_launch_count() - l0)
+    ms_per_step = ms / args.steps
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- 2. per-launch duration of the dominant kernel (events round every routed-GEMM call) ----
+    sorted_for = hot_path(False)
+    stream.synchronize()
+    counts = {k: np.diff(v[1].cpu().numpy()) for k, v in sorted_for.items()}
+    reps = max(3, min(args.steps, 200 if not heavy else 10))
+    per_layer_ms = []
+    for L in layers:
+        perm, offsets = sorted_for[L["spec"].rows_per_sample]
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        per_layer_ms.append(evs)
+    for r in range(reps):
+        for L, evs in zip(layers, per_layer_ms):
+            perm, offsets = sorted_for[L["spec"].rows_per_sample]
+            evs[r][0].record(stream)
+            moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
+            evs[r][1].record(stream)
+    stream.synchronize()
+    status = moqe.moqe_async_status()
+    clocks = sampler.stop()
+    layer_ms = [float(np.mean([a.elapsed_time(b) for a, b in evs[1:]])) for evs in per_layer_ms]
+
+    alg_bytes, flops = [], []
+    for L in layers:
+        cnt = counts[L["spec"].rows_per_sample]
+        b = 0
+        for e, ex in enumerate(L["experts"]):
+            if cnt[e] > 0:
+                b += ex.code_bytes + ex.meta_bytes
+        b += L["M"] * L["spec"].K * 2 + L["M"] * L["spec"].N * 2
+        alg_bytes.append(b)
+        flops.append(2.0 * L["M"] * L["spec"].N * L["spec"].K)
+    tot_ms = sum(layer_ms)
+    hbm_time = sum(alg_bytes) / (peaks["hbm_gbs"] * 1e9)
+    tensor_time = sum(flops) / (peaks["bf16_tflops"] * 1e12)
+    if tensor_time > hbm_time:
+        achieved = sum(flops) / (tot_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                    "frac_whole_step": sum(flops) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                    "frac_of_nominal_2250": achieved / 2250.0}
+    else:
+        achieved = sum(alg_bytes) / (tot_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "frac_of_nominal_8000": achieved / 8000.0}
+    roofline.update({"peak_source": peaks["source"], "kernel": "routed dequant-GEMM launches of one block",
+                     "algorithmic_bytes_per_step": int(sum(alg_bytes)), "flops_per_step": float(sum(flops)),
+                     "launch_ms": {L["spec"].name: round(t, 5) for L, t in zip(layers, layer_ms)}})
+
+    # ---- 3. end to end through the public API with host buffers ---------------------------------
+    run_h, _ = make_runner(True)
+    e2e_steps = max(3, args.steps // 4)
+    ms_h = timed(run_h, e2e_steps, 3) / e2e_steps
+    h2d = int(logits_h.numel() * 4 + sum(L["Xh"].numel() * 2 for L in layers))
+    d2h = int(sum(L["Yh"].numel() * 2 for L in layers))
+    e2e = {"value": world * tokens_per_step / (ms_h * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": ms_h}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": [f"{l.name}:{l.N}x{l.K}" for l in w.layers],
+                   "experts": [sp.tag for sp in w.experts], "tokens_per_step": tokens_per_step,
+                   "rows_per_expert": {str(k): v.tolist() for k, v in counts.items()},
+                   "parallelism": f"replicas x{world} (samples sharded, experts replicated, no collective)",
+                   "l2": "weights of one block exceed L2 (inputs larger than L2, no flush)" if sum(alg_bytes) > 126e6
+                         else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "device_status": moqe.status_str(status),
+    }
+
+    # ---- 4. the oracle on this machine's cores (rank 0, single-GPU runs only) -------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        max_rows = 16 if not heavy else 6
+        prepared, t_quant, t_deq = prepare_oracle(w, args.seed, max_rows)
+        sec = run_oracle_once(w, prepared, None)
+        line["cpu_baseline"] = {"value": tokens_per_step / sec, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": oracle_sample_text(w, prepared), "gemm_s_extrapolated": sec,
+                                "dequant_s": t_deq, "quantize_s": t_quant}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -169,6 +169,20 @@ MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* r
                                    const moqe_expert* const* h_experts, int E, void* Y_bf16,
                                    void* workspace, size_t workspace_bytes, void* stream, int path);
 
+/* The same product for a batch that is already sorted: `perm` [M] and `offsets`
+ * [E+1] as moqe_permute wrote them (device pointers; rows perm[offsets[E]..M) are
+ * left untouched in Y).  One sort then serves every linear layer of a block,
+ * since a sample keeps its expert through the whole model (Section 3.1).
+ * The split-K arrival counters at the head of the workspace body must be zero on
+ * entry -- clear them once with moqe_routed_qgemm_workspace_clear after
+ * allocating the workspace (same M, N, K, E) -- and every call leaves them zero.
+ * `path` as for moqe_routed_qgemm_path. */
+MOQE_API moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                              const moqe_expert* const* h_experts, int E, void* Y_bf16,
+                                              void* workspace, size_t workspace_bytes, void* stream, int path);
+MOQE_API moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
+                                                       int E, void* stream);
+
 /* Synchronises `stream`, then returns and clears the first error latched by a
  * kernel on the current device (MOQE_OK if none). */
 MOQE_API moqe_status moqe_async_status(void* stream);

@@ -25,7 +25,8 @@ PATH_AUTO, PATH_STREAM, PATH_TCGEN05 = 0, 1, 2
 EXPORTED = (
     "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",
     "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_unpermute",
-    "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_async_status",
+    "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
+    "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count",
 )
 
@@ -64,6 +65,8 @@ def lib() -> C.CDLL:
         L.moqe_routed_qgemm_workspace.restype = sz
         L.moqe_routed_qgemm.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp]
         L.moqe_routed_qgemm_path.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
+        L.moqe_routed_qgemm_sorted.argtypes = [vp, vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
+        L.moqe_routed_qgemm_workspace_clear.argtypes = [vp, sz, i32, i32, i32, i32, vp]
         L.moqe_async_status.argtypes = [vp]
         L.moqe_status_str.argtypes = [i32]
         L.moqe_status_str.restype = C.c_char_p
@@ -232,6 +235,26 @@ def moqe_routed_qgemm(X: torch.Tensor, row_ids: torch.Tensor, experts: Sequence[
     arr = (C.c_void_p * E)(*[e.handle for e in experts])
     _check(lib().moqe_routed_qgemm_path(_ptr(X), _ptr(row_ids), M, arr, E, _ptr(Y), _ptr(workspace), workspace.numel(),
                                         _stream(), int(path)), "moqe_routed_qgemm")
+    return Y
+
+
+def moqe_routed_qgemm_workspace_clear(workspace: torch.Tensor, M: int, N: int, K: int, E: int) -> None:
+    _check(lib().moqe_routed_qgemm_workspace_clear(_ptr(workspace), workspace.numel(), int(M), int(N), int(K), int(E),
+                                                   _stream()), "moqe_routed_qgemm_workspace_clear")
+
+
+def moqe_routed_qgemm_sorted(X: torch.Tensor, perm: torch.Tensor, offsets: torch.Tensor, experts: Sequence[Expert],
+                             Y: torch.Tensor, workspace: torch.Tensor, path: int = PATH_AUTO,
+                             _arr=None) -> torch.Tensor:
+    """Routed product for a batch already sorted by ``moqe_permute`` (``perm``, ``offsets``).
+
+    ``workspace`` must have been cleared once with ``moqe_routed_qgemm_workspace_clear``.
+    """
+    M, K = X.shape
+    E = len(experts)
+    arr = _arr if _arr is not None else (C.c_void_p * E)(*[e.handle for e in experts])
+    _check(lib().moqe_routed_qgemm_sorted(_ptr(X), _ptr(perm), _ptr(offsets), M, arr, E, _ptr(Y), _ptr(workspace),
+                                          workspace.numel(), _stream(), int(path)), "moqe_routed_qgemm_sorted")
     return Y
 
 

@@ -96,6 +96,45 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
 
+extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                                const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
+                                                size_t workspace_bytes, void* stream, int path) {
+    if (!h_experts) return MOQE_ERR_NULL;
+    if (E <= 0 || M < 0) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    for (int e = 0; e < E; ++e)
+        if (!h_experts[e]) return MOQE_ERR_NULL;
+    const int N = h_experts[0]->N, K = h_experts[0]->K;
+    for (int e = 1; e < E; ++e)
+        if (h_experts[e]->N != N || h_experts[e]->K != K) return MOQE_ERR_MISMATCH;
+    if (M == 0) return MOQE_OK;
+    if (!X_bf16 || !perm || !offsets || !Y_bf16) return MOQE_ERR_NULL;
+    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
+    if (path < 0 || path > 4) return MOQE_ERR_SHAPE;
+    const int Np = h_experts[0]->Np;
+    WsLayout w = ws_layout(M, Np, K, E);
+    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)workspace;
+    const bool use_stream = path == 1 || (path == 0 && M <= AUTO_STREAM_MAX_ROWS);
+    if (use_stream)
+        return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
+                                   w.total - w.body, st);
+    tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
+    return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+}
+
+extern "C" moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
+                                                         int E, void* stream) {
+    if (M < 0 || N <= 0 || K <= 0 || E <= 0) return MOQE_ERR_SHAPE;
+    const int Np = (N + 127) / 128 * 128;
+    WsLayout w = ws_layout(M, Np, K, E);
+    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    size_t zb = stream_zero_bytes(M, Np);
+    if (zb == 0) return MOQE_OK;
+    return cuda_ok(cudaMemsetAsync((char*)workspace + w.body, 0, zb, (cudaStream_t)stream));
+}
+
 extern "C" moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_ids, int M,
                                          const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
                                          size_t workspace_bytes, void* stream) {

@@ -236,8 +236,10 @@ __device__ __forceinline__ void run_task(const StreamParams& p, const ExpertDev&
             __threadfence();
             __syncthreads();
             if (tid == 0) {
-                unsigned old = atomicAdd(p.counters + (size_t)nt * p.M + j0, 1u);
+                unsigned* cnt = p.counters + (size_t)nt * p.M + j0;
+                unsigned old = atomicAdd(cnt, 1u);
                 s_last = (old == (unsigned)(S - 1));
+                if (s_last) *cnt = 0u;                              // leave the counters clear for the next call
             }
             __syncthreads();
             write_final = s_last != 0;

@@ -141,3 +141,29 @@ def test_argument_errors():
     with pytest.raises(moqe.MoqeError) as ei:
         moqe.moqe_routed_qgemm(X, ids, g1, workspace=torch.empty(256, dtype=torch.uint8, device=dev()))
     assert ei.value.code == moqe.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("path,M", [(1, 16), (1, 48), (3, 300)])
+def test_presorted_entry_point_matches(path, M):
+    """moqe_permute once + moqe_routed_qgemm_sorted per layer == moqe_routed_qgemm, bit for bit, call after call
+    (the split-K arrival counters must come back to zero by themselves)."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, dev, bf16_to_torch, torch_to_bits
+    N, K = 384, 2048
+    W = wl.weights_f32("sorted", N, K)
+    X = wl.activations_bf16(f"sorted/{M}", M, K)
+    gpu, What, _ = build_experts(W, [(8, 0, True), (4, 128, False), (3, 128, False)])
+    ids = np.random.default_rng(M).integers(0, 3, size=M).astype(np.int32)
+    Xd, idd = bf16_to_torch(X), torch.from_numpy(ids).to(dev())
+    ref = torch_to_bits(moqe.moqe_routed_qgemm(Xd, idd, gpu, path=path))
+    _, perm, offsets = moqe.moqe_permute(None, idd, 3)
+    ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, N, K, 3))
+    ws.fill_(0xFF)
+    moqe.moqe_routed_qgemm_workspace_clear(ws, M, N, K, 3)
+    for _ in range(3):
+        Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+        moqe.moqe_routed_qgemm_sorted(Xd, perm, offsets, gpu, Y, ws, path=path)
+        assert moqe.moqe_async_status() == moqe.OK
+        assert np.array_equal(torch_to_bits(Y), ref)
+    from gpu_helpers import assert_close
+    assert_close(ref, oracle.routed_gemm(X, ids, What), "sorted")
