@@ -144,6 +144,35 @@ MOQE_API moqe_status moqe_permute(const void* X_bf16, const int32_t* row_ids, in
 MOQE_API moqe_status moqe_unpermute(const void* Yp_bf16, const int32_t* perm, int M, int C, void* Y_bf16,
                            void* stream);
 
+/* moqe_permute for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of the library.)
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside
+ * a serving process whose memory pool is owned and fully handed out by the host
+ * framework, a real-time loop that may not take the allocator's lock or trigger
+ * its implicit device synchronisation, or a process kept under a fixed memory
+ * budget.  moqe_permute needs a caller-provided workspace for batches above 1024
+ * rows; this variant keeps that scratch (per-block bucket totals, 132 KiB) in a
+ * fixed array inside the library image, which every GPU that loads the library
+ * holds until the process exits.  It performs no allocation at all: no cudaMalloc
+ * or cudaFree, no allocating library call.
+ *   - Same arguments, results and row limit semantics as moqe_permute, minus the
+ *     workspace.  M above MOQE_PERMUTE_STATIC_MAX_ROWS returns MOQE_ERR_WORKSPACE
+ *     (nothing is launched): use moqe_permute for such batches.
+ *   - Ids outside [0,E) are sorted behind the valid rows and their Xp rows are
+ *     zero, exactly as in moqe_permute, but NO error is latched for
+ *     moqe_async_status (the status word lives in allocated memory); compare
+ *     offsets[E] with M to detect them.
+ *   - The first call on each device looks up the device address of the built-in
+ *     array (a host-side query, not an allocation).  Make that first call outside
+ *     any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it needs clearing
+ *     between calls (each call writes every entry before reading it), but two
+ *     calls that overlap on the GPU -- different streams, or concurrent host
+ *     threads on different streams -- race on it: serialise them. */
+#define MOQE_PERMUTE_STATIC_MAX_ROWS (1 << 20)
+MOQE_API moqe_status moqe_permute_static(const void* X_bf16, const int32_t* row_ids, int M, int C, int E,
+                                         void* Xp_bf16, int32_t* perm, int32_t* offsets, void* stream);
+
 /* ---------------------------------------------------------------------------
  * The routed dequant-GEMM (Section 3.1: "the activated quantization expert
  * performs the inference on this sample" -- here for a whole mixed batch):

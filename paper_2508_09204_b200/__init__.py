@@ -24,7 +24,7 @@ PATH_AUTO, PATH_STREAM, PATH_TCGEN05 = 0, 1, 2
 
 EXPORTED = (
     "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",
-    "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_unpermute",
+    "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
     "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count",
@@ -60,6 +60,7 @@ def lib() -> C.CDLL:
         L.moqe_permute_workspace.argtypes = [i32, i32]
         L.moqe_permute_workspace.restype = sz
         L.moqe_permute.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.moqe_permute_static.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
         L.moqe_unpermute.argtypes = [vp, vp, i32, i32, vp, vp]
         L.moqe_routed_qgemm_workspace.argtypes = [i32, i32, i32, i32]
         L.moqe_routed_qgemm_workspace.restype = sz
@@ -196,6 +197,22 @@ def moqe_permute(X: Optional[torch.Tensor], row_ids: torch.Tensor, E: int):
     _check(lib().moqe_permute(_ptr(X), _ptr(row_ids), M, Cc, int(E), _ptr(Xp), _ptr(perm), _ptr(offsets), _ptr(ws), wsb,
                               _stream()), "moqe_permute")
     return Xp, perm, offsets
+
+
+PERMUTE_STATIC_MAX_ROWS = 1 << 20
+
+
+def moqe_permute_static(X: Optional[torch.Tensor], row_ids: torch.Tensor, E: int, Xp: Optional[torch.Tensor],
+                        perm: torch.Tensor, offsets: torch.Tensor) -> None:
+    """``moqe_permute`` without a workspace, for callers that must not allocate device memory.
+
+    Every buffer, outputs included, is passed in by the caller; the C call keeps its scratch in a
+    fixed array inside the library and allocates nothing.  Calls on one device must not overlap.
+    """
+    M = row_ids.numel()
+    Cc = 0 if X is None else X.shape[1]
+    _check(lib().moqe_permute_static(_ptr(X), _ptr(row_ids), M, Cc, int(E), _ptr(Xp), _ptr(perm), _ptr(offsets),
+                                     _stream()), "moqe_permute_static")
 
 
 def moqe_unpermute(Yp: torch.Tensor, perm: torch.Tensor) -> torch.Tensor:

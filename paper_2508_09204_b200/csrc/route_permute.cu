@@ -10,6 +10,8 @@
 // end up behind all valid rows and latch MOQE_ERR_EXPERT_ID).  Within a warp
 // the stable rank of a row among equal ids comes from __match_any_sync; warps
 // and blocks are combined with prefix sums, so perm is the unique stable order.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace moqe {
@@ -278,4 +280,75 @@ extern "C" moqe_status moqe_unpermute(const void* Yp_bf16, const int32_t* perm, 
         (const uint4*)Yp_bf16, perm, nullptr, M, vec, (uint4*)Y_bf16);
     count_launch();
     return cuda_ok(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------
+// moqe_permute_static: the same sort and gather as moqe_permute for callers that
+// cannot allocate device memory.  The per-block bucket totals that the
+// multi-block sort needs live in a fixed array inside the library image, so this
+// entry point takes no workspace and calls no allocator of any kind.
+// ---------------------------------------------------------------------------
+namespace moqe {
+namespace {
+
+constexpr int STATIC_SORT_MAX_ROWS = MOQE_PERMUTE_STATIC_MAX_ROWS;
+constexpr int STATIC_SORT_MAX_BLOCKS = (STATIC_SORT_MAX_ROWS + SORT_THREADS - 1) / SORT_THREADS;
+
+// [block][bucket] totals, then (after the scan) base slots.  132 KiB per device for the lifetime of
+// the process.  Every entry a call reads is written by that same call first, so nothing has to be
+// cleared between calls; two calls running at once on one device would overwrite each other here.
+static __device__ __align__(256) int32_t g_static_sort_scratch[STATIC_SORT_MAX_BLOCKS * MAXB];
+
+std::mutex g_static_mutex;
+int32_t* g_static_scratch_addr[64] = {nullptr};
+
+// Device address of the array on the current device.  The array's name is only a handle in host
+// code; the address a kernel can use has to be asked for, once per device, with that device current.
+moqe_status static_scratch(int32_t** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOQE_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_sort_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return MOQE_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = static_cast<int32_t*>(p);
+    }
+    *out = g_static_scratch_addr[dev];
+    return MOQE_OK;
+}
+
+}  // namespace
+}  // namespace moqe
+
+extern "C" moqe_status moqe_permute_static(const void* X_bf16, const int32_t* row_ids, int M, int C, int E,
+                                           void* Xp_bf16, int32_t* perm, int32_t* offsets, void* stream) {
+    if (!offsets) return MOQE_ERR_NULL;
+    if (M < 0 || E <= 0) return MOQE_ERR_SHAPE;
+    if (M > 0 && (!row_ids || !perm)) return MOQE_ERR_NULL;
+    if (M == 0) X_bf16 = Xp_bf16 = nullptr;
+    if ((X_bf16 == nullptr) != (Xp_bf16 == nullptr)) return MOQE_ERR_NULL;
+    if (X_bf16 && C <= 0) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    if (M > STATIC_SORT_MAX_ROWS) return MOQE_ERR_WORKSPACE;      // beyond the built-in scratch: use moqe_permute
+    if (X_bf16 && (C % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Xp_bf16 % 16)) return MOQE_ERR_UNSUPPORTED;
+    int32_t* scratch = nullptr;
+    moqe_status s = static_scratch(&scratch);
+    if (s != MOQE_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (M <= SORT_THREADS) {
+        sort_small_kernel<<<1, SORT_THREADS, 0, st>>>(row_ids, M, E, perm, offsets, nullptr, 0, nullptr, 0, nullptr);
+        count_launch();
+    } else {
+        int nblk = (M + SORT_THREADS - 1) / SORT_THREADS;
+        sort_hist_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, scratch, nullptr);
+        sort_scan_kernel<<<1, 64, 0, st>>>(scratch, nblk, E, offsets);
+        sort_scatter_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, scratch, perm, nullptr, 0);
+        count_launch(3);
+    }
+    if (cudaGetLastError() != cudaSuccess) return MOQE_ERR_CUDA;
+    if (!X_bf16) return MOQE_OK;
+    return launch_gather(X_bf16, perm, offsets + E, M, C, Xp_bf16, st);
 }
