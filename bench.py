@@ -223,6 +223,7 @@ def main():
     ap.add_argument("--seed", type=int, default=wl.BASE_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--tune", action="append", default=[], help="key=value passed to moqe_tune (measurement knob)")
     args = ap.parse_args()
     w = wl.get(args.workload)
     heavy = w.kind in ("prefill", "mixed", "conv")
@@ -243,6 +244,9 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the routed path has no CPU fallback")
     moqe.lib()                                              # fails loudly if the CUDA library is not built
+    for kv in args.tune:
+        k, v = kv.split("=")
+        moqe.moqe_tune(k, int(v))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

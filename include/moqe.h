@@ -218,6 +218,13 @@ MOQE_API moqe_status moqe_async_status(void* stream);
 
 MOQE_API const char* moqe_status_str(moqe_status s);
 
+/* Measurement knobs (process-wide, not thread-safe; defaults are the tuned values):
+ *   "stream_tile_cost_w8" / "_w4" / "_w3" : relative cost of one packed 128x128 tile of
+ *                            that bit-width in the streaming kernel's work split
+ *                            (defaults 9 / 5 / 4: bytes in 2 KiB units plus a fixed part).
+ * Unknown key: MOQE_ERR_UNSUPPORTED. */
+MOQE_API moqe_status moqe_tune(const char* key, int value);
+
 /* Number of kernels this library has launched so far in this process. */
 MOQE_API unsigned long long moqe_launch_count(void);
 

@@ -27,7 +27,7 @@ EXPORTED = (
     "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
     "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
-    "moqe_status_str", "moqe_launch_count",
+    "moqe_status_str", "moqe_launch_count", "moqe_tune",
 )
 
 
@@ -71,6 +71,7 @@ def lib() -> C.CDLL:
         L.moqe_async_status.argtypes = [vp]
         L.moqe_status_str.argtypes = [i32]
         L.moqe_status_str.restype = C.c_char_p
+        L.moqe_tune.argtypes = [C.c_char_p, i32]
         L.moqe_launch_count.argtypes = []
         L.moqe_launch_count.restype = C.c_ulonglong
         _lib = L
@@ -278,6 +279,10 @@ def moqe_routed_qgemm_sorted(X: torch.Tensor, perm: torch.Tensor, offsets: torch
 def moqe_async_status() -> int:
     """Synchronises the current stream and returns (and clears) the latched device error."""
     return int(lib().moqe_async_status(_stream()))
+
+
+def moqe_tune(key: str, value: int) -> None:
+    _check(lib().moqe_tune(key.encode(), int(value)), "moqe_tune")
 
 
 def moqe_launch_count() -> int:

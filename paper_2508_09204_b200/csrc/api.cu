@@ -1,6 +1,7 @@
 // C-ABI entry points that tie the kernels together: the routed dequant-GEMM
 // call, the device status word, status strings and the launch counter.
 #include <atomic>
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -139,6 +140,14 @@ extern "C" moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_
                                          const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
                                          size_t workspace_bytes, void* stream) {
     return moqe_routed_qgemm_path(X_bf16, row_ids, M, h_experts, E, Y_bf16, workspace, workspace_bytes, stream, 0);
+}
+
+extern "C" moqe_status moqe_tune(const char* key, int value) {
+    if (!key) return MOQE_ERR_NULL;
+    if (!strcmp(key, "stream_tile_cost_w8")) { stream_set_tile_cost(8, value); return MOQE_OK; }
+    if (!strcmp(key, "stream_tile_cost_w4")) { stream_set_tile_cost(4, value); return MOQE_OK; }
+    if (!strcmp(key, "stream_tile_cost_w3")) { stream_set_tile_cost(3, value); return MOQE_OK; }
+    return MOQE_ERR_UNSUPPORTED;
 }
 
 extern "C" moqe_status moqe_async_status(void* stream) {

@@ -5,12 +5,14 @@
 // (Np, Kp); padded codes are 0 and padded scales are 0.
 //
 //   tile (nt, kb)   : 128 output channels x 128 input features, contiguous,
-//                     tiles ordered [nt][kb]  ->  one bulk copy per tile
+//                     tiles ordered [nt][kb], tile_stride bytes apart  ->  one bulk copy per tile
 //   blob  nb (0..7) : 16 channels x 128 k inside the tile, contiguous
 //   piece (row, q)  : 32 codes of one channel: k = 128*kb + 32*G + 8*q + t,
 //                     G = 0..3 ("chunk": 8 consecutive k), t = 0..7
 //                     row = 16*nb + 8*half + r
-//   slot            : q*8 + r (32 slots per half)
+//   slot            : q*8 + (r ^ 2q) (32 slots per half).  The xor makes the 16-byte slots
+//                     bank-conflict free for both readers: lanes (r, q) = (lane/4, lane%4) of an
+//                     mma.sync fragment and lanes (q, r') = (lane/8, lane%8) of the UMMA dequant warps
 //
 //   W4  blob 1024 B : [half][slot] 16 B = 4 words, word G = chunk G; code t sits in
 //                     nibble t/2 (t even) or 4 + t/2 (t odd), so that
@@ -26,9 +28,12 @@
 // m16n8k16 fragment owns 4 k of every MMA (chunk halves), and every unpacked
 // word is one 16-byte chunk of 8 consecutive k of a K-major UMMA operand tile.
 //
-//   scales_t [Gp][Np] fp16, zeros_t [Gp][Np] bf16 (the integer zero-point;
-//   absent for symmetric experts whose zero-point is 2^(bits-1)).
-//   Gp = 1 for per-channel experts, else Kp / group.
+// Scales and zero-points travel WITH the tile they belong to, so that one bulk copy brings
+// everything a k-block needs: a tile is [codes][meta], meta = for each of the tile's groups
+// (group 32: 4, group 64: 2, group >= 128: 1 -- a group wider than 128 k is repeated in each
+// tile it spans) 128 fp16 scales followed, for asymmetric experts, by 128 bf16 zero-points
+// (the integer zero-point; symmetric experts use 2^(bits-1)).  Per-channel experts have no
+// per-tile meta: their scales / zero-points are plain [Np] arrays.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -37,29 +42,49 @@
 
 #include "../../include/moqe.h"
 
+static __host__ __device__ inline int moqe_blob_bytes(int bits) { return 16 * 128 * bits / 8; }
+static __host__ __device__ inline int moqe_tile_bytes(int bits) { return 128 * 128 * bits / 8; }   // codes only
+static __host__ __device__ inline int moqe_groups_per_tile(int group) { return group == 0 ? 0 : (group >= 128 ? 1 : 128 / group); }
+static __host__ __device__ inline int moqe_meta_group_bytes(int has_zeros) { return has_zeros ? 512 : 256; }
+static __host__ __device__ inline int moqe_tile_stride(int bits, int group, int has_zeros) {
+    return moqe_tile_bytes(bits) + moqe_groups_per_tile(group) * moqe_meta_group_bytes(has_zeros);
+}
+
+// What a kernel needs to know about one expert's device buffers.
+struct ExpertDev {
+    const uint8_t* tiles;           // [nt][kb] tiles of tile_stride bytes: codes then per-tile scales / zero-points
+    const __half* scales_pc;        // per-channel experts only: [Np]
+    const __nv_bfloat16* zeros_pc;  // per-channel asymmetric experts only: [Np]
+    int bits;
+    int group;                      // 0 = per channel
+    int has_zeros;                  // asymmetric
+    int tile_stride;
+};
+
+// scale / zero-point of channel row (0..127 inside the tile) for sub-group j of a tile in shared or global memory
+static __device__ inline const __half* moqe_tile_scales(const unsigned char* tile, int bits, int has_zeros, int j) {
+    return reinterpret_cast<const __half*>(tile + moqe_tile_bytes(bits) + j * moqe_meta_group_bytes(has_zeros));
+}
+static __device__ inline const __nv_bfloat16* moqe_tile_zeros(const unsigned char* tile, int bits, int j) {
+    return reinterpret_cast<const __nv_bfloat16*>(tile + moqe_tile_bytes(bits) + j * 512 + 256);
+}
+
 struct moqe_expert {
     int N, K, bits, group, sym;   // as given by the caller (group 0 = per channel)
     int Np, Kp;                   // padded to multiples of 128
     int G;                        // real groups per row  (1 when group == 0)
-    int Gp;                       // allocated groups per row
     int device;
-    uint8_t* codes;               // packed tiles
-    __half* scales_t;             // [Gp][Np]
-    __nv_bfloat16* zeros_t;       // [Gp][Np], nullptr when symmetric
-    size_t codes_alloc, meta_alloc;
+    uint8_t* tiles;               // packed tiles with their meta
+    __half* scales_pc;            // per-channel: [Np], else nullptr
+    __nv_bfloat16* zeros_pc;      // per-channel asymmetric: [Np], else nullptr
+    size_t tiles_alloc, pc_alloc;
+    ExpertDev dev() const {
+        ExpertDev d;
+        d.tiles = tiles; d.scales_pc = scales_pc; d.zeros_pc = zeros_pc; d.bits = bits; d.group = group;
+        d.has_zeros = sym ? 0 : 1; d.tile_stride = moqe_tile_stride(bits, group, d.has_zeros);
+        return d;
+    }
 };
-
-// What a GEMM kernel needs to know about one expert.
-struct ExpertDev {
-    const uint8_t* codes;
-    const __half* scales_t;
-    const __nv_bfloat16* zeros_t;   // nullptr: symmetric
-    int bits;
-    int group;                      // 0 = per channel
-};
-
-static __host__ __device__ inline int moqe_blob_bytes(int bits) { return 16 * 128 * bits / 8; }
-static __host__ __device__ inline int moqe_tile_bytes(int bits) { return 128 * 128 * bits / 8; }
 
 namespace moqe {
 
@@ -83,6 +108,7 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
                                 const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes,
                                 cudaStream_t st);
 size_t stream_zero_bytes(int M, int Np);
+void stream_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split (measurement knob)
 
 // qgemm_tcgen05.cu
 void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)

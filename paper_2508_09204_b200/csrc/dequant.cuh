@@ -60,6 +60,27 @@ __device__ __forceinline__ void unpack_chunk(const uint32_t (&w)[PieceWords<BITS
     }
 }
 
+// Chunk G of a 4- or 3-bit piece as the bf16 numbers 128 + c (no zero-point): two instructions per pair.
+// The caller removes (128 + z) * sum_k X with the help of a second MMA against an all-ones operand.
+template <int BITS, int G>
+__device__ __forceinline__ void unpack_chunk_biased(const uint32_t (&w)[PieceWords<BITS>::n], uint32_t (&out)[4]) {
+    static_assert(BITS == 4 || BITS == 3, "biased form exists for 4- and 3-bit codes");
+    if constexpr (BITS == 4) {
+        const uint32_t v = w[G];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = ((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = 4 * G + i;
+            uint32_t v;
+            if (p < 15) v = (w[p / 5] >> (3 * (p % 5))) & 0x00070007u;
+            else v = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u);
+            out[i] = v | 0x43004300u;
+        }
+    }
+}
+
 // group index of chunk G of k-block kb:  per channel -> 0;  g = 32 -> 4*kb + G;  g = 64 -> 2*kb + G/2;
 // g >= 128 -> 128*kb / g
 __device__ __forceinline__ int group_of_chunk(int group, int kb, int G) {

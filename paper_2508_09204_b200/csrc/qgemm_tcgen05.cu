@@ -31,6 +31,7 @@
 #include <type_traits>
 
 #include "dequant.cuh"
+#include "ptx.cuh"
 
 namespace moqe {
 namespace {
@@ -39,7 +40,7 @@ constexpr int TC_THREADS = 512;
 constexpr int NS = 3;                 // operand stages (A tile + X tile, 64 k each)
 constexpr int NWS = 3;                // packed-weight stages (128 k each)
 constexpr int A_STAGE_BYTES = 128 * 128;          // 128 channels x 64 bf16
-constexpr int W_STAGE_BYTES = 128 * 128;          // largest packed tile (W8)
+constexpr int W_STAGE_BYTES = 128 * 128 + 4 * 512;   // largest packed tile (W8 codes) + largest per-tile meta
 constexpr int XBOX_ROWS = 64;
 constexpr int XBOX_BYTES = XBOX_ROWS * 128;
 
@@ -67,63 +68,12 @@ struct Smem {
     static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
 };
 
-// ---------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-
-// Bounded wait.  Returns false if the CTA is aborting (someone's wait ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_test(bar, parity)) return true;
-    unsigned long long t0 = global_ns();
-    for (unsigned spin = 1;; ++spin) {
-        if (mbar_test(bar, parity)) return true;
-        if ((spin & 63u) == 0) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                latch_status(status, (int)MOQE_ERR_TIMEOUT);
-                return false;
-            }
-            __nanosleep(64);
-        }
-    }
-}
-
+// ---------------------------------------------------------------------------- PTX wrappers (tensor-core side)
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -187,12 +137,6 @@ __device__ __forceinline__ bool decode_tile(const int* s_off, int E, int n_tiles
     return false;
 }
 
-struct Ring {
-    int stage = 0;
-    uint32_t phase = 0;
-    __device__ __forceinline__ void advance(int n) { if (++stage == n) { stage = 0; phase ^= 1u; } }
-};
-
 // ---------------------------------------------------------------------------- dequant role
 template <int BITS>
 __device__ __forceinline__ void load_piece_smem(const unsigned char* blob, int half, int slot, uint32_t (&w)[PieceWords<BITS>::n]) {
@@ -218,37 +162,42 @@ __device__ __forceinline__ void load_piece_smem(const unsigned char* blob, int h
 // One k-block (128 k) of one tile: wait for the packed tile, pull this thread's four pieces into
 // registers, release the packed stage, then fill the two 64-k operand stages.
 template <int BITS>
-__device__ __forceinline__ bool dequant_kblock(const ExpertDev& ex, int Np, int nt, int kb, unsigned char* smem_w,
+__device__ __forceinline__ bool dequant_kblock(const ExpertDev& ex, int nt, unsigned char* smem_w,
                                                unsigned char* smem_a_base, uint32_t bar_wfull, uint32_t bar_wempty,
                                                uint32_t wphase, uint32_t bar_empty0, uint32_t bar_afull0, Ring& ring,
                                                volatile int* abort_flag, int* status) {
     const int lane = threadIdx.x & 31, dw = (threadIdx.x >> 5) & 3;
-    const int q = lane >> 3, r = lane & 7;
+    const int q = lane >> 3, r = (lane & 7) ^ (2 * q);          // slot = lane holds piece (q, r)
     constexpr int NWORDS = PieceWords<BITS>::n;
     const float sym_z = (float)(1 << (BITS - 1));
-    // zero-points of the four pieces' channels, per chunk
+    // zero-points of the four pieces' channels, per chunk: per-channel experts read theirs from global memory
+    // before the wait, the others from the tile's own meta once it has landed
     float z[4][4];
+    const bool tile_zeros = ex.has_zeros && ex.group != 0;
 #pragma unroll
     for (int pi = 0; pi < 4; ++pi) {
         const int n = nt * 128 + (2 * dw + (pi >> 1)) * 16 + (pi & 1) * 8 + r;
-        if (!ex.zeros_t) {
+        const float v = (ex.has_zeros && ex.group == 0) ? __bfloat162float(ex.zeros_pc[n]) : sym_z;
 #pragma unroll
-            for (int G = 0; G < 4; ++G) z[pi][G] = sym_z;
-        } else if (ex.group == 32 || ex.group == 64) {
-#pragma unroll
-            for (int G = 0; G < 4; ++G)
-                z[pi][G] = __bfloat162float(ex.zeros_t[(size_t)group_of_chunk(ex.group, kb, G) * Np + n]);
-        } else {
-            float v = __bfloat162float(ex.zeros_t[(size_t)group_of_chunk(ex.group, kb, 0) * Np + n]);
-#pragma unroll
-            for (int G = 0; G < 4; ++G) z[pi][G] = v;
-        }
+        for (int G = 0; G < 4; ++G) z[pi][G] = v;
     }
     if (!mbar_wait(bar_wfull, wphase, abort_flag, status)) return false;
     uint32_t w[4][NWORDS];
 #pragma unroll
     for (int pi = 0; pi < 4; ++pi)
         load_piece_smem<BITS>(smem_w + (2 * dw + (pi >> 1)) * moqe_blob_bytes(BITS), pi & 1, lane, w[pi]);
+    if (tile_zeros) {
+        const int per_tile = moqe_groups_per_tile(ex.group);
+#pragma unroll
+        for (int pi = 0; pi < 4; ++pi) {
+            const int row = (2 * dw + (pi >> 1)) * 16 + (pi & 1) * 8 + r;
+#pragma unroll
+            for (int G = 0; G < 4; ++G) {
+                const int j = per_tile == 4 ? G : (per_tile == 2 ? (G >> 1) : 0);
+                z[pi][G] = __bfloat162float(moqe_tile_zeros(smem_w, BITS, j)[row]);
+            }
+        }
+    }
     mbar_arrive(bar_wempty);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -332,8 +281,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
             bool ok = true;
             for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
                 const ExpertDev& ex = p.ex[ti.e];
-                const uint32_t bytes = (uint32_t)moqe_tile_bytes(ex.bits);
-                const uint8_t* src = ex.codes + (size_t)ti.nt * p.KB * bytes;
+                const uint32_t bytes = (uint32_t)ex.tile_stride;          // codes + the tile's scales / zero-points
+                const uint8_t* src = ex.tiles + (size_t)ti.nt * p.KB * bytes;
                 for (int kb = 0; kb < p.KB; ++kb) {
                     if (!(ok = mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status))) break;
                     const uint32_t full = bar_wfull + 8 * ring.stage;
@@ -393,11 +342,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                 unsigned char* sw = smem + L::w_off + wring.stage * W_STAGE_BYTES;
                 const uint32_t wf = bar_wfull + 8 * wring.stage, we = bar_wempty + 8 * wring.stage;
                 if (ex.bits == 4)
-                    ok = dequant_kblock<4>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                    ok = dequant_kblock<4>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 else if (ex.bits == 8)
-                    ok = dequant_kblock<8>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                    ok = dequant_kblock<8>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 else
-                    ok = dequant_kblock<3>(ex, p.Np, ti.nt, kb, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                    ok = dequant_kblock<3>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 wring.advance(NWS);
             }
         }
@@ -426,8 +375,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
             const int group_k = ex.group == 0 ? p.KB * 128 : min(ex.group, 128);
             const int ngroups = p.KB * 128 / group_k;
             for (int gi = 0; ok && gi < ngroups; ++gi) {
-                const int sidx = ex.group == 0 ? 0 : (ex.group >= 128 ? gi * 128 / ex.group : gi);
-                const float s = __half2float(ex.scales_t[(size_t)sidx * p.Np + n]);
+                float s;
+                if (ex.group == 0) {
+                    s = __half2float(ex.scales_pc[n]);
+                } else {                                   // the scale sits in the meta of the tile the group lies in
+                    const int per_tile = moqe_groups_per_tile(ex.group);
+                    const unsigned char* tile = ex.tiles + ((size_t)ti.nt * p.KB + gi / per_tile) * (size_t)ex.tile_stride;
+                    s = __half2float(moqe_tile_scales(tile, ex.bits, ex.has_zeros, gi % per_tile)[row]);
+                }
                 if (!(ok = mbar_wait(bar_accfull + 8 * buf, acc_use[buf] & 1u, s_abort, p.status))) break;
                 tc_fence_after();
 #pragma unroll
@@ -521,11 +476,7 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
         return MOQE_ERR_CUDA;
     TcParams p;
     for (int e = 0; e < E; ++e) {
-        p.ex[e].codes = ex[e]->codes;
-        p.ex[e].scales_t = ex[e]->scales_t;
-        p.ex[e].zeros_t = ex[e]->zeros_t;
-        p.ex[e].bits = ex[e]->bits;
-        p.ex[e].group = ex[e]->group;
+        p.ex[e] = ex[e]->dev();
     }
     p.perm = perm; p.offsets = offsets; p.Y = (uint16_t*)Y; p.status = device_status_word();
     p.M = M; p.N = N; p.K = K; p.Np = ex[0]->Np; p.KB = ex[0]->Kp / 128; p.E = E; p.n_tiles = p.Np / 128;

@@ -113,7 +113,7 @@ __device__ __forceinline__ void load_piece(const uint8_t* blob, int half, int sl
 
 // piece id -> coordinates.  Pieces are numbered so that consecutive threads own
 // consecutive slots of one half of one blob (coalesced packed accesses).
-struct PieceCoord { int nt, kb, nb, half, slot, q, r, n; size_t blob_index; };
+struct PieceCoord { int nt, kb, nb, half, slot, q, r, n; size_t tile_index; };
 __device__ __forceinline__ PieceCoord piece_coord(long long pid, int KB) {
     PieceCoord pc;
     pc.slot = (int)(pid & 31);
@@ -123,21 +123,45 @@ __device__ __forceinline__ PieceCoord piece_coord(long long pid, int KB) {
     pc.kb = (int)(tile % KB);
     pc.nt = (int)(tile / KB);
     pc.q = pc.slot >> 3;
-    pc.r = pc.slot & 7;
+    pc.r = (pc.slot & 7) ^ (2 * pc.q);
     pc.n = pc.nt * 128 + pc.nb * 16 + pc.half * 8 + pc.r;
-    pc.blob_index = (size_t)tile * 8 + pc.nb;
+    pc.tile_index = (size_t)tile;
     return pc;
 }
 
 // ---------------------------------------------------------------------------
 // K1a: per (channel, group) scale and zero-point.  One warp per group.
 // ---------------------------------------------------------------------------
-__global__ void rtn_scales_kernel(const float* __restrict__ W, int N, int K, int bits, int g, int G, int sym, int Np,
-                                  __half* __restrict__ scales_t, __nv_bfloat16* __restrict__ zeros_t) {
+// where the scale / zero-point of (channel n, canonical group gi) live; a group wider than 128 k is
+// stored once per tile it spans: copy 0 .. copies-1
+struct MetaSlot { __half* s; __nv_bfloat16* z; };
+__device__ __forceinline__ int meta_copies(int group) { return group > 128 ? group / 128 : 1; }
+__device__ __forceinline__ MetaSlot meta_slot(uint8_t* tiles, __half* scales_pc, __nv_bfloat16* zeros_pc, int bits, int group,
+                                              int has_zeros, int KB, int n, int gi, int copy) {
+    MetaSlot m;
+    if (group == 0) {
+        m.s = scales_pc + n;
+        m.z = has_zeros ? zeros_pc + n : nullptr;
+        return m;
+    }
+    const int per_tile = moqe_groups_per_tile(group);
+    const int kb = group >= 128 ? gi * (group / 128) + copy : gi / per_tile;
+    const int j = group >= 128 ? 0 : gi % per_tile;
+    uint8_t* tile = tiles + ((size_t)(n >> 7) * KB + kb) * (size_t)moqe_tile_stride(bits, group, has_zeros);
+    uint8_t* meta = tile + moqe_tile_bytes(bits) + j * moqe_meta_group_bytes(has_zeros);
+    m.s = reinterpret_cast<__half*>(meta) + (n & 127);
+    m.z = has_zeros ? reinterpret_cast<__nv_bfloat16*>(meta + 256) + (n & 127) : nullptr;
+    return m;
+}
+
+__global__ void rtn_scales_kernel(const float* __restrict__ W, int N, int K, int bits, int group, int G, int sym, int KB,
+                                  uint8_t* __restrict__ tiles, __half* __restrict__ scales_pc,
+                                  __nv_bfloat16* __restrict__ zeros_pc) {
     long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (warp >= (long long)N * G) return;
     int n = (int)(warp / G), gi = (int)(warp % G);
+    const int g = group ? group : K;
     const float* w = W + (size_t)n * K + (size_t)gi * g;
     float lo = 0.f, hi = 0.f, a = 0.f;
     for (int k = lane; k < g; k += 32) {
@@ -159,11 +183,15 @@ __global__ void rtn_scales_kernel(const float* __restrict__ W, int N, int K, int
     __half sh = __float2half_rn(s32);
     float s = __half2float(sh);
     if (!(s > 0.f) || isinf(s)) { sh = __float2half_rn(1.0f); s = 1.0f; }
-    scales_t[(size_t)gi * Np + n] = sh;
+    int z = 0;
     if (!sym) {
-        int z = (int)rintf(__fdiv_rn(-lo, s));
+        z = (int)rintf(__fdiv_rn(-lo, s));
         z = max(0, min(L, z));
-        zeros_t[(size_t)gi * Np + n] = __float2bfloat16_rn((float)z);   // exact: z <= 255
+    }
+    for (int c = 0; c < meta_copies(group); ++c) {
+        MetaSlot m = meta_slot(tiles, scales_pc, zeros_pc, bits, group, !sym, KB, n, gi, c);
+        *m.s = sh;
+        if (!sym) *m.z = __float2bfloat16_rn((float)z);            // exact: z <= 255
     }
 }
 
@@ -172,9 +200,8 @@ __global__ void rtn_scales_kernel(const float* __restrict__ W, int N, int K, int
 // ---------------------------------------------------------------------------
 template <int BITS, bool FROM_CODES>
 __global__ void encode_pack_kernel(const float* __restrict__ W, const uint8_t* __restrict__ canon, int N, int K,
-                                   int g /*0 = per channel*/, int sym, int Np, int KB,
-                                   const __half* __restrict__ scales_t, const __nv_bfloat16* __restrict__ zeros_t,
-                                   uint8_t* __restrict__ packed, long long npieces) {
+                                   int g /*0 = per channel*/, int sym, int KB, uint8_t* __restrict__ tiles,
+                                   __half* __restrict__ scales_pc, __nv_bfloat16* __restrict__ zeros_pc, long long npieces) {
     long long pid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (pid >= npieces) return;
     PieceCoord pc = piece_coord(pid, KB);
@@ -199,9 +226,9 @@ __global__ void encode_pack_kernel(const float* __restrict__ W, const uint8_t* _
                 c[8 * G + 4 + t] = (v.y >> (8 * t)) & 0xFFu;
             }
         } else {
-            int gi = g ? k0 / g : 0;
-            float s = __half2float(scales_t[(size_t)gi * Np + pc.n]);
-            int z = sym ? half_code : (int)__bfloat162float(zeros_t[(size_t)gi * Np + pc.n]);
+            MetaSlot m = meta_slot(tiles, scales_pc, zeros_pc, BITS, g, !sym, KB, pc.n, g ? k0 / g : 0, 0);
+            float s = __half2float(*m.s);
+            int z = sym ? half_code : (int)__bfloat162float(*m.z);
             const float4* src = reinterpret_cast<const float4*>(W + (size_t)pc.n * K + k0);
             float4 v0 = src[0], v1 = src[1];
             float wv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
@@ -216,18 +243,19 @@ __global__ void encode_pack_kernel(const float* __restrict__ W, const uint8_t* _
     }
     uint32_t w[PieceWords<BITS>::n];
     encode_piece<BITS>(c, w);
-    store_piece<BITS>(packed + pc.blob_index * (size_t)moqe_blob_bytes(BITS), pc.half, pc.slot, w);
+    store_piece<BITS>(tiles + pc.tile_index * (size_t)moqe_tile_stride(BITS, g, !sym) + pc.nb * moqe_blob_bytes(BITS), pc.half,
+                      pc.slot, w);
 }
 
 template <int BITS>
-__global__ void unpack_kernel(const uint8_t* __restrict__ packed, int N, int K, int KB, uint8_t* __restrict__ canon,
-                              long long npieces) {
+__global__ void unpack_kernel(const uint8_t* __restrict__ tiles, int N, int K, int KB, int tile_stride,
+                              uint8_t* __restrict__ canon, long long npieces) {
     long long pid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (pid >= npieces) return;
     PieceCoord pc = piece_coord(pid, KB);
     if (pc.n >= N) return;
     uint32_t w[PieceWords<BITS>::n];
-    load_piece<BITS>(packed + pc.blob_index * (size_t)moqe_blob_bytes(BITS), pc.half, pc.slot, w);
+    load_piece<BITS>(tiles + pc.tile_index * (size_t)tile_stride + pc.nb * moqe_blob_bytes(BITS), pc.half, pc.slot, w);
     uint32_t c[32];
     decode_piece<BITS>(w, c);
 #pragma unroll
@@ -241,27 +269,33 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ packed, int N, int K, 
     }
 }
 
-// canonical [N][G] fp16 scales / zero-points  <->  transposed padded device arrays
-__global__ void meta_export_kernel(const __half* __restrict__ scales_t, const __nv_bfloat16* __restrict__ zeros_t, int N,
-                                   int G, int Np, int bits, uint16_t* __restrict__ scales_out,
-                                   uint16_t* __restrict__ zeros_out) {
+// canonical [N][G] fp16 scales / zero-points  <->  the per-tile (or per-channel) device copies
+__global__ void meta_export_kernel(const uint8_t* __restrict__ tiles, const __half* __restrict__ scales_pc,
+                                   const __nv_bfloat16* __restrict__ zeros_pc, int N, int G, int KB, int bits, int group, int sym,
+                                   uint16_t* __restrict__ scales_out, uint16_t* __restrict__ zeros_out) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)N * G) return;
     int n = (int)(i / G), gi = (int)(i % G);
-    if (scales_out) scales_out[i] = __half_as_ushort(scales_t[(size_t)gi * Np + n]);
+    MetaSlot m = meta_slot(const_cast<uint8_t*>(tiles), const_cast<__half*>(scales_pc), const_cast<__nv_bfloat16*>(zeros_pc), bits,
+                           group, !sym, KB, n, gi, 0);
+    if (scales_out) scales_out[i] = __half_as_ushort(*m.s);
     if (zeros_out) {
-        float z = zeros_t ? __bfloat162float(zeros_t[(size_t)gi * Np + n]) : (float)(1 << (bits - 1));
+        float z = sym ? (float)(1 << (bits - 1)) : __bfloat162float(*m.z);
         zeros_out[i] = __half_as_ushort(__float2half_rn(z));
     }
 }
 
-__global__ void meta_import_kernel(const uint16_t* __restrict__ scales_in, const uint16_t* __restrict__ zeros_in, int N,
-                                   int G, int Np, __half* __restrict__ scales_t, __nv_bfloat16* __restrict__ zeros_t) {
+__global__ void meta_import_kernel(const uint16_t* __restrict__ scales_in, const uint16_t* __restrict__ zeros_in, int N, int G,
+                                   int KB, int bits, int group, int sym, uint8_t* __restrict__ tiles,
+                                   __half* __restrict__ scales_pc, __nv_bfloat16* __restrict__ zeros_pc) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (long long)N * G) return;
     int n = (int)(i / G), gi = (int)(i % G);
-    scales_t[(size_t)gi * Np + n] = __ushort_as_half(scales_in[i]);
-    if (zeros_t) zeros_t[(size_t)gi * Np + n] = __float2bfloat16_rn(__half2float(__ushort_as_half(zeros_in[i])));
+    for (int c = 0; c < meta_copies(group); ++c) {
+        MetaSlot m = meta_slot(tiles, scales_pc, zeros_pc, bits, group, !sym, KB, n, gi, c);
+        *m.s = __ushort_as_half(scales_in[i]);
+        if (!sym) *m.z = __float2bfloat16_rn(__half2float(__ushort_as_half(zeros_in[i])));
+    }
 }
 
 moqe_status check_format(int N, int K, int bits, int group) {
@@ -283,22 +317,25 @@ moqe_status alloc_expert(int N, int K, int bits, int group, int sym, cudaStream_
     e->Np = (N + 127) / 128 * 128;
     e->Kp = (K + 127) / 128 * 128;
     e->G = group ? K / group : 1;
-    e->Gp = group ? e->Kp / group : 1;
-    e->codes = nullptr; e->scales_t = nullptr; e->zeros_t = nullptr;
+    e->tiles = nullptr; e->scales_pc = nullptr; e->zeros_pc = nullptr;
     if (cudaGetDevice(&e->device) != cudaSuccess) { delete e; return MOQE_ERR_CUDA; }
-    e->codes_alloc = (size_t)e->Np * e->Kp * bits / 8;
-    e->meta_alloc = (size_t)e->Gp * e->Np * 2;
-    bool ok = cudaMalloc(&e->codes, e->codes_alloc) == cudaSuccess &&
-              cudaMalloc(&e->scales_t, e->meta_alloc) == cudaSuccess &&
-              (e->sym || cudaMalloc(&e->zeros_t, e->meta_alloc) == cudaSuccess);
+    e->tiles_alloc = (size_t)(e->Np / 128) * (e->Kp / 128) * moqe_tile_stride(bits, group, !e->sym);
+    e->pc_alloc = group == 0 ? (size_t)e->Np * 2 : 0;
+    bool ok = cudaMalloc(&e->tiles, e->tiles_alloc) == cudaSuccess;
+    if (ok && group == 0) {
+        ok = cudaMalloc(&e->scales_pc, e->pc_alloc) == cudaSuccess &&
+             (e->sym || cudaMalloc(&e->zeros_pc, e->pc_alloc) == cudaSuccess);
+    }
     if (!ok) {
         cudaGetLastError();
-        cudaFree(e->codes); cudaFree(e->scales_t); cudaFree(e->zeros_t);
+        cudaFree(e->tiles); cudaFree(e->scales_pc); cudaFree(e->zeros_pc);
         delete e;
         return MOQE_ERR_ALLOC;
     }
-    cudaMemsetAsync(e->scales_t, 0, e->meta_alloc, st);
-    if (e->zeros_t) cudaMemsetAsync(e->zeros_t, 0, e->meta_alloc, st);
+    // padded channels / padded k: codes 0, scale 0, zero-point 0
+    cudaMemsetAsync(e->tiles, 0, e->tiles_alloc, st);
+    if (e->scales_pc) cudaMemsetAsync(e->scales_pc, 0, e->pc_alloc, st);
+    if (e->zeros_pc) cudaMemsetAsync(e->zeros_pc, 0, e->pc_alloc, st);
     *out = e;
     return MOQE_OK;
 }
@@ -309,8 +346,8 @@ moqe_status launch_encode(const moqe_expert* e, const float* W, const uint8_t* c
     long long npieces = (long long)(e->Np / 128) * KB * 512;
     unsigned blocks = (unsigned)((npieces + 127) / 128);
 #define MOQE_ENC(B)                                                                                                  \
-    encode_pack_kernel<B, FROM_CODES><<<blocks, 128, 0, st>>>(W, canon, e->N, e->K, e->group, e->sym, e->Np, KB,      \
-                                                              e->scales_t, e->zeros_t, e->codes, npieces)
+    encode_pack_kernel<B, FROM_CODES><<<blocks, 128, 0, st>>>(W, canon, e->N, e->K, e->group, e->sym, KB, e->tiles,   \
+                                                              e->scales_pc, e->zeros_pc, npieces)
     if (e->bits == 4) MOQE_ENC(4);
     else if (e->bits == 8) MOQE_ENC(8);
     else MOQE_ENC(3);
@@ -334,10 +371,10 @@ extern "C" moqe_status moqe_quantize_rtn(const float* W, int N, int K, int bits,
     moqe_expert* e = nullptr;
     s = alloc_expert(N, K, bits, group, sym, st, &e);
     if (s != MOQE_OK) return s;
-    int g = group ? group : K;
     long long warps = (long long)N * e->G;
     unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-    rtn_scales_kernel<<<blocks, 256, 0, st>>>(W, N, K, bits, g, e->G, e->sym, e->Np, e->scales_t, e->zeros_t);
+    rtn_scales_kernel<<<blocks, 256, 0, st>>>(W, N, K, bits, group, e->G, e->sym, e->Kp / 128, e->tiles, e->scales_pc,
+                                              e->zeros_pc);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) { moqe_expert_destroy(e); return MOQE_ERR_CUDA; }
     s = launch_encode<false>(e, W, nullptr, st);
@@ -359,8 +396,8 @@ extern "C" moqe_status moqe_expert_import(int N, int K, int bits, int group, int
     s = alloc_expert(N, K, bits, group, sym, st, &e);
     if (s != MOQE_OK) return s;
     long long n = (long long)N * e->G;
-    meta_import_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(scales_f16, zeros_f16, N, e->G, e->Np, e->scales_t,
-                                                                    e->zeros_t);
+    meta_import_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(scales_f16, zeros_f16, N, e->G, e->Kp / 128, bits, group,
+                                                                    e->sym, e->tiles, e->scales_pc, e->zeros_pc);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) { moqe_expert_destroy(e); return MOQE_ERR_CUDA; }
     s = launch_encode<true>(e, nullptr, codes, st);
@@ -378,15 +415,17 @@ extern "C" moqe_status moqe_expert_export(const moqe_expert* e, uint8_t* codes, 
         int KB = e->Kp / 128;
         long long npieces = (long long)(e->Np / 128) * KB * 512;
         unsigned blocks = (unsigned)((npieces + 127) / 128);
-        if (e->bits == 4) unpack_kernel<4><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
-        else if (e->bits == 8) unpack_kernel<8><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
-        else unpack_kernel<3><<<blocks, 128, 0, st>>>(e->codes, e->N, e->K, KB, codes, npieces);
+        const int stride = moqe_tile_stride(e->bits, e->group, !e->sym);
+        if (e->bits == 4) unpack_kernel<4><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
+        else if (e->bits == 8) unpack_kernel<8><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
+        else unpack_kernel<3><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
         count_launch();
     }
     if (scales_f16 || zeros_f16) {
         long long n = (long long)e->N * e->G;
-        meta_export_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e->scales_t, e->zeros_t, e->N, e->G, e->Np,
-                                                                        e->bits, scales_f16, zeros_f16);
+        meta_export_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(e->tiles, e->scales_pc, e->zeros_pc, e->N, e->G,
+                                                                        e->Kp / 128, e->bits, e->group, e->sym, scales_f16,
+                                                                        zeros_f16);
         count_launch();
     }
     return cuda_ok(cudaGetLastError());
@@ -402,13 +441,13 @@ extern "C" moqe_status moqe_expert_info(const moqe_expert* e, int* N, int* K, in
     if (sym) *sym = e->sym;
     if (code_bytes) *code_bytes = (size_t)e->N * e->K * e->bits / 8;
     if (meta_bytes) *meta_bytes = (size_t)e->N * e->G * 2 * (e->sym ? 1 : 2);
-    if (alloc_bytes) *alloc_bytes = e->codes_alloc + e->meta_alloc * (e->sym ? 1 : 2);
+    if (alloc_bytes) *alloc_bytes = e->tiles_alloc + e->pc_alloc * (e->sym ? 1 : 2);
     return MOQE_OK;
 }
 
 extern "C" moqe_status moqe_expert_destroy(moqe_expert* e) {
     if (!e) return MOQE_ERR_NULL;
-    cudaError_t a = cudaFree(e->codes), b = cudaFree(e->scales_t), c = cudaFree(e->zeros_t);
+    cudaError_t a = cudaFree(e->tiles), b = cudaFree(e->scales_pc), c = cudaFree(e->zeros_pc);
     delete e;
     return (a == cudaSuccess && b == cudaSuccess && c == cudaSuccess) ? MOQE_OK : MOQE_ERR_CUDA;
 }
