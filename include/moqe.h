@@ -221,7 +221,7 @@ MOQE_API const char* moqe_status_str(moqe_status s);
 /* Measurement knobs (process-wide, not thread-safe; defaults are the tuned values):
  *   "stream_tile_cost_w8" / "_w4" / "_w3" : relative cost of one packed 128x128 tile of
  *                            that bit-width in the streaming kernel's work split
- *                            (defaults 9 / 5 / 4: bytes in 2 KiB units plus a fixed part).
+ *                            (defaults 8 / 8 / 8).
  * Unknown key: MOQE_ERR_UNSUPPORTED. */
 MOQE_API moqe_status moqe_tune(const char* key, int value);
 

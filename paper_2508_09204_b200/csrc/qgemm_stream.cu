@@ -488,8 +488,12 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) qgemm_stream_kernel(const _
                 const unsigned old = atomicAdd(cnt, 1u);
                 const int last = (old == (unsigned)(c_last - c_first));
                 if (last) *cnt = 0u;                               // leave the counters clear for the next call
+                int slots = 0;                                     // bit i: contributor c_first + i parked its piece in slot 1
+                if (last)
+                    for (int cc = c_first; cc <= c_last && cc - c_first < 24; ++cc)
+                        if (sched_tbegin(sch, cc, e, base) <= nt * p.KB) slots |= 1 << (cc - c_first);
                 rec[6] = c_first;
-                rec[7] = c_last;
+                rec[7] = (c_last - c_first) | (slots << 8);
                 rec[0] = last;
             }
             mbar_arrive(bar_fixdone);
@@ -574,19 +578,17 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) qgemm_stream_kernel(const _
             for (int pi = 0; pi < n_pending && pi < MAX_PENDING; ++pi) {
                 volatile int* rec = s_pend + 8 * pi;
                 if (rec[0] != 1) continue;                   // the fix-up warp's atomic and the barrier order the reads below
-                const int e = rec[1], nt = rec[2], pend_j0 = rec[3], pend_tv = rec[4], pend_chunk = rec[5];
-                const int c_first = rec[6], c_last = rec[7];
-                const int seg_t0 = nt * p.KB;
-                const long long base = sched_base(sch, e);
+                const int nt = rec[2], pend_j0 = rec[3], pend_tv = rec[4], pend_chunk = rec[5];
+                const int c_first = rec[6], n_contrib = (rec[7] & 0xFF) + 1, slots = rec[7] >> 8;
                 for (int i = tid; i < pend_tv * 64; i += CONSUMER_WARPS * 32) {
                     const int tok = i >> 6, v = i & 63;
                     const int n = nt * 128 + v * 2;
                     if (n >= p.N) continue;
                     float a = 0.f, b = 0.f;
-                    for (int cc = c_first; cc <= c_last; ++cc) {
-                        // contributor cc's piece starts where its range or the segment starts, whichever is later
-                        const int slot = sched_tbegin(sch, cc, e, base) > seg_t0 ? 0 : 1;
-                        const float* src = p.partials + (((size_t)cc * 2 + slot) * MAX_CHUNKS_SPLIT + pend_chunk) * (T * 128);
+                    for (int ci = 0; ci < n_contrib; ++ci) {
+                        // a contributor whose piece starts at the segment's start parked it in slot 1, else in slot 0
+                        const int slot = (slots >> ci) & 1;
+                        const float* src = p.partials + (((size_t)(c_first + ci) * 2 + slot) * MAX_CHUNKS_SPLIT + pend_chunk) * (T * 128);
                         const float2 pv = __ldcg(reinterpret_cast<const float2*>(src + tok * 128 + v * 2));
                         a += pv.x;
                         b += pv.y;
@@ -620,8 +622,9 @@ int sm_count() {
     return g_sm_count;
 }
 
-// relative cost of streaming one packed tile: its bytes (in units of 2 KiB) plus a fixed part
-int g_tile_cost[9] = {0, 0, 0, 4, 5, 0, 0, 0, 9};
+// relative cost of one packed tile in the work split.  Measured: a tile costs about the same time whatever its
+// width (the per-tile latency of a consumer warp, not its bytes, sets the pace), hence equal costs.
+int g_tile_cost[9] = {0, 0, 0, 8, 8, 0, 0, 0, 8};
 
 }  // namespace
 
@@ -665,7 +668,14 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
     int wmax = 1;
     for (int e = 0; e < E; ++e) wmax = s.w[e] > wmax ? s.w[e] : wmax;
     const long long work_items = s.split ? s.C / wmax : (long long)E * p.ntiles;
-    const int grid = (int)(work_items < ctas ? (work_items < 1 ? 1 : work_items) : ctas);
+    long long grid_ll = work_items < ctas ? (work_items < 1 ? 1 : work_items) : ctas;
+    if (s.split) {
+        // the reduction records which slot each contributor used in a 24-bit mask: keep a segment's contributors
+        // below that (one segment costs KB * w, one CTA carries C / G)
+        const long long cap = 22 * s.C / ((long long)p.KB * wmax);
+        if (grid_ll > cap) grid_ll = cap < 1 ? 1 : cap;
+    }
+    const int grid = (int)grid_ll;
     s.G = grid;
     p.X = (const uint16_t*)X;
     p.Y = (uint16_t*)Y;
