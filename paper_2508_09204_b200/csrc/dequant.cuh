@@ -46,19 +46,26 @@ __device__ __forceinline__ void unpack_chunk(const uint32_t (&w)[PieceWords<BITS
             out[i] = hsub2_bf16(v | 0x43004300u, zz);
         }
     } else {
-        // 0x4B000000 | c is the fp32 number 2^23 + c; subtracting 2^23 + z is exact and |c - z| <= 255
-        // has at most 8 significant bits, so the conversion to bf16 is exact too.
-        const float f = 8388608.f + z;
+        // A byte c zero-extended to 16 bits IS the bf16 number c * 2^-133 (subnormal below 128, and the encoding
+        // runs on continuously into the first normal binade).  One fused multiply-add per PAIR of codes,
+        // c * 2^-133 * 2^120 - z * 2^-13, gives (c - z) * 2^-13 exactly (|c - z| <= 255 has 8 significant bits);
+        // the callers fold the factor 2^13 (W8_PRESCALE) into the fp32 scale.
+        const float zs = z * 0.0001220703125f;                       // z * 2^-13, exact
+        const uint32_t negz = pack_bf16x2(-zs, -zs);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint32_t s = w[2 * G + (i >> 1)];
-            const uint32_t sel = 0x7540u + 2 * (i & 1);
-            float a = __uint_as_float(__byte_perm(s, 0x4B000000u, sel)) - f;
-            float b = __uint_as_float(__byte_perm(s, 0x4B000000u, sel + 1)) - f;
-            out[i] = pack_bf16x2(a, b);
+            const uint32_t pair = __byte_perm(w[2 * G + (i >> 1)], 0u, (i & 1) ? 0x4342u : 0x4140u);   // {c_hi, c_lo} as 16-bit
+            __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&pair);
+            const uint32_t k120 = 0x7B807B80u;                      // 2^120 in both halves
+            __nv_bfloat162 r = __hfma2(v, *reinterpret_cast<const __nv_bfloat162*>(&k120),
+                                       *reinterpret_cast<const __nv_bfloat162*>(&negz));
+            out[i] = *reinterpret_cast<uint32_t*>(&r);
         }
     }
 }
+
+// what an 8-bit chunk unpacked by unpack_chunk must still be multiplied by
+constexpr float W8_PRESCALE = 8192.f;
 
 // Chunk G of a 4- or 3-bit piece as the bf16 numbers 128 + c (no zero-point): two instructions per pair.
 // The caller removes (128 + z) * sum_k X with the help of a second MMA against an all-ones operand.

@@ -251,8 +251,8 @@ __device__ __forceinline__ void consume_stage(const unsigned char* stage, int x_
         constexpr bool group_begins = ngrp == 4 || (ngrp == 2 && (G & 1) == 0) || G == 0;
         if constexpr (!per_channel && group_begins) {
             const __half* sc = moqe_tile_scales(stage, BITS, hz, gj) + row;
-            slg = __half2float(sc[0]);
-            shg = __half2float(sc[8]);
+            slg = __half2float(sc[0]) * (BITS == 8 ? W8_PRESCALE : 1.f);
+            shg = __half2float(sc[8]) * (BITS == 8 ? W8_PRESCALE : 1.f);
             // symmetric experts have no zero-point rows: the (in-bounds) loads below are then ignored
             const __nv_bfloat16* zp = moqe_tile_zeros(stage, BITS, gj) + row;
             const float zl_t = __bfloat162float(zp[0]), zh_t = __bfloat162float(zp[8]);
@@ -323,8 +323,8 @@ __device__ __noinline__ int mainloop_to_out(const StreamParams* pp, int e, int n
     float s_lo = 0.f, s_hi = 0.f;                                         // per-channel scales and zero-points
     float pc_zl = (float)(1 << (BITS - 1)), pc_zh = pc_zl;
     if constexpr (GM == 0) {
-        s_lo = __half2float(ex.scales_pc[n_lo]);
-        s_hi = __half2float(ex.scales_pc[n_lo + 8]);
+        s_lo = __half2float(ex.scales_pc[n_lo]) * (BITS == 8 ? W8_PRESCALE : 1.f);
+        s_hi = __half2float(ex.scales_pc[n_lo + 8]) * (BITS == 8 ? W8_PRESCALE : 1.f);
         if (has_zeros) { pc_zl = __bfloat162float(ex.zeros_pc[n_lo]); pc_zh = __bfloat162float(ex.zeros_pc[n_lo + 8]); }
     }
     float acc[NT][4], part[NSETS][NT][4], xs[NT][4];

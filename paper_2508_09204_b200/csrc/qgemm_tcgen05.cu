@@ -383,6 +383,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                     const unsigned char* tile = ex.tiles + ((size_t)ti.nt * p.KB + gi / per_tile) * (size_t)ex.tile_stride;
                     s = __half2float(moqe_tile_scales(tile, ex.bits, ex.has_zeros, gi % per_tile)[row]);
                 }
+                if (ex.bits == 8) s *= W8_PRESCALE;          // 8-bit chunks are unpacked as (c - z) * 2^-13
                 if (!(ok = mbar_wait(bar_accfull + 8 * buf, acc_use[buf] & 1u, s_abort, p.status))) break;
                 tc_fence_after();
 #pragma unroll
