@@ -102,6 +102,11 @@ size_t sort_workspace_bytes(int M, int E);
 moqe_status launch_gather(const void* X, const int32_t* perm, const int32_t* offsets_E, int M, int C, void* Xp,
                           cudaStream_t st);
 
+// 64-row boxes of the expert-sorted activations: copied to Xp only where the rows are not already consecutive in X
+size_t gather_boxes_bytes(int M, int E);
+moqe_status launch_gather_boxes(const void* X, const int32_t* perm, const int32_t* offsets, int M, int C, int E, void* Xp,
+                                int32_t* box_src, cudaStream_t st);
+
 // qgemm_stream.cu
 size_t stream_workspace_bytes(int M, int Np, int E);
 moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,

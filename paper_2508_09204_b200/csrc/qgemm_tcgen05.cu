@@ -48,6 +48,7 @@ struct TcParams {
     ExpertDev ex[MOQE_MAX_EXPERTS];
     const int32_t* perm;
     const int32_t* offsets;
+    const int32_t* box_src;   // per 64-row box: first source row in X if its rows are consecutive there, else -1 (use Xp)
     uint16_t* Y;
     int* status;
     int M, N, K, Np, KB, E, n_tiles;
@@ -227,7 +228,8 @@ __device__ __forceinline__ bool dequant_kblock(const ExpertDev& ex, int nt, unsi
 // ---------------------------------------------------------------------------- the kernel
 template <int TN, bool REGSPLIT>
 __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_constant__ TcParams p,
-                                                                const __grid_constant__ CUtensorMap tmap) {
+                                                                const __grid_constant__ CUtensorMap tmap,
+                                                                const __grid_constant__ CUtensorMap tmap_x) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     using L = Smem<TN>;
@@ -265,12 +267,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
             bool ok = true;
             for (int t = blockIdx.x; ok && decode_tile<TN>(s_off, p.E, p.n_tiles, t, ti); t += gridDim.x) {
                 const int nbox = (ti.rows + XBOX_ROWS - 1) / XBOX_ROWS;
+                // where each 64-row box of this tile comes from: straight from X when its rows are consecutive there
+                int box0 = (ti.m0 - s_off[ti.e]) / XBOX_ROWS;
+                for (int e2 = 0; e2 < ti.e; ++e2) box0 += (s_off[e2 + 1] - s_off[e2] + XBOX_ROWS - 1) / XBOX_ROWS;
+                int src_row[TN / XBOX_ROWS];
+#pragma unroll
+                for (int b = 0; b < TN / XBOX_ROWS; ++b) src_row[b] = b < nbox ? p.box_src[box0 + b] : -1;
                 for (int ks = 0; ks < 2 * p.KB; ++ks) {
                     if (!(ok = mbar_wait(bar_empty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status))) break;
                     const uint32_t full = bar_xfull + 8 * ring.stage;
                     mbar_expect_tx(full, nbox * XBOX_BYTES);
                     const uint32_t dst = sbase + L::x_off + ring.stage * (TN * 128);
-                    for (int b = 0; b < nbox; ++b) tma_load_2d(dst + b * XBOX_BYTES, &tmap, ks * 64, ti.m0 + b * XBOX_ROWS, full);
+#pragma unroll
+                    for (int b = 0; b < TN / XBOX_ROWS; ++b) {
+                        if (b < nbox) {
+                            if (src_row[b] >= 0) tma_load_2d(dst + b * XBOX_BYTES, &tmap_x, ks * 64, src_row[b], full);
+                            else tma_load_2d(dst + b * XBOX_BYTES, &tmap, ks * 64, ti.m0 + b * XBOX_ROWS, full);
+                        }
+                    }
                     ring.advance(NS);
                 }
             }
@@ -452,8 +466,8 @@ int g_tile_tokens_override = 0;
 void tc_set_tile_tokens(int tn) { g_tile_tokens_override = tn; }
 
 size_t tc_workspace_bytes(int M, int K, int E, int Np) {
-    (void)E; (void)Np;
-    return ((size_t)M * K * 2 + 255) / 256 * 256;
+    (void)Np;
+    return ((size_t)M * K * 2 + 255) / 256 * 256 + gather_boxes_bytes(M, E);
 }
 
 moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
@@ -464,7 +478,8 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
     if (!enc) return MOQE_ERR_CUDA;
     // 1. expert-sorted copy of the activations (rows with an invalid id become zero rows at the end)
     void* Xp = ws;
-    moqe_status s = launch_gather(X, perm, offsets + E, M, K, Xp, st);
+    int32_t* box_src = (int32_t*)((char*)ws + ((size_t)M * K * 2 + 255) / 256 * 256);
+    moqe_status s = launch_gather_boxes(X, perm, offsets, M, K, E, Xp, box_src, st);
     if (s != MOQE_OK) return s;
     // 2. tensor map over Xp[M][K] bf16: boxes of 64 k x 64 rows, 128-byte swizzle, zero fill outside
     CUtensorMap tmap;
@@ -475,10 +490,15 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Xp, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return MOQE_ERR_CUDA;
+    CUtensorMap tmap_x;                                   // the same boxes over the caller's X (unsorted rows)
+    if (enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return MOQE_ERR_CUDA;
     TcParams p;
     for (int e = 0; e < E; ++e) {
         p.ex[e] = ex[e]->dev();
     }
+    p.box_src = box_src;
     p.perm = perm; p.offsets = offsets; p.Y = (uint16_t*)Y; p.status = device_status_word();
     p.M = M; p.N = N; p.K = K; p.Np = ex[0]->Np; p.KB = ex[0]->Kp / 128; p.E = E; p.n_tiles = p.Np / 128;
     int dev = 0, sms = 148;
@@ -495,7 +515,7 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
                 return MOQE_ERR_CUDA;
             attr = true;
         }
-        qgemm_tc_kernel<256, true><<<grid, TC_THREADS, Smem<256>::dyn_bytes, st>>>(p, tmap);
+        qgemm_tc_kernel<256, true><<<grid, TC_THREADS, Smem<256>::dyn_bytes, st>>>(p, tmap, tmap_x);
     } else {
         static bool attr = false;
         if (!attr) {
@@ -503,7 +523,7 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
                 return MOQE_ERR_CUDA;
             attr = true;
         }
-        qgemm_tc_kernel<128, false><<<grid, TC_THREADS, Smem<128>::dyn_bytes, st>>>(p, tmap);
+        qgemm_tc_kernel<128, false><<<grid, TC_THREADS, Smem<128>::dyn_bytes, st>>>(p, tmap, tmap_x);
     }
     err = cudaGetLastError();
     count_launch();

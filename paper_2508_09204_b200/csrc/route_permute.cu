@@ -180,6 +180,34 @@ __global__ void move_rows_kernel(const uint4* __restrict__ src, const int32_t* _
     }
 }
 
+// Gather for the tcgen05 kernel, 64-row box by box.  Boxes are counted per expert from the start of the
+// expert's segment (box id = sum over earlier experts of ceil(rows/64) + local box).  A box whose rows are
+// consecutive rows of X anyway (the usual case: a sample's rows are contiguous and share an expert) is NOT
+// copied: box_src[id] = its first source row, and the GEMM's TMA reads X directly; otherwise the rows are
+// copied to Xp[offsets[e] + 64*box ..] and box_src[id] = -1.
+__global__ void __launch_bounds__(256) gather_boxes_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ perm,
+                                                           const int32_t* __restrict__ offsets, int E, int vec_per_row,
+                                                           uint4* __restrict__ Xp, int32_t* __restrict__ box_src) {
+    int b = blockIdx.x, e = 0, rows_e = 0;
+    for (; e < E; ++e) {
+        rows_e = offsets[e + 1] - offsets[e];
+        const int nb = (rows_e + 63) >> 6;
+        if (b < nb) break;
+        b -= nb;
+    }
+    if (e == E) return;
+    const int j0 = offsets[e] + b * 64, cnt = min(64, rows_e - b * 64);
+    const int first = perm[j0];
+    const int ok = (threadIdx.x >= cnt) || (perm[j0 + threadIdx.x] == first + (int)threadIdx.x);
+    const int all_ok = __syncthreads_and(ok);
+    if (threadIdx.x == 0) box_src[blockIdx.x] = all_ok ? first : -1;
+    if (all_ok) return;
+    for (int i = threadIdx.x; i < cnt * vec_per_row; i += blockDim.x) {
+        const int r = i / vec_per_row, v = i - r * vec_per_row;
+        Xp[(size_t)(j0 + r) * vec_per_row + v] = X[(size_t)perm[j0 + r] * vec_per_row + v];
+    }
+}
+
 }  // namespace
 
 size_t sort_workspace_bytes(int M, int E) {
@@ -221,6 +249,16 @@ moqe_status launch_gather(const void* X, const int32_t* perm, const int32_t* n_v
     long long total = (long long)M * vec;
     move_rows_kernel<true><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint4*)X, perm, n_valid_ptr, M, vec,
                                                                            (uint4*)Xp);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+size_t gather_boxes_bytes(int M, int E) { return ((size_t)(M / 64 + E + 1) * sizeof(int32_t) + 255) / 256 * 256; }
+
+moqe_status launch_gather_boxes(const void* X, const int32_t* perm, const int32_t* offsets, int M, int C, int E, void* Xp,
+                                int32_t* box_src, cudaStream_t st) {
+    if (M == 0) return MOQE_OK;
+    gather_boxes_kernel<<<M / 64 + E, 256, 0, st>>>((const uint4*)X, perm, offsets, E, C / 8, (uint4*)Xp, box_src);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
