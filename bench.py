@@ -35,6 +35,15 @@ import moqe_workloads as wl  # noqa: E402
 METRIC = "routed_qgemm_tokens_per_s"
 UNIT = "tokens/s"
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from one ncu capture of the
+# q_proj launch of the workload (profiles/), as a ratio to that launch's algorithmic bytes; traffic grows in
+# proportion with the bytes streamed, so the ratio is applied to the average launch of the block.
+# None = no capture of the current kernel.
+TRAFFIC_RATIO = {
+    "llama7b_decode": 32.755 / 32.513,      # 32.73 MB read + 0.02 MB written vs 32.51 MB algorithmic
+    "llama7b_prefill": 267.12 / 300.95,     # 158.4 MB read + 108.7 MB written (part of Y still in L2) vs 300.9 MB
+}
+
 
 # --------------------------------------------------------------------------- helpers
 def load_peaks():
@@ -390,21 +399,28 @@ def main():
         alg_bytes.append(b)
         flops.append(2.0 * L["M"] * L["spec"].N * L["spec"].K)
     tot_ms = sum(layer_ms)
+    n_launch = len(layers)
+    ratio = TRAFFIC_RATIO.get(w.name) if args.path == 0 and not args.tune else None
+    traffic = None if ratio is None else ratio * sum(alg_bytes) / n_launch
     hbm_time = sum(alg_bytes) / (peaks["hbm_gbs"] * 1e9)
     tensor_time = sum(flops) / (peaks["bf16_tflops"] * 1e12)
     if tensor_time > hbm_time:
         achieved = sum(flops) / (tot_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": None,
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
                     "frac_whole_step": sum(flops) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
                     "frac_of_nominal_2250": achieved / 2250.0}
     else:
         achieved = sum(alg_bytes) / (tot_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic,
                     "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     "frac_of_nominal_8000": achieved / 8000.0}
-    roofline.update({"peak_source": peaks["source"], "kernel": "routed dequant-GEMM launches of one block",
+    roofline.update({"peak_source": peaks["source"],
+                     "kernel": ("qgemm_tc_kernel" if tensor_time > hbm_time else "qgemm_stream_kernel") +
+                               f": average of the {n_launch} routed-GEMM launches of one block",
+                     "launches_per_step": n_launch, "algorithmic_bytes_per_launch": sum(alg_bytes) / n_launch,
+                     "traffic_unit": "bytes per launch",
                      "algorithmic_bytes_per_step": int(sum(alg_bytes)), "flops_per_step": float(sum(flops)),
                      "launch_ms": {L["spec"].name: round(t, 5) for L, t in zip(layers, layer_ms)}})
 
