@@ -249,6 +249,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2508_09204_b200 as moqe
+    from paper_2508_09204_b200 import replicas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the routed path has no CPU fallback")
@@ -265,7 +266,7 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
-    seed = args.seed + 1000 * rank                          # every rank owns its own shard of samples (weak scaling)
+    seed = replicas.shard_seed(args.seed, rank)             # every rank owns its own shard of samples (weak scaling)
     E = w.n_experts
 
     # ---- experts (replicated on every rank) and resident inputs ---------------------------------
@@ -337,8 +338,7 @@ def main():
         for _ in range(warmup):
             run()
         stream.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -346,14 +346,8 @@ def main():
             run()
         e1.record(stream)
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        replicas.barrier()
+        return replicas.max_over_ranks(e0.elapsed_time(e1), dev)
 
     tokens_per_step = sum(w.sample_rows) if w.layers[0].rows_per_sample is None else w.n_samples
     sampler = ClockSampler(physical_gpu_index(local))
@@ -365,7 +359,7 @@ def main():
     ms = timed(run, args.steps, args.warmup)
     launches = (graph_launches * args.steps) if graph_launches else (moqe.moqe_launch_count() - l0)
     ms_per_step = ms / args.steps
-    value = world * tokens_per_step / (ms_per_step * 1e-3)
+    value = replicas.whole_job_value(tokens_per_step, world, ms_per_step)
 
     # ---- 2. per-launch duration of the dominant kernel (events round every routed-GEMM call) ----
     sorted_for = hot_path(False)
@@ -430,7 +424,7 @@ def main():
     ms_h = timed(run_h, e2e_steps, 3) / e2e_steps
     h2d = int(logits_h.numel() * 4 + sum(L["Xh"].numel() * 2 for L in layers))
     d2h = int(sum(L["Yh"].numel() * 2 for L in layers))
-    e2e = {"value": world * tokens_per_step / (ms_h * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": replicas.whole_job_value(tokens_per_step, world, ms_h), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": ms_h}
 
     line = {
