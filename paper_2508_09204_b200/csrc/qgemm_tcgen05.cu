@@ -75,6 +75,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// One lane of a converged warp (tcgen05.mma and tcgen05.commit are issued by one thread, from warp-uniform code).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -305,8 +311,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                     ring.advance(NWS);
                 }
             }
-        } else if (warp == 1 && lane == 0) {
+        } else if (warp == 1) {
             // ---------------- MMA issuer ----------------
+            // The WHOLE warp walks the tiles, so that control flow stays warp-uniform, and one elected lane issues
+            // straight-line MMAs whose operands were all computed beforehand.  Measured on B200: issued this way a
+            // 128x256x16 MMA costs its 128 tensor-pipe cycles (and a 16-column one 24); issued from a loop that
+            // only lane 0 runs (`if (lane == 0)`) and that builds descriptors between MMAs, every MMA costs ~250.
             Ring ring;
             TileInfo ti;
             bool ok = true;
@@ -319,27 +329,57 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                 const int group_k = ex.group == 0 ? p.KB * 128 : min(ex.group, 128);
                 int kcount = 0;
                 for (int ks = 0; ok && ks < 2 * p.KB; ++ks) {
-                    if (!(ok = mbar_wait(bar_xfull + 8 * ring.stage, ring.phase, s_abort, p.status))) break;
-                    if (!(ok = mbar_wait(bar_afull + 8 * ring.stage, ring.phase, s_abort, p.status))) break;
-                    tc_fence_after();
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
                     const uint64_t adesc = umma_desc_sw128(sbase + L::a_off + ring.stage * A_STAGE_BYTES);
                     const uint64_t bdesc = umma_desc_sw128(sbase + L::x_off + ring.stage * (TN * 128));
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (kcount == 0) {
-                            if (!(ok = mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status))) break;
-                            tc_fence_after();
+                    const uint32_t empty_bar = bar_empty + 8 * ring.stage;
+                    if (group_k >= 64) {
+                        // the stage's four MMAs feed one accumulator buffer
+                        if (kcount == 0 &&
+                            !(ok = __all_sync(0xffffffffu, mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
+                        tc_fence_after();
+                        const uint32_t d = tmem_base + buf * TN;
+                        const bool group_ends = kcount + 64 == group_k;
+                        if (elect_one()) {
+                            umma_bf16(d, adesc, bdesc, idesc, kcount > 0 ? 1u : 0u);
+                            umma_bf16(d, adesc + 2, bdesc + 2, idesc, 1u);
+                            umma_bf16(d, adesc + 4, bdesc + 4, idesc, 1u);
+                            umma_bf16(d, adesc + 6, bdesc + 6, idesc, 1u);
+                            if (group_ends) umma_commit(bar_accfull + 8 * buf);
+                            umma_commit(empty_bar);
                         }
-                        umma_bf16(tmem_base + buf * TN, adesc + 2 * j, bdesc + 2 * j, idesc, kcount > 0 ? 1u : 0u);
-                        kcount += 16;
-                        if (kcount == group_k) {
-                            umma_commit(bar_accfull + 8 * buf);
+                        __syncwarp();
+                        kcount += 64;
+                        if (group_ends) {
                             acc_use[buf]++;
                             buf ^= 1;
                             kcount = 0;
                         }
+                    } else {
+                        // groups of 32 k: two accumulator buffers per stage
+                        tc_fence_after();
+                        for (int j = 0; ok && j < 4; ++j) {
+                            if (kcount == 0) {
+                                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
+                                tc_fence_after();
+                            }
+                            const bool group_ends = kcount + 16 == group_k;
+                            if (elect_one()) {
+                                umma_bf16(tmem_base + buf * TN, adesc + 2 * j, bdesc + 2 * j, idesc, kcount > 0 ? 1u : 0u);
+                                if (group_ends) umma_commit(bar_accfull + 8 * buf);
+                                if (j == 3) umma_commit(empty_bar);
+                            }
+                            __syncwarp();
+                            kcount += 16;
+                            if (group_ends) {
+                                acc_use[buf]++;
+                                buf ^= 1;
+                                kcount = 0;
+                            }
+                        }
+                        if (!ok) break;
                     }
-                    umma_commit(bar_empty + 8 * ring.stage);
                     ring.advance(NS);
                 }
             }
