@@ -88,6 +88,29 @@ __device__ __forceinline__ void unpack_chunk_biased(const uint32_t (&w)[PieceWor
     }
 }
 
+// The packed words of one piece -- the 32 codes of channel row (half, r) and k quarter q of a 16-channel blob in
+// shared memory -- at slot = q*8 + (r ^ 2q).
+template <int BITS>
+__device__ __forceinline__ void load_piece_smem(const unsigned char* blob, int half, int slot, uint32_t (&w)[PieceWords<BITS>::n]) {
+    if constexpr (BITS == 4) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if constexpr (BITS == 8) {
+        uint4 v = *reinterpret_cast<const uint4*>(blob + half * 1024 + slot * 16);
+        uint4 u = *reinterpret_cast<const uint4*>(blob + half * 1024 + 512 + slot * 16);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; w[4] = u.x; w[5] = u.y; w[6] = u.z; w[7] = u.w;
+    } else {
+        if (half == 0) {
+            uint4 v = *reinterpret_cast<const uint4*>(blob + slot * 16);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z;
+        } else {
+            w[0] = *reinterpret_cast<const uint32_t*>(blob + slot * 16 + 12);
+            uint2 u = *reinterpret_cast<const uint2*>(blob + 512 + slot * 8);
+            w[1] = u.x; w[2] = u.y;
+        }
+    }
+}
+
 // group index of chunk G of k-block kb:  per channel -> 0;  g = 32 -> 4*kb + G;  g = 64 -> 2*kb + G/2;
 // g >= 128 -> 128*kb / g
 __device__ __forceinline__ int group_of_chunk(int group, int kb, int G) {
