@@ -44,13 +44,31 @@ WsLayout ws_layout(int M, int Np, int K, int E) {
     w.offsets = off; off += align256((MOQE_MAX_EXPERTS + 2) * sizeof(int32_t));
     w.sort = off;    off += align256(sort_workspace_bytes(M, E));
     w.body = off;
-    size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np);
-    off += align256(a > b ? a : b);
+    size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np), c = decode_workspace_bytes(M, Np, E);
+    a = a > b ? a : b;
+    off += align256(a > c ? a : c);
     w.total = off;
     return w;
 }
 
 constexpr int AUTO_STREAM_MAX_ROWS = 128;
+constexpr int LAST_PATH = 5;
+
+bool g_auto_decode = false;   // whether the automatic choice takes the tcgen05 decode kernel where it applies
+
+// 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = tcgen05 decode kernel
+int pick_kernel(int path, int M, const moqe_expert* const* ex, int E) {
+    if (path == 5) return 2;
+    if (path == 1) return 1;
+    if (path == 0) return (g_auto_decode && decode_supported(M, ex, E)) ? 2 : (M <= AUTO_STREAM_MAX_ROWS ? 1 : 0);
+    return 0;
+}
+
+// the arrival counters at the head of the workspace body (both split-K kernels keep theirs there)
+size_t body_zero_bytes(int M, int Np) {
+    const size_t a = stream_zero_bytes(M, Np), b = decode_zero_bytes(M, Np);
+    return a > b ? a : b;
+}
 
 }  // namespace
 }  // namespace moqe
@@ -77,7 +95,7 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     if (M == 0) return MOQE_OK;
     if (!X_bf16 || !row_ids || !Y_bf16) return MOQE_ERR_NULL;
     if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
-    if (path < 0 || path > 4) return MOQE_ERR_SHAPE;
+    if (path < 0 || path > LAST_PATH) return MOQE_ERR_SHAPE;
     const int Np = h_experts[0]->Np;
     WsLayout w = ws_layout(M, Np, K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
@@ -85,12 +103,16 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     char* base = (char*)workspace;
     int32_t* perm = (int32_t*)(base + w.perm);
     int32_t* offsets = (int32_t*)(base + w.offsets);
-    const bool use_stream = path == 1 || (path == 0 && M <= AUTO_STREAM_MAX_ROWS);
-    size_t zero_bytes = use_stream ? stream_zero_bytes(M, Np) : 0;
+    const int kernel = pick_kernel(path, M, h_experts, E);
+    if (kernel == 2 && !decode_supported(M, h_experts, E)) return MOQE_ERR_UNSUPPORTED;
+    size_t zero_bytes = kernel != 0 ? body_zero_bytes(M, Np) : 0;
     moqe_status s = launch_sort(row_ids, M, E, perm, offsets, base + w.sort, w.body - w.sort, base + w.body, zero_bytes,
                                 Y_bf16, N, st);
     if (s != MOQE_OK) return s;
-    if (use_stream)
+    if (kernel == 2)
+        return launch_qgemm_decode(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
+                                   w.total - w.body, st);
+    if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
     tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
@@ -111,14 +133,18 @@ extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_
     if (M == 0) return MOQE_OK;
     if (!X_bf16 || !perm || !offsets || !Y_bf16) return MOQE_ERR_NULL;
     if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
-    if (path < 0 || path > 4) return MOQE_ERR_SHAPE;
+    if (path < 0 || path > LAST_PATH) return MOQE_ERR_SHAPE;
     const int Np = h_experts[0]->Np;
     WsLayout w = ws_layout(M, Np, K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)workspace;
-    const bool use_stream = path == 1 || (path == 0 && M <= AUTO_STREAM_MAX_ROWS);
-    if (use_stream)
+    const int kernel = pick_kernel(path, M, h_experts, E);
+    if (kernel == 2 && !decode_supported(M, h_experts, E)) return MOQE_ERR_UNSUPPORTED;
+    if (kernel == 2)
+        return launch_qgemm_decode(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
+                                   w.total - w.body, st);
+    if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
     tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
@@ -131,7 +157,7 @@ extern "C" moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t
     const int Np = (N + 127) / 128 * 128;
     WsLayout w = ws_layout(M, Np, K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
-    size_t zb = stream_zero_bytes(M, Np);
+    size_t zb = body_zero_bytes(M, Np);
     if (zb == 0) return MOQE_OK;
     return cuda_ok(cudaMemsetAsync((char*)workspace + w.body, 0, zb, (cudaStream_t)stream));
 }
@@ -147,6 +173,10 @@ extern "C" moqe_status moqe_tune(const char* key, int value) {
     if (!strcmp(key, "stream_tile_cost_w8")) { stream_set_tile_cost(8, value); return MOQE_OK; }
     if (!strcmp(key, "stream_tile_cost_w4")) { stream_set_tile_cost(4, value); return MOQE_OK; }
     if (!strcmp(key, "stream_tile_cost_w3")) { stream_set_tile_cost(3, value); return MOQE_OK; }
+    if (!strcmp(key, "auto_decode")) { g_auto_decode = value != 0; return MOQE_OK; }
+    if (!strcmp(key, "decode_tile_cost_w8")) { decode_set_tile_cost(8, value); return MOQE_OK; }
+    if (!strcmp(key, "decode_tile_cost_w4")) { decode_set_tile_cost(4, value); return MOQE_OK; }
+    if (!strcmp(key, "decode_tile_cost_w3")) { decode_set_tile_cost(3, value); return MOQE_OK; }
     return MOQE_ERR_UNSUPPORTED;
 }
 

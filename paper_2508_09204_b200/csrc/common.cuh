@@ -115,6 +115,16 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
 size_t stream_zero_bytes(int M, int Np);
 void stream_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split (measurement knob)
 
+// qgemm_decode.cu: decode shapes -- at most DECODE_MAX_ROWS rows, experts per-channel or with groups of >= 128 k
+constexpr int DECODE_MAX_ROWS = 16;
+bool decode_supported(int M, const moqe_expert* const* ex, int E);
+size_t decode_workspace_bytes(int M, int Np, int E);
+size_t decode_zero_bytes(int M, int Np);
+moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
+                                const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes,
+                                cudaStream_t st);
+void decode_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split; 0 = its bytes
+
 // qgemm_tcgen05.cu
 void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)
 size_t tc_workspace_bytes(int M, int K, int E, int Np);

@@ -1,0 +1,627 @@
+// Routed dequant-GEMM for decode shapes (at most 16 token rows in the batch): every touched
+// expert's packed weights are streamed from HBM exactly once.
+//
+//   producer (1 thread)     : cp.async.bulk copies of whole packed 128x128-code tiles (codes + the
+//                             tile's scales / zero-points, contiguous in HBM) into a shared-memory
+//                             ring guarded by full/empty mbarriers.
+//   dequant (4 warpgroups)  : warpgroup w takes the CTA's tiles t = w (mod 4).  Thread r of a
+//                             warpgroup owns channel row r of the tile: it reads the row's packed
+//                             words with conflict-free 128-bit shared loads, unpacks them in registers
+//                             to the exact integers (c - z) in bf16 and stores them straight into
+//                             TENSOR MEMORY (tcgen05.st, lane r) as operand A of the MMA -- no
+//                             shared-memory round trip.  The same warpgroup fetches the token rows of
+//                             its next tile (gathered through `perm`: the fused permutation) with
+//                             16-byte async copies into a K-major, 128-byte-swizzled operand tile.
+//                             Sixteen warps run this one loop, which is what hides the latency of the
+//                             half-rate integer / bf16x2 instructions the unpacking consists of.
+//   MMA issuer (1 warp)     : tcgen05.mma, A from TMEM (128 channels x 16 k), B = the token tile in
+//                             shared memory (N = 16), fp32 accumulators in TMEM, one buffer per
+//                             quantization group:
+//                               Y[m][n] = sum_G s[n][G] * (sum_{k in G} X[m][k] * (c[n][k] - z[n][G]))
+//                             so the tensor core only multiplies exactly representable numbers.
+//                             The whole warp walks the tiles; one elected lane issues eight
+//                             straight-line MMAs per tile and the commits.
+//   epilogue (1 warpgroup)  : drains a finished group buffer (tcgen05.ld), multiplies by the group's
+//                             fp32 scale, accumulates in registers, and at the end of a piece writes
+//                             bf16 rows to their ORIGINAL positions (fused un-permutation) or parks an
+//                             fp32 partial sum.
+//
+// Work split ("stream-K" over packed tiles): all tiles of the call form one sequence
+// [expert][channel tile nt][k-block kb]; tile (e, nt, kb) costs w[e].  CTA c of G owns the tiles
+// whose start cost lies in [c*C/G, (c+1)*C/G) -- equal work to within one tile, at most two partial
+// pieces per CTA.  Partial sums go to the workspace; the CTA that announces last for an (expert, nt)
+// segment adds them in CTA order (deterministic) and stores the rows.
+//
+// Takes experts that are per-channel or have groups of 128 k or more, and batches of at most 16
+// rows; the caller routes everything else to the other kernels.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, latches
+// MOQE_ERR_TIMEOUT, lets copies in flight land, frees its TMEM and returns.
+//
+// The operation is Section 3.1 of the paper (the selected quantization expert runs the sample);
+// the paper describes no kernel.
+#include <type_traits>
+
+#include "dequant.cuh"
+#include "tc_ptx.cuh"
+
+namespace moqe {
+namespace {
+
+constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
+constexpr int DQ_WARPS = 16, EP_WARP0 = 16, MMA_WARP = 20, W_WARP = 21;
+constexpr int DEC_THREADS = 22 * 32;
+constexpr int RING_BYTES = 168 * 1024;                  // packed-weight ring
+constexpr int MAX_STAGES = 16;
+constexpr int NA = 4;                                   // A-operand buffers in TMEM (64 columns each), one per warpgroup
+constexpr int ND = 4;                                   // accumulator buffers (TOK columns each)
+constexpr int NXS = 8;                                  // token-tile stages
+constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
+constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
+constexpr int SCALE_SLOTS = 16;                         // group scales handed from the dequant to the epilogue threads
+constexpr int TMEM_COLS = 512;
+constexpr int D_COL0 = NA * 64;
+
+struct DecSmem {
+    static constexpr int ring_off = 0;
+    static constexpr int x_off = RING_BYTES;
+    static constexpr int scale_off = x_off + NXS * X_STAGE;
+    static constexpr int bar_off = scale_off + SCALE_SLOTS * 512;
+    // wfull[16] wempty[16] afull[NA] done[8] accfull[ND] accempty[ND] esync
+    static constexpr int n_bars = 2 * MAX_STAGES + NA + DONE_RING + 2 * ND + 1;
+    static constexpr int misc_off = bar_off + n_bars * 8;              // tmem address, abort flag, ring geometry
+    static constexpr int off_off = misc_off + 32;
+    static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;   // perm of the batch's rows
+    static constexpr int rng_off = perm_off + TOK * 4;
+    static constexpr int red_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // reduction verdicts
+    static constexpr int total = red_off + 32;
+    static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
+};
+
+struct DecSched {
+    long long C;            // total cost
+    int G, E, KB, TT;       // CTAs, experts, k-blocks per segment, tiles per expert (= ntiles * KB)
+    int w[MOQE_MAX_EXPERTS];
+};
+
+struct DecParams {
+    ExpertDev ex[MOQE_MAX_EXPERTS];
+    DecSched sched;
+    const uint16_t* X;
+    uint16_t* Y;
+    const int32_t* perm;
+    const int32_t* offsets;
+    float* partials;        // [CTA][slot 0/1][TOK][128]
+    uint32_t* counters;     // [expert][ntiles], zero on entry, left zero
+    int* status;
+    int M, N, K, KB, ntiles;
+};
+
+__device__ __forceinline__ long long dsched_base(const DecSched& s, int e) {
+    long long b = 0;
+    for (int i = 0; i < e; ++i) b += (long long)s.TT * s.w[i];
+    return b;
+}
+// first tile of expert e owned by CTA c or a later CTA
+__device__ __forceinline__ int dsched_tbegin(const DecSched& s, int c, int e, long long base) {
+    const long long num = (long long)c * s.C - base * s.G;
+    if (num <= 0) return 0;
+    const long long den = (long long)s.w[e] * s.G;
+    const long long t = (num + den - 1) / den;
+    return t > s.TT ? s.TT : (int)t;
+}
+__device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long base, int t) {
+    return (int)(((base + (long long)t * s.w[e]) * s.G) / s.C);
+}
+
+// Does an accumulation group END with k-block kb?  Per-channel experts: the piece is one group.  Groups of 128 k or
+// more: a group ends with its last k-block or with the piece (the scale is constant over the group, so a piece may
+// cut it).
+__device__ __forceinline__ bool group_ends(int group, int kb, bool last) {
+    if (last || group == 128) return true;
+    if (group == 0) return false;
+    return ((kb + 1) * 128) % group == 0;
+}
+
+// Walks the tiles of one CTA in order: pieces (expert e, channel tile nt, k-blocks [kb0, kb1)) of the CTA's
+// cost range, experts without rows skipped.  rng[2e], rng[2e+1] = the CTA's tile range inside expert e.
+struct TileWalk {
+    int e = -1, tb = 0, te = 0;          // expert and the rest of the CTA's tile range in it
+    int nt = 0, kb0 = 0, kb1 = 0, kb = 0;   // current piece and k-block
+    int row0 = 0, rows = 0;
+    int group = 0, bits = 0, has_zeros = 0, stride = 0;   // the expert's format, read once per expert: per-tile code touches registers only
+    const uint8_t* tiles = nullptr;
+    bool valid = false;
+    __device__ __forceinline__ bool next_piece(const DecParams& p, const volatile int* rng, const volatile int* off) {
+        const DecSched& s = p.sched;
+        for (;;) {
+            if (e >= 0 && tb < te) {
+                nt = tb / s.KB;
+                kb0 = tb - nt * s.KB;
+                const int len = min(s.KB - kb0, te - tb);
+                kb1 = kb0 + len;
+                tb += len;
+                kb = kb0;
+                return true;
+            }
+            for (;;) {
+                if (++e >= s.E) return false;
+                row0 = off[e];
+                rows = min(off[e + 1] - row0, TOK);
+                if (rows > 0) break;
+            }
+            group = p.ex[e].group; bits = p.ex[e].bits; has_zeros = p.ex[e].has_zeros; stride = p.ex[e].tile_stride;
+            tiles = p.ex[e].tiles;
+            tb = rng[2 * e];
+            te = rng[2 * e + 1];
+        }
+    }
+    __device__ __forceinline__ void init(const DecParams& p, const volatile int* rng, const volatile int* off) {
+        valid = next_piece(p, rng, off);
+    }
+    __device__ __forceinline__ void step(const DecParams& p, const volatile int* rng, const volatile int* off) {
+        if (++kb == kb1) valid = next_piece(p, rng, off);
+    }
+    // does an accumulation group end with the current k-block?
+    __device__ __forceinline__ bool ends() const { return group_ends(group, kb, kb + 1 == kb1); }
+    __device__ __forceinline__ bool first() const { return kb == kb0; }
+    __device__ __forceinline__ bool last() const { return kb + 1 == kb1; }
+    __device__ __forceinline__ bool whole(int KB) const { return kb0 == 0 && kb1 == KB; }
+};
+
+// ---------------------------------------------------------------------------- dequant role
+// Chunk G (8 consecutive k) of a piece as four bf16x2 registers holding the exact integers c - z.  `zc` is the
+// tile's zero-point constant, packed once per tile: bf16x2(128 + z) for 4- and 3-bit codes (0x4300 | c is the
+// bf16 number 128 + c), bf16x2(-z * 2^-13) for 8-bit codes (a zero-extended byte is the bf16 number c * 2^-133;
+// one FMA with 2^120 gives (c - z) * 2^-13, and the fp32 scale carries the 2^13).
+template <int BITS, int G>
+__device__ __forceinline__ void unpack_chunk_zc(const uint32_t (&w)[PieceWords<BITS>::n], uint32_t zc, uint32_t* out) {
+    if constexpr (BITS == 4) {
+        const uint32_t v = w[G];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = hsub2_bf16(((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zc);
+    } else if constexpr (BITS == 3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int pr = 4 * G + i;                 // pair index inside the piece
+            uint32_t v;
+            if (pr < 15) v = (w[pr / 5] >> (3 * (pr % 5))) & 0x00070007u;
+            else v = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u);
+            out[i] = hsub2_bf16(v | 0x43004300u, zc);
+        }
+    } else {
+        const uint32_t k120 = 0x7B807B80u;           // 2^120 in both halves
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t pair = __byte_perm(w[2 * G + (i >> 1)], 0u, (i & 1) ? 0x4342u : 0x4140u);
+            __nv_bfloat162 r = __hfma2(*reinterpret_cast<const __nv_bfloat162*>(&pair), *reinterpret_cast<const __nv_bfloat162*>(&k120),
+                                       *reinterpret_cast<const __nv_bfloat162*>(&zc));
+            out[i] = *reinterpret_cast<uint32_t*>(&r);
+        }
+    }
+}
+
+// One packed tile -> operand A in tensor memory, for the thread that owns channel row `row` (= its TMEM lane).
+// MMA k index k' = 32q + 8G + t holds the code of real k = 32G + 8q + t (piece q, chunk G): a piece then fills 16
+// consecutive TMEM columns with one store, and the token-tile loader applies the same permutation to its
+// 16-byte chunks.
+template <int BITS>
+__device__ __forceinline__ void dequant_tile(const unsigned char* stage, int row, uint32_t zc, uint32_t a_taddr) {
+    const unsigned char* blob = stage + (row >> 4) * moqe_blob_bytes(BITS);
+    const int half = (row >> 3) & 1, r = row & 7;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t w[PieceWords<BITS>::n];
+        load_piece_smem<BITS>(blob, half, q * 8 + (r ^ (2 * q)), w);
+        uint32_t o[16];
+        unpack_chunk_zc<BITS, 0>(w, zc, o);
+        unpack_chunk_zc<BITS, 1>(w, zc, o + 4);
+        unpack_chunk_zc<BITS, 2>(w, zc, o + 8);
+        unpack_chunk_zc<BITS, 3>(w, zc, o + 12);
+        tmem_st16(a_taddr + 16 * q, o);
+    }
+}
+
+// The token rows of one tile (expert rows [row0, row0 + rows) of the sorted batch, k-block kb) as a K-major,
+// 128-byte-swizzled UMMA operand: two halves of 64 k', each TOK rows x 128 bytes; 16-byte chunk (G, q) of real k
+// goes to chunk 4q + G of k'.  Issued by the 128 threads of one warpgroup (t = thread index in it); k >= K is
+// zero-filled.  Rows beyond `rows` are left as they are: their columns of the accumulator are never read.
+__device__ __forceinline__ void load_token_tile(const DecParams& p, const volatile int* s_perm, uint32_t xs, int row0, int rows, int kb,
+                                                int t) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int id = t + 128 * i, m = id >> 4, a = id & 15;
+        if (m < rows) {
+            const int src_row = s_perm[row0 + m];
+            const int k = kb * 128 + a * 8;
+            const int nbytes = max(0, min(16, (p.K - k) * 2));
+            const uint16_t* src = nbytes > 0 ? p.X + (size_t)src_row * p.K + k : p.X;
+            const int ap = 4 * (a & 3) + (a >> 2);
+            cp_async16(xs + (ap >> 3) * (TOK * 128) + m * 128 + (((ap & 7) ^ (m & 7)) << 4), src, nbytes);
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __grid_constant__ DecParams p) {
+    using L = DecSmem;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::bar_off;
+    const uint32_t bar_wfull = bar0, bar_wempty = bar0 + 8 * MAX_STAGES, bar_afull = bar_wempty + 8 * MAX_STAGES;
+    const uint32_t bar_done = bar_afull + 8 * NA, bar_accfull = bar_done + 8 * DONE_RING;
+    const uint32_t bar_accempty = bar_accfull + 8 * ND, bar_esync = bar_accempty + 8 * ND;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::misc_off);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
+    volatile int* s_geom = reinterpret_cast<volatile int*>(smem + L::misc_off + 8);    // {stages, stage bytes}
+    volatile int* s_off = reinterpret_cast<volatile int*>(smem + L::off_off);
+    volatile int* s_rng = reinterpret_cast<volatile int*>(smem + L::rng_off);
+    volatile int* s_perm = reinterpret_cast<volatile int*>(smem + L::perm_off);
+    volatile int* s_red = reinterpret_cast<volatile int*>(smem + L::red_off);
+    float* s_scale = reinterpret_cast<float*>(smem + L::scale_off);
+    const DecSched& sch = p.sched;
+    // warp-uniform bounded wait: every lane polls, the warp agrees on the verdict
+    auto wwait = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(bar, parity, s_abort, p.status));
+    };
+    // one arrival per warp, after all its lanes are done with what the barrier hands over
+    auto warrive = [&](uint32_t bar) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar);
+    };
+    // done[t % 8] completes when the MMAs of the CTA's t-th tile have
+    auto wait_done = [&](int t) -> bool {
+        return t < 0 || wwait(bar_done + 8 * (t & (DONE_RING - 1)), (uint32_t)(t >> 3) & 1u);
+    };
+
+    // ---- prologue: launch parameters only, so it may overlap the tail of the previous kernel in the stream
+    if (tid == 0) {
+        for (int i = 0; i < MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, 4); }
+        for (int i = 0; i < NA; ++i) mbar_init(bar_afull + 8 * i, 4);
+        for (int i = 0; i < DONE_RING; ++i) mbar_init(bar_done + 8 * i, 1);
+        for (int i = 0; i < ND; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accempty + 8 * i, 4); }
+        mbar_init(bar_esync, 128);
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid >= 32 && tid < 32 + sch.E) {                    // this CTA's tile range inside each expert
+        const int e = tid - 32;
+        const long long base = dsched_base(sch, e);
+        s_rng[2 * e] = dsched_tbegin(sch, blockIdx.x, e, base);
+        s_rng[2 * e + 1] = dsched_tbegin(sch, blockIdx.x + 1, e, base);
+    }
+    if (warp == MMA_WARP) tmem_alloc(sbase + L::misc_off, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0) {
+        // ring stage = the largest packed tile among the experts this CTA's share touches
+        int wmax = 0;
+        for (int e = 0; e < sch.E; ++e)
+            if (s_rng[2 * e] < s_rng[2 * e + 1]) wmax = max(wmax, p.ex[e].tile_stride);
+        const int stage_bytes = (max(wmax, 128) + 127) & ~127;
+        s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
+        s_geom[1] = stage_bytes;
+    }
+    // from here on the previous kernel's results are needed (sort tables, activations, workspace)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid <= sch.E) s_off[tid] = p.offsets[tid];
+    if (tid >= 64 && tid < 64 + TOK) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+    __syncthreads();
+    const uint32_t tmem_base = *s_tmem;
+    const int nstg = s_geom[0], stage_bytes = s_geom[1];
+    TileWalk tw;
+    tw.init(p, s_rng, s_off);
+
+    if (warp == W_WARP) {
+        // ------------------------------------------------------------------ packed-weight producer
+        if (lane == 0) {
+            Ring ring;
+            for (; tw.valid; tw.step(p, s_rng, s_off)) {
+                const uint32_t wbytes = (uint32_t)tw.stride;
+                if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) break;
+                const uint32_t full = bar_wfull + 8 * ring.stage;
+                mbar_expect_tx(full, wbytes);
+                bulk_load(sbase + L::ring_off + ring.stage * stage_bytes,
+                          tw.tiles + ((size_t)tw.nt * p.KB + tw.kb) * wbytes, wbytes, full);
+                ring.advance(nstg);
+            }
+        }
+    } else if (warp == MMA_WARP) {
+        // ------------------------------------------------------------------ MMA issuer
+        // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.
+        const uint32_t idesc = umma_idesc(TOK);
+        int g = 0;                                   // accumulation groups started so far
+        bool fresh = true;                           // the next MMA starts a group
+        for (int t = 0; tw.valid; tw.step(p, s_rng, s_off), ++t) {
+            const int a = t & (NA - 1), d = g & (ND - 1);
+            const bool ends = tw.ends();
+            if (!wwait(bar_afull + 8 * a, (uint32_t)(t >> 2) & 1u)) break;
+            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(g >> 2) & 1u) ^ 1u)) break;
+            tc_fence_after();
+            const uint32_t xs = sbase + L::x_off + (t & (NXS - 1)) * X_STAGE;
+            const uint32_t dt = tmem_base + D_COL0 + d * TOK, a0 = tmem_base + a * 64;
+            const uint64_t b0 = umma_desc_sw128(xs), b1 = umma_desc_sw128(xs + TOK * 128);
+            if (elect_one()) {
+                umma_bf16_ts(dt, a0, b0, idesc, fresh ? 0u : 1u);
+                umma_bf16_ts(dt, a0 + 8, b0 + 2, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 16, b0 + 4, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 24, b0 + 6, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 32, b1, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 40, b1 + 2, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 48, b1 + 4, idesc, 1u);
+                umma_bf16_ts(dt, a0 + 56, b1 + 6, idesc, 1u);
+                if (ends) umma_commit(bar_accfull + 8 * d);
+                umma_commit(bar_done + 8 * (t & (DONE_RING - 1)));
+            }
+            __syncwarp();
+            fresh = ends;
+            if (ends) ++g;
+        }
+    } else if (warp < DQ_WARPS) {
+        // ------------------------------------------------------------------ dequant warpgroups
+        const int wg = warp >> 2, row = (warp & 3) * 32 + lane, twg = tid & 127;
+        const uint32_t a_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + wg * 64;
+        Ring ring;
+        int g = 0;
+        TileWalk xw = tw;                            // runs ahead: the warpgroup's next tile, for its token rows
+        int xt = 0;
+        auto x_seek = [&](int target) {              // move xw to tile `target` (or past the end)
+            for (; xw.valid && xt < target; ++xt) xw.step(p, s_rng, s_off);
+        };
+        x_seek(wg);
+        if (xw.valid) load_token_tile(p, s_perm, sbase + L::x_off + (xt & (NXS - 1)) * X_STAGE, xw.row0, xw.rows, xw.kb, twg);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        bool ok = true;
+        for (int t = 0; ok && tw.valid; tw.step(p, s_rng, s_off), ++t, ring.advance(nstg)) {
+            const bool ends = tw.ends();
+            if ((t & 3) == wg) {
+                // the warpgroup's previous tile is done: its A buffer and its token-tile stage (t + 4) % 8 are free
+                if (!(ok = wait_done(t - 4))) break;
+                x_seek(t + 4);
+                if (xw.valid) load_token_tile(p, s_perm, sbase + L::x_off + (xt & (NXS - 1)) * X_STAGE, xw.row0, xw.rows, xw.kb, twg);
+                else asm volatile("cp.async.commit_group;" ::: "memory");
+                if (!(ok = wwait(bar_wfull + 8 * ring.stage, ring.phase))) break;
+                tc_fence_after();
+                const unsigned char* stage = smem + L::ring_off + ring.stage * stage_bytes;
+                // zero-point of this row for the tile: the tile's own meta, the per-channel array, or 2^(bits-1)
+                float z = (float)(1 << (tw.bits - 1));
+                if (tw.has_zeros)
+                    z = tw.group == 0 ? __bfloat162float(p.ex[tw.e].zeros_pc[tw.nt * 128 + row])
+                                      : __bfloat162float(moqe_tile_zeros(stage, tw.bits, 0)[row]);
+                if (tw.bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
+                else if (tw.bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), a_taddr);
+                else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
+                // the scale of a group that ends in this tile, for the epilogue thread of the same row
+                if (ends && tw.group != 0)
+                    s_scale[(g & (SCALE_SLOTS - 1)) * 128 + row] =
+                        __half2float(moqe_tile_scales(stage, tw.bits, tw.has_zeros, 0)[row]) * (tw.bits == 8 ? W8_PRESCALE : 1.f);
+                warrive(bar_wempty + 8 * ring.stage);
+                asm volatile("cp.async.wait_group 1;" ::: "memory");      // this tile's token rows have landed
+                fence_proxy_async();
+                tmem_st_wait();
+                tc_fence_before();
+                warrive(bar_afull + 8 * (t & (NA - 1)));
+            }
+            if (ends) ++g;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (warp >= EP_WARP0 && warp < EP_WARP0 + 4) {
+        // ------------------------------------------------------------------ epilogue warpgroup
+        const int et = tid - EP_WARP0 * 32, row = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + D_COL0;
+        uint32_t esync_phase = 0;
+        int g = 0, n_pending = 0;
+        int pend_e[2], pend_nt[2], pend_j0[2], pend_rows[2];
+        float acc[TOK];
+        float pc_s = 0.f;
+        bool ok = true;
+        for (; ok && tw.valid; tw.step(p, s_rng, s_off)) {
+            const int n = tw.nt * 128 + row;
+            if (tw.first()) {
+#pragma unroll
+                for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
+                if (tw.group == 0) pc_s = __half2float(p.ex[tw.e].scales_pc[n]) * (tw.bits == 8 ? W8_PRESCALE : 1.f);
+            }
+            if (tw.ends()) {
+                const int d = g & (ND - 1);
+                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(g >> 2) & 1u))) break;
+                tc_fence_after();
+                const float s = tw.group == 0 ? pc_s : s_scale[(g & (SCALE_SLOTS - 1)) * 128 + row];
+                uint32_t v[16];
+                tmem_ld16(lane_base + d * TOK, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = fmaf(s, __uint_as_float(v[i]), acc[i]);
+                tc_fence_before();
+                warrive(bar_accempty + 8 * d);
+                ++g;
+            }
+            if (!tw.last()) continue;
+            const int j0 = tw.row0, rows = tw.rows;
+            if (tw.whole(p.KB)) {
+                // the whole K of this segment was ours: round and store rows at their original positions
+                if (n < p.N) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m)
+                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                }
+            } else {
+                // partial sum: park it in this CTA's slot (0: the piece starts inside its segment, 1: at its start)
+                float* dst = p.partials + ((size_t)(blockIdx.x * 2 + (tw.kb0 != 0 ? 0 : 1)) * TOK) * 128 + row;
+#pragma unroll
+                for (int m = 0; m < TOK; ++m)
+                    if (m < rows) dst[m * 128] = acc[m];
+                if (n_pending < 2) {
+                    pend_e[n_pending] = tw.e; pend_nt[n_pending] = tw.nt; pend_j0[n_pending] = j0; pend_rows[n_pending] = rows;
+                    ++n_pending;
+                }
+            }
+        }
+        // ---- announce the parked pieces; whoever announces last for a segment adds its pieces up in CTA order
+        if (ok && n_pending > 0) {
+            __threadfence();
+            mbar_arrive(bar_esync);
+            ok = wwait(bar_esync, esync_phase);
+            esync_phase ^= 1u;
+            if (ok && et == 0) {
+                for (int i = 0; i < n_pending; ++i) {
+                    const long long base = dsched_base(sch, pend_e[i]);
+                    const int t0 = pend_nt[i] * p.KB;
+                    const int c_first = dsched_owner(sch, pend_e[i], base, t0);
+                    const int c_last = dsched_owner(sch, pend_e[i], base, t0 + p.KB - 1);
+                    unsigned* cnt = p.counters + (size_t)pend_e[i] * p.ntiles + pend_nt[i];
+                    const unsigned old = atomicAdd(cnt, 1u);
+                    const int last = old == (unsigned)(c_last - c_first) ? 1 : 0;
+                    if (last) *cnt = 0u;                               // leave the counters clear for the next call
+                    s_red[4 * i] = last; s_red[4 * i + 1] = c_first; s_red[4 * i + 2] = c_last - c_first + 1;
+                }
+                __threadfence();
+            }
+            if (ok) {
+                mbar_arrive(bar_esync);
+                ok = wwait(bar_esync, esync_phase);
+                esync_phase ^= 1u;
+            }
+            for (int i = 0; ok && i < n_pending; ++i) {
+                if (!s_red[4 * i]) continue;
+                const int c_first = s_red[4 * i + 1], n_contrib = s_red[4 * i + 2];
+                const int e = pend_e[i], nt = pend_nt[i], rows = pend_rows[i], n = nt * 128 + row;
+                const long long base = dsched_base(sch, e);
+                float sum[TOK];
+#pragma unroll
+                for (int m = 0; m < TOK; ++m) sum[m] = 0.f;
+                for (int ci = 0; ci < n_contrib; ++ci) {
+                    const int cc = c_first + ci;
+                    const int slot = dsched_tbegin(sch, cc, e, base) <= nt * p.KB ? 1 : 0;
+                    const float* src = p.partials + ((size_t)(cc * 2 + slot) * TOK) * 128 + row;
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m)
+                        if (m < rows) sum[m] += __ldcg(src + m * 128);
+                }
+                if (n < p.N) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m)
+                        if (m < rows) p.Y[(size_t)s_perm[pend_j0[i] + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum[m]));
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*s_abort) {
+        // let bulk copies that may still be in flight land before the shared memory is released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == MMA_WARP) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+int g_dec_sm_count = 0;
+int dec_sm_count() {
+    if (!g_dec_sm_count) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&g_dec_sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (g_dec_sm_count <= 0) g_dec_sm_count = 148;
+    }
+    return g_dec_sm_count;
+}
+
+constexpr int DEC_MAX_GRID = 256;             // bound on CTAs the partial slots are sized for
+
+// relative cost of one packed tile in the work split; 0 = its bytes
+int g_dec_tile_cost[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+
+}  // namespace
+
+void decode_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost >= 0) g_dec_tile_cost[bits] = cost; }
+
+bool decode_supported(int M, const moqe_expert* const* ex, int E) {
+    if (M > DECODE_MAX_ROWS) return false;
+    for (int e = 0; e < E; ++e)
+        if (ex[e]->group != 0 && (ex[e]->group < 128 || ex[e]->group % 128 != 0)) return false;
+    return true;
+}
+
+size_t decode_zero_bytes(int M, int Np) {
+    if (M > DECODE_MAX_ROWS) return 0;
+    return (size_t)MOQE_MAX_EXPERTS * (Np / 128) * sizeof(uint32_t);
+}
+
+size_t decode_workspace_bytes(int M, int Np, int E) {
+    (void)E;
+    if (M > DECODE_MAX_ROWS) return 0;
+    const size_t counters = (decode_zero_bytes(M, Np) + 255) / 256 * 256;
+    const size_t partials = (size_t)DEC_MAX_GRID * 2 * TOK * 128 * sizeof(float);
+    return counters + partials;
+}
+
+moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
+                                const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
+    if (M == 0) return MOQE_OK;
+    if (!decode_supported(M, ex, E)) return MOQE_ERR_UNSUPPORTED;
+    DecParams p;
+    p.KB = ex[0]->Kp / 128;
+    p.ntiles = ex[0]->Np / 128;
+    DecSched& s = p.sched;
+    s.E = E;
+    s.KB = p.KB;
+    s.TT = p.ntiles * p.KB;
+    s.C = 0;
+    int wmax = 1;
+    for (int e = 0; e < E; ++e) {
+        p.ex[e] = ex[e]->dev();
+        const int cost = g_dec_tile_cost[ex[e]->bits];
+        s.w[e] = cost > 0 ? cost : p.ex[e].tile_stride / 256;
+        s.C += (long long)s.TT * s.w[e];
+        wmax = s.w[e] > wmax ? s.w[e] : wmax;
+    }
+    // every CTA's cost share must be at least one tile of the dearest kind, so that every CTA between the owners of
+    // a segment's first and last tile really owns a tile of it (the reduction counts them)
+    int grid = dec_sm_count();
+    if (grid > DEC_MAX_GRID) grid = DEC_MAX_GRID;
+    const long long work_items = s.C / wmax;
+    if (work_items < grid) grid = work_items < 1 ? 1 : (int)work_items;
+    s.G = grid;
+    if (!ws || ws_bytes < decode_workspace_bytes(M, ex[0]->Np, E)) return MOQE_ERR_WORKSPACE;
+    p.counters = (uint32_t*)ws;
+    p.partials = (float*)((char*)ws + (decode_zero_bytes(M, ex[0]->Np) + 255) / 256 * 256);
+    p.X = (const uint16_t*)X;
+    p.Y = (uint16_t*)Y;
+    p.perm = perm;
+    p.offsets = offsets;
+    p.M = M; p.N = N; p.K = K;
+    p.status = device_status_word();
+    static bool attr_set = false;
+    cudaError_t err = cudaSuccess;
+    if (!attr_set) {
+        err = cudaFuncSetAttribute(qgemm_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecSmem::dyn_bytes);
+        attr_set = (err == cudaSuccess);
+    }
+    if (err == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = DecSmem::dyn_bytes; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, qgemm_decode_kernel, p);
+    }
+    if (err != cudaSuccess) return MOQE_ERR_CUDA;
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace moqe

@@ -70,6 +70,46 @@ def test_all_formats_small_shapes(path, M, N, K):
     assert_close(Y, oracle.routed_gemm(X, ids, What), f"M{M} N{N} K{K}")
 
 
+DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True), (4, 0, False), (8, 128, False),
+                  (4, 256, False), (3, 0, True), (8, 0, False), (3, 256, True)]
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (13, 136, 2304), (16, 1000, 640),
+                                   (7, 4096, 1024), (16, 512, 11008)])
+def test_decode_kernel_all_formats(M, N, K):
+    """The tcgen05 decode kernel (path 5: at most 16 rows, per-channel experts or groups of >= 128 k): every such
+    format as its own expert, ragged N, K not a multiple of 128, split K with several contributors per segment,
+    an expert that gets no rows."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close
+    specs = [f for f in DECODE_FORMATS if f[1] == 0 or K % f[1] == 0]
+    W = wl.weights_f32(f"dq/{N}/{K}", N, K)
+    X = wl.activations_bf16(f"dq/{M}/{K}", M, K)
+    gpu, What, _ = build_experts(W, specs)
+    rs = np.random.default_rng(7 * M + N + K)
+    ids = rs.integers(0, len(specs), size=M).astype(np.int32)
+    if M > 4:
+        ids[ids == 2] = 0                                        # expert 2 idle
+    for _ in range(2):                                           # twice: the arrival counters must come back to zero
+        Y, st = _run(X, ids, gpu, moqe.PATH_DECODE)
+        assert st == moqe.OK
+        assert_close(Y, oracle.routed_gemm(X, ids, What), f"decode M{M} N{N} K{K}")
+    # batch shuffle: rows move with their inputs, bit for bit
+    pm = rs.permutation(M)
+    Yp, _ = _run(X[pm], ids[pm], gpu, moqe.PATH_DECODE)
+    assert np.array_equal(Yp, Y[pm])
+
+
+def test_decode_kernel_refuses_what_it_cannot_take():
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, dev, bf16_to_torch
+    W = wl.weights_f32("dq/refuse", 128, 256)
+    gpu, _, _ = build_experts(W, [(4, 32, False)])
+    X = wl.activations_bf16("dq/refuse/X", 4, 256)
+    with pytest.raises(Exception):
+        moqe.moqe_routed_qgemm(bf16_to_torch(X), torch.zeros(4, dtype=torch.int32, device=dev()), gpu, path=moqe.PATH_DECODE)
+
+
 @pytest.mark.parametrize("path", [1, 3, 4])
 def test_exact_integer_case_on_gpu(path):
     """On-grid W8 weights with power-of-two scale and small-integer activations: the exact int64 product."""
@@ -149,7 +189,7 @@ def test_argument_errors():
     assert ei.value.code == moqe.ERR_WORKSPACE
 
 
-@pytest.mark.parametrize("path,M", [(1, 16), (1, 48), (3, 300)])
+@pytest.mark.parametrize("path,M", [(1, 16), (1, 48), (3, 300), (5, 16), (5, 9)])
 def test_presorted_entry_point_matches(path, M):
     """moqe_permute once + moqe_routed_qgemm_sorted per layer == moqe_routed_qgemm, bit for bit, call after call
     (the split-K arrival counters must come back to zero by themselves)."""
