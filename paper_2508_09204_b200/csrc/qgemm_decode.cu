@@ -51,7 +51,7 @@ namespace {
 constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
 constexpr int DQ_WARPS = 16, EP_WARP0 = 16, MMA_WARP = 20, W_WARP = 21;
 constexpr int DEC_THREADS = 22 * 32;
-constexpr int RING_BYTES = 168 * 1024;                  // packed-weight ring
+constexpr int RING_BYTES = 160 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 4;                                   // A-operand buffers in TMEM (64 columns each), one per warpgroup
 constexpr int ND = 4;                                   // accumulator buffers (TOK columns each)
@@ -61,6 +61,7 @@ constexpr int DONE_RING = 8;                            // "MMAs of tile t have 
 constexpr int SCALE_SLOTS = 16;                         // group scales handed from the dequant to the epilogue threads
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL0 = NA * 64;
+constexpr int MAX_TILES = 512;                          // tiles one CTA can take (its tile table)
 
 struct DecSmem {
     static constexpr int ring_off = 0;
@@ -74,7 +75,9 @@ struct DecSmem {
     static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;   // perm of the batch's rows
     static constexpr int rng_off = perm_off + TOK * 4;
     static constexpr int red_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // reduction verdicts
-    static constexpr int total = red_off + 32;
+    static constexpr int ex_off = red_off + 32;                        // ExpertSm[MOQE_MAX_EXPERTS]
+    static constexpr int tile_off = ex_off + MOQE_MAX_EXPERTS * 48;    // uint4[MAX_TILES]
+    static constexpr int total = tile_off + MAX_TILES * 16;
     static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
 };
 
@@ -114,59 +117,32 @@ __device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long 
     return (int)(((base + (long long)t * s.w[e]) * s.G) / s.C);
 }
 
-// Does an accumulation group END with k-block kb?  Per-channel experts: the piece is one group.  Groups of 128 k or
-// more: a group ends with its last k-block or with the piece (the scale is constant over the group, so a piece may
-// cut it).
-__device__ __forceinline__ bool group_ends(int group, int kb, bool last) {
-    if (last || group == 128) return true;
-    if (group == 0) return false;
-    return ((kb + 1) * 128) % group == 0;
-}
+// The CTA's tiles, in order, as a table in shared memory (one 16-byte entry per tile), built once by the whole CTA
+// after the routing offsets are known: every role then reads its tile with one load instead of walking pieces.
+//   x = kb | nt << 16        y = flags | e << 8 | rows << 16 | row0 << 24        z = accumulation-group index g
+// An accumulation group (one accumulator buffer handed to the epilogue) is: the whole piece for per-channel
+// experts; for groups of 128 k or more, the k-blocks of one quantization group inside the piece (the scale is
+// constant over the group, so a piece may cut it).
+constexpr int TF_FIRST = 1, TF_LAST = 2, TF_ENDS = 4, TF_WHOLE = 8, TF_KB0NZ = 16;
 
-// Walks the tiles of one CTA in order: pieces (expert e, channel tile nt, k-blocks [kb0, kb1)) of the CTA's
-// cost range, experts without rows skipped.  rng[2e], rng[2e+1] = the CTA's tile range inside expert e.
-struct TileWalk {
-    int e = -1, tb = 0, te = 0;          // expert and the rest of the CTA's tile range in it
-    int nt = 0, kb0 = 0, kb1 = 0, kb = 0;   // current piece and k-block
-    int row0 = 0, rows = 0;
-    int group = 0, bits = 0, has_zeros = 0, stride = 0;   // the expert's format, read once per expert: per-tile code touches registers only
-    const uint8_t* tiles = nullptr;
-    bool valid = false;
-    __device__ __forceinline__ bool next_piece(const DecParams& p, const volatile int* rng, const volatile int* off) {
-        const DecSched& s = p.sched;
-        for (;;) {
-            if (e >= 0 && tb < te) {
-                nt = tb / s.KB;
-                kb0 = tb - nt * s.KB;
-                const int len = min(s.KB - kb0, te - tb);
-                kb1 = kb0 + len;
-                tb += len;
-                kb = kb0;
-                return true;
-            }
-            for (;;) {
-                if (++e >= s.E) return false;
-                row0 = off[e];
-                rows = min(off[e + 1] - row0, TOK);
-                if (rows > 0) break;
-            }
-            group = p.ex[e].group; bits = p.ex[e].bits; has_zeros = p.ex[e].has_zeros; stride = p.ex[e].tile_stride;
-            tiles = p.ex[e].tiles;
-            tb = rng[2 * e];
-            te = rng[2 * e + 1];
-        }
-    }
-    __device__ __forceinline__ void init(const DecParams& p, const volatile int* rng, const volatile int* off) {
-        valid = next_piece(p, rng, off);
-    }
-    __device__ __forceinline__ void step(const DecParams& p, const volatile int* rng, const volatile int* off) {
-        if (++kb == kb1) valid = next_piece(p, rng, off);
-    }
-    // does an accumulation group end with the current k-block?
-    __device__ __forceinline__ bool ends() const { return group_ends(group, kb, kb + 1 == kb1); }
-    __device__ __forceinline__ bool first() const { return kb == kb0; }
-    __device__ __forceinline__ bool last() const { return kb + 1 == kb1; }
-    __device__ __forceinline__ bool whole(int KB) const { return kb0 == 0 && kb1 == KB; }
+struct ExpertSm {            // per-expert facts of this CTA, in shared memory
+    int tb, te;              // the CTA's tile range inside the expert ([nt][kb] order); empty if the expert has no rows
+    int cum;                 // tiles of earlier experts
+    int gbase;               // accumulation groups of earlier experts
+    int gkb;                 // k-blocks per accumulation group (KB for per-channel experts)
+    int row0, rows;
+    int bits, group, has_zeros, stride;
+    int pad;
+};
+
+struct Tile {
+    int kb, nt, flags, e, rows, row0, g;
+    __device__ __forceinline__ explicit Tile(const uint4& v)
+        : kb((int)(v.x & 0xFFFFu)), nt((int)(v.x >> 16)), flags((int)(v.y & 0xFFu)), e((int)((v.y >> 8) & 0xFFu)),
+          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z) {}
+    __device__ __forceinline__ bool first() const { return flags & TF_FIRST; }
+    __device__ __forceinline__ bool last() const { return flags & TF_LAST; }
+    __device__ __forceinline__ bool ends() const { return flags & TF_ENDS; }
 };
 
 // ---------------------------------------------------------------------------- dequant role
@@ -256,11 +232,13 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     const uint32_t bar_accempty = bar_accfull + 8 * ND, bar_esync = bar_accempty + 8 * ND;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::misc_off);
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
-    volatile int* s_geom = reinterpret_cast<volatile int*>(smem + L::misc_off + 8);    // {stages, stage bytes}
+    volatile int* s_geom = reinterpret_cast<volatile int*>(smem + L::misc_off + 8);    // {stages, stage bytes, tiles}
     volatile int* s_off = reinterpret_cast<volatile int*>(smem + L::off_off);
     volatile int* s_rng = reinterpret_cast<volatile int*>(smem + L::rng_off);
     volatile int* s_perm = reinterpret_cast<volatile int*>(smem + L::perm_off);
     volatile int* s_red = reinterpret_cast<volatile int*>(smem + L::red_off);
+    ExpertSm* s_ex = reinterpret_cast<ExpertSm*>(smem + L::ex_off);
+    const uint4* s_tile = reinterpret_cast<const uint4*>(smem + L::tile_off);
     float* s_scale = reinterpret_cast<float*>(smem + L::scale_off);
     const DecSched& sch = p.sched;
     // warp-uniform bounded wait: every lane polls, the warp agrees on the verdict
@@ -294,40 +272,74 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         s_rng[2 * e + 1] = dsched_tbegin(sch, blockIdx.x + 1, e, base);
     }
     if (warp == MMA_WARP) tmem_alloc(sbase + L::misc_off, TMEM_COLS);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (tid == 0) {
-        // ring stage = the largest packed tile among the experts this CTA's share touches
-        int wmax = 0;
-        for (int e = 0; e < sch.E; ++e)
-            if (s_rng[2 * e] < s_rng[2 * e + 1]) wmax = max(wmax, p.ex[e].tile_stride);
-        const int stage_bytes = (max(wmax, 128) + 127) & ~127;
-        s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
-        s_geom[1] = stage_bytes;
-    }
     // from here on the previous kernel's results are needed (sort tables, activations, workspace)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid <= sch.E) s_off[tid] = p.offsets[tid];
     if (tid >= 64 && tid < 64 + TOK) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0) {
+        // per-expert facts, the ring geometry (stage = the largest packed tile this CTA will see) and the tile count
+        int cum = 0, gbase = 0, wmax = 0;
+        for (int e = 0; e < sch.E; ++e) {
+            ExpertSm x;
+            x.row0 = s_off[e];
+            x.rows = min(s_off[e + 1] - x.row0, TOK);
+            x.tb = s_rng[2 * e];
+            x.te = x.rows > 0 ? s_rng[2 * e + 1] : x.tb;
+            x.bits = p.ex[e].bits; x.group = p.ex[e].group; x.has_zeros = p.ex[e].has_zeros; x.stride = p.ex[e].tile_stride;
+            x.gkb = x.group == 0 ? p.KB : x.group / 128;
+            x.cum = cum;
+            x.gbase = gbase;
+            x.pad = 0;
+            if (x.te > x.tb) {
+                cum += x.te - x.tb;
+                gbase += x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
+                wmax = max(wmax, x.stride);
+            }
+            s_ex[e] = x;
+        }
+        const int stage_bytes = (max(wmax, 128) + 127) & ~127;
+        s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
+        s_geom[1] = stage_bytes;
+        s_geom[2] = min(cum, MAX_TILES);
+    }
     __syncthreads();
     const uint32_t tmem_base = *s_tmem;
-    const int nstg = s_geom[0], stage_bytes = s_geom[1];
-    TileWalk tw;
-    tw.init(p, s_rng, s_off);
+    const int nstg = s_geom[0], stage_bytes = s_geom[1], T = s_geom[2];
+    for (int i = tid; i < T; i += DEC_THREADS) {            // the tile table, one thread per tile
+        int e = 0;
+        while (e + 1 < sch.E && s_ex[e + 1].cum <= i) ++e;
+        while (s_ex[e].te <= s_ex[e].tb) ++e;               // (experts without tiles share their successor's cum)
+        const ExpertSm x = s_ex[e];
+        const int tile = x.tb + i - x.cum, nt = tile / p.KB, kb = tile - nt * p.KB;
+        const int kb0 = max(x.tb - nt * p.KB, 0), kb1 = min(x.te - nt * p.KB, p.KB);
+        const bool last = kb + 1 == kb1;
+        int flags = (kb == kb0 ? TF_FIRST : 0) | (last ? TF_LAST : 0) | ((last || (kb + 1) % x.gkb == 0) ? TF_ENDS : 0) |
+                    ((kb0 == 0 && kb1 == p.KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0);
+        uint4 v;
+        v.x = (uint32_t)kb | ((uint32_t)nt << 16);
+        v.y = (uint32_t)flags | ((uint32_t)e << 8) | ((uint32_t)x.rows << 16) | ((uint32_t)x.row0 << 24);
+        v.z = (uint32_t)(x.gbase + tile / x.gkb - x.tb / x.gkb);
+        v.w = 0;
+        *reinterpret_cast<uint4*>(smem + L::tile_off + 16 * i) = v;
+    }
+    __syncthreads();
 
     if (warp == W_WARP) {
         // ------------------------------------------------------------------ packed-weight producer
         if (lane == 0) {
             Ring ring;
-            for (; tw.valid; tw.step(p, s_rng, s_off)) {
-                const uint32_t wbytes = (uint32_t)tw.stride;
+            for (int t = 0; t < T; ++t) {
+                const Tile ti(s_tile[t]);
+                const uint32_t wbytes = (uint32_t)s_ex[ti.e].stride;
                 if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) break;
                 const uint32_t full = bar_wfull + 8 * ring.stage;
                 mbar_expect_tx(full, wbytes);
                 bulk_load(sbase + L::ring_off + ring.stage * stage_bytes,
-                          tw.tiles + ((size_t)tw.nt * p.KB + tw.kb) * wbytes, wbytes, full);
+                          p.ex[ti.e].tiles + ((size_t)ti.nt * p.KB + ti.kb) * wbytes, wbytes, full);
                 ring.advance(nstg);
             }
         }
@@ -335,13 +347,13 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.
         const uint32_t idesc = umma_idesc(TOK);
-        int g = 0;                                   // accumulation groups started so far
         bool fresh = true;                           // the next MMA starts a group
-        for (int t = 0; tw.valid; tw.step(p, s_rng, s_off), ++t) {
-            const int a = t & (NA - 1), d = g & (ND - 1);
-            const bool ends = tw.ends();
+        for (int t = 0; t < T; ++t) {
+            const Tile ti(s_tile[t]);
+            const int a = t & (NA - 1), d = ti.g & (ND - 1);
+            const bool ends = ti.ends();
             if (!wwait(bar_afull + 8 * a, (uint32_t)(t >> 2) & 1u)) break;
-            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(g >> 2) & 1u) ^ 1u)) break;
+            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(ti.g >> 2) & 1u) ^ 1u)) break;
             tc_fence_after();
             const uint32_t xs = sbase + L::x_off + (t & (NXS - 1)) * X_STAGE;
             const uint32_t dt = tmem_base + D_COL0 + d * TOK, a0 = tmem_base + a * 64;
@@ -360,54 +372,50 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             }
             __syncwarp();
             fresh = ends;
-            if (ends) ++g;
         }
     } else if (warp < DQ_WARPS) {
         // ------------------------------------------------------------------ dequant warpgroups
         const int wg = warp >> 2, row = (warp & 3) * 32 + lane, twg = tid & 127;
         const uint32_t a_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + wg * 64;
-        Ring ring;
-        int g = 0;
-        TileWalk xw = tw;                            // runs ahead: the warpgroup's next tile, for its token rows
-        int xt = 0;
-        auto x_seek = [&](int target) {              // move xw to tile `target` (or past the end)
-            for (; xw.valid && xt < target; ++xt) xw.step(p, s_rng, s_off);
-        };
-        x_seek(wg);
-        if (xw.valid) load_token_tile(p, s_perm, sbase + L::x_off + (xt & (NXS - 1)) * X_STAGE, xw.row0, xw.rows, xw.kb, twg);
-        else asm volatile("cp.async.commit_group;" ::: "memory");
-        bool ok = true;
-        for (int t = 0; ok && tw.valid; tw.step(p, s_rng, s_off), ++t, ring.advance(nstg)) {
-            const bool ends = tw.ends();
-            if ((t & 3) == wg) {
-                // the warpgroup's previous tile is done: its A buffer and its token-tile stage (t + 4) % 8 are free
-                if (!(ok = wait_done(t - 4))) break;
-                x_seek(t + 4);
-                if (xw.valid) load_token_tile(p, s_perm, sbase + L::x_off + (xt & (NXS - 1)) * X_STAGE, xw.row0, xw.rows, xw.kb, twg);
-                else asm volatile("cp.async.commit_group;" ::: "memory");
-                if (!(ok = wwait(bar_wfull + 8 * ring.stage, ring.phase))) break;
-                tc_fence_after();
-                const unsigned char* stage = smem + L::ring_off + ring.stage * stage_bytes;
-                // zero-point of this row for the tile: the tile's own meta, the per-channel array, or 2^(bits-1)
-                float z = (float)(1 << (tw.bits - 1));
-                if (tw.has_zeros)
-                    z = tw.group == 0 ? __bfloat162float(p.ex[tw.e].zeros_pc[tw.nt * 128 + row])
-                                      : __bfloat162float(moqe_tile_zeros(stage, tw.bits, 0)[row]);
-                if (tw.bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
-                else if (tw.bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), a_taddr);
-                else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
-                // the scale of a group that ends in this tile, for the epilogue thread of the same row
-                if (ends && tw.group != 0)
-                    s_scale[(g & (SCALE_SLOTS - 1)) * 128 + row] =
-                        __half2float(moqe_tile_scales(stage, tw.bits, tw.has_zeros, 0)[row]) * (tw.bits == 8 ? W8_PRESCALE : 1.f);
-                warrive(bar_wempty + 8 * ring.stage);
-                asm volatile("cp.async.wait_group 1;" ::: "memory");      // this tile's token rows have landed
-                fence_proxy_async();
-                tmem_st_wait();
-                tc_fence_before();
-                warrive(bar_afull + 8 * (t & (NA - 1)));
+        auto x_load = [&](int t) {                   // token rows of tile t (an empty group past the end)
+            if (t < T) {
+                const Tile xi(s_tile[t]);
+                load_token_tile(p, s_perm, sbase + L::x_off + (t & (NXS - 1)) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
+            } else {
+                asm volatile("cp.async.commit_group;" ::: "memory");
             }
-            if (ends) ++g;
+        };
+        x_load(wg);
+        for (int t = wg; t < T; t += 4) {
+            const Tile ti(s_tile[t]);
+            const ExpertSm& ex = s_ex[ti.e];
+            const int stg = t % nstg;
+            const uint32_t wphase = (uint32_t)(t / nstg) & 1u;
+            // the warpgroup's previous tile is done: its A buffer and its token-tile stage (t + 4) % 8 are free
+            if (!wait_done(t - 4)) break;
+            x_load(t + 4);
+            if (!wwait(bar_wfull + 8 * stg, wphase)) break;
+            tc_fence_after();
+            const unsigned char* stage = smem + L::ring_off + stg * stage_bytes;
+            const int bits = ex.bits, group = ex.group, has_zeros = ex.has_zeros;
+            // zero-point of this row for the tile: the tile's own meta, the per-channel array, or 2^(bits-1)
+            float z = (float)(1 << (bits - 1));
+            if (has_zeros)
+                z = group == 0 ? __bfloat162float(p.ex[ti.e].zeros_pc[ti.nt * 128 + row])
+                               : __bfloat162float(moqe_tile_zeros(stage, bits, 0)[row]);
+            if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
+            else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), a_taddr);
+            else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
+            // the scale of a group that ends in this tile, for the epilogue thread of the same row
+            if (ti.ends() && group != 0)
+                s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row] =
+                    __half2float(moqe_tile_scales(stage, bits, has_zeros, 0)[row]) * (bits == 8 ? W8_PRESCALE : 1.f);
+            warrive(bar_wempty + 8 * stg);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");      // this tile's token rows have landed
+            fence_proxy_async();
+            tmem_st_wait();
+            tc_fence_before();
+            warrive(bar_afull + 8 * (t & (NA - 1)));
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp >= EP_WARP0 && warp < EP_WARP0 + 4) {
@@ -415,23 +423,26 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         const int et = tid - EP_WARP0 * 32, row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + D_COL0;
         uint32_t esync_phase = 0;
-        int g = 0, n_pending = 0;
+        int n_pending = 0;
         int pend_e[2], pend_nt[2], pend_j0[2], pend_rows[2];
         float acc[TOK];
         float pc_s = 0.f;
         bool ok = true;
-        for (; ok && tw.valid; tw.step(p, s_rng, s_off)) {
-            const int n = tw.nt * 128 + row;
-            if (tw.first()) {
+        for (int t = 0; ok && t < T; ++t) {
+            const Tile ti(s_tile[t]);
+            if (!(ti.flags & (TF_FIRST | TF_ENDS))) continue;
+            const ExpertSm& ex = s_ex[ti.e];
+            const int n = ti.nt * 128 + row, bits = ex.bits, group = ex.group;
+            if (ti.first()) {
 #pragma unroll
                 for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
-                if (tw.group == 0) pc_s = __half2float(p.ex[tw.e].scales_pc[n]) * (tw.bits == 8 ? W8_PRESCALE : 1.f);
+                if (group == 0) pc_s = __half2float(p.ex[ti.e].scales_pc[n]) * (bits == 8 ? W8_PRESCALE : 1.f);
             }
-            if (tw.ends()) {
-                const int d = g & (ND - 1);
-                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(g >> 2) & 1u))) break;
+            if (ti.ends()) {
+                const int d = ti.g & (ND - 1);
+                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(ti.g >> 2) & 1u))) break;
                 tc_fence_after();
-                const float s = tw.group == 0 ? pc_s : s_scale[(g & (SCALE_SLOTS - 1)) * 128 + row];
+                const float s = group == 0 ? pc_s : s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row];
                 uint32_t v[16];
                 tmem_ld16(lane_base + d * TOK, v);
                 tmem_ld_wait();
@@ -439,11 +450,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 for (int i = 0; i < 16; ++i) acc[i] = fmaf(s, __uint_as_float(v[i]), acc[i]);
                 tc_fence_before();
                 warrive(bar_accempty + 8 * d);
-                ++g;
             }
-            if (!tw.last()) continue;
-            const int j0 = tw.row0, rows = tw.rows;
-            if (tw.whole(p.KB)) {
+            if (!ti.last()) continue;
+            const int j0 = ti.row0, rows = ti.rows;
+            if (ti.flags & TF_WHOLE) {
                 // the whole K of this segment was ours: round and store rows at their original positions
                 if (n < p.N) {
 #pragma unroll
@@ -452,12 +462,12 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 }
             } else {
                 // partial sum: park it in this CTA's slot (0: the piece starts inside its segment, 1: at its start)
-                float* dst = p.partials + ((size_t)(blockIdx.x * 2 + (tw.kb0 != 0 ? 0 : 1)) * TOK) * 128 + row;
+                float* dst = p.partials + ((size_t)(blockIdx.x * 2 + ((ti.flags & TF_KB0NZ) ? 0 : 1)) * TOK) * 128 + row;
 #pragma unroll
                 for (int m = 0; m < TOK; ++m)
                     if (m < rows) dst[m * 128] = acc[m];
                 if (n_pending < 2) {
-                    pend_e[n_pending] = tw.e; pend_nt[n_pending] = tw.nt; pend_j0[n_pending] = j0; pend_rows[n_pending] = rows;
+                    pend_e[n_pending] = ti.e; pend_nt[n_pending] = ti.nt; pend_j0[n_pending] = j0; pend_rows[n_pending] = rows;
                     ++n_pending;
                 }
             }
@@ -548,11 +558,40 @@ int g_dec_tile_cost[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
 
 void decode_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost >= 0) g_dec_tile_cost[bits] = cost; }
 
+namespace {
+// the work split of one call: costs, grid, and whether every CTA's tiles fit its tile table
+bool decode_plan(const moqe_expert* const* ex, int E, DecSched& s, int& grid) {
+    const int KB = ex[0]->Kp / 128, ntiles = ex[0]->Np / 128;
+    s.E = E;
+    s.KB = KB;
+    s.TT = ntiles * KB;
+    s.C = 0;
+    int wmax = 1, wmin = 1 << 30;
+    for (int e = 0; e < E; ++e) {
+        const int cost = g_dec_tile_cost[ex[e]->bits];
+        s.w[e] = cost > 0 ? cost : ex[e]->dev().tile_stride / 256;
+        s.C += (long long)s.TT * s.w[e];
+        wmax = s.w[e] > wmax ? s.w[e] : wmax;
+        wmin = s.w[e] < wmin ? s.w[e] : wmin;
+    }
+    // every CTA's cost share must be at least one tile of the dearest kind, so that every CTA between the owners of
+    // a segment's first and last tile really owns a tile of it (the reduction counts them)
+    grid = dec_sm_count();
+    if (grid > DEC_MAX_GRID) grid = DEC_MAX_GRID;
+    const long long work_items = s.C / wmax;
+    if (work_items < grid) grid = work_items < 1 ? 1 : (int)work_items;
+    s.G = grid;
+    return s.C / grid / wmin + E + 2 <= MAX_TILES;
+}
+}  // namespace
+
 bool decode_supported(int M, const moqe_expert* const* ex, int E) {
     if (M > DECODE_MAX_ROWS) return false;
     for (int e = 0; e < E; ++e)
         if (ex[e]->group != 0 && (ex[e]->group < 128 || ex[e]->group % 128 != 0)) return false;
-    return true;
+    DecSched s;
+    int grid;
+    return decode_plan(ex, E, s, grid);
 }
 
 size_t decode_zero_bytes(int M, int Np) {
@@ -576,25 +615,9 @@ moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_e
     p.KB = ex[0]->Kp / 128;
     p.ntiles = ex[0]->Np / 128;
     DecSched& s = p.sched;
-    s.E = E;
-    s.KB = p.KB;
-    s.TT = p.ntiles * p.KB;
-    s.C = 0;
-    int wmax = 1;
-    for (int e = 0; e < E; ++e) {
-        p.ex[e] = ex[e]->dev();
-        const int cost = g_dec_tile_cost[ex[e]->bits];
-        s.w[e] = cost > 0 ? cost : p.ex[e].tile_stride / 256;
-        s.C += (long long)s.TT * s.w[e];
-        wmax = s.w[e] > wmax ? s.w[e] : wmax;
-    }
-    // every CTA's cost share must be at least one tile of the dearest kind, so that every CTA between the owners of
-    // a segment's first and last tile really owns a tile of it (the reduction counts them)
-    int grid = dec_sm_count();
-    if (grid > DEC_MAX_GRID) grid = DEC_MAX_GRID;
-    const long long work_items = s.C / wmax;
-    if (work_items < grid) grid = work_items < 1 ? 1 : (int)work_items;
-    s.G = grid;
+    int grid = 1;
+    if (!decode_plan(ex, E, s, grid)) return MOQE_ERR_UNSUPPORTED;
+    for (int e = 0; e < E; ++e) p.ex[e] = ex[e]->dev();
     if (!ws || ws_bytes < decode_workspace_bytes(M, ex[0]->Np, E)) return MOQE_ERR_WORKSPACE;
     p.counters = (uint32_t*)ws;
     p.partials = (float*)((char*)ws + (decode_zero_bytes(M, ex[0]->Np) + 255) / 256 * 256);
