@@ -51,11 +51,11 @@ namespace {
 constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
 constexpr int DQ_WARPS = 16, EP_WARP0 = 16, MMA_WARP = 20, W_WARP = 21;
 constexpr int DEC_THREADS = 22 * 32;
-constexpr int RING_BYTES = 160 * 1024;                  // packed-weight ring
+constexpr int RING_BYTES = 152 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
-constexpr int NA = 4;                                   // A-operand buffers in TMEM (64 columns each), one per warpgroup
+constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
 constexpr int ND = 4;                                   // accumulator buffers (TOK columns each)
-constexpr int NXS = 8;                                  // token-tile stages
+constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
 constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
 constexpr int SCALE_SLOTS = 16;                         // group scales handed from the dequant to the epilogue threads
@@ -348,14 +348,16 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.
         const uint32_t idesc = umma_idesc(TOK);
         bool fresh = true;                           // the next MMA starts a group
+        int a = 0, xst = 0;
+        uint32_t aphase = 0;
         for (int t = 0; t < T; ++t) {
             const Tile ti(s_tile[t]);
-            const int a = t & (NA - 1), d = ti.g & (ND - 1);
+            const int d = ti.g & (ND - 1);
             const bool ends = ti.ends();
-            if (!wwait(bar_afull + 8 * a, (uint32_t)(t >> 2) & 1u)) break;
+            if (!wwait(bar_afull + 8 * a, aphase)) break;
             if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(ti.g >> 2) & 1u) ^ 1u)) break;
             tc_fence_after();
-            const uint32_t xs = sbase + L::x_off + (t & (NXS - 1)) * X_STAGE;
+            const uint32_t xs = sbase + L::x_off + xst * X_STAGE;
             const uint32_t dt = tmem_base + D_COL0 + d * TOK, a0 = tmem_base + a * 64;
             const uint64_t b0 = umma_desc_sw128(xs), b1 = umma_desc_sw128(xs + TOK * 128);
             if (elect_one()) {
@@ -372,27 +374,29 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             }
             __syncwarp();
             fresh = ends;
+            if (++a == NA) { a = 0; aphase ^= 1u; }
+            if (++xst == NXS) xst = 0;
         }
     } else if (warp < DQ_WARPS) {
         // ------------------------------------------------------------------ dequant warpgroups
         const int wg = warp >> 2, row = (warp & 3) * 32 + lane, twg = tid & 127;
-        const uint32_t a_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + wg * 64;
+        const uint32_t lane_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         auto x_load = [&](int t) {                   // token rows of tile t (an empty group past the end)
             if (t < T) {
                 const Tile xi(s_tile[t]);
-                load_token_tile(p, s_perm, sbase + L::x_off + (t & (NXS - 1)) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
+                load_token_tile(p, s_perm, sbase + L::x_off + (t % NXS) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
             } else {
                 asm volatile("cp.async.commit_group;" ::: "memory");
             }
         };
         x_load(wg);
+        int stg = wg % nstg, a = wg;                 // ring stage and A buffer of tile t, kept incrementally
+        uint32_t wphase = (uint32_t)(wg / nstg) & 1u;
         for (int t = wg; t < T; t += 4) {
             const Tile ti(s_tile[t]);
             const ExpertSm& ex = s_ex[ti.e];
-            const int stg = t % nstg;
-            const uint32_t wphase = (uint32_t)(t / nstg) & 1u;
-            // the warpgroup's previous tile is done: its A buffer and its token-tile stage (t + 4) % 8 are free
-            if (!wait_done(t - 4)) break;
+            // tile t - 6 is done: A buffer t % 6 and token-tile stage (t + 4) % 10 are free
+            if (!wait_done(t - NA)) break;
             x_load(t + 4);
             if (!wwait(bar_wfull + 8 * stg, wphase)) break;
             tc_fence_after();
@@ -403,9 +407,9 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             if (has_zeros)
                 z = group == 0 ? __bfloat162float(p.ex[ti.e].zeros_pc[ti.nt * 128 + row])
                                : __bfloat162float(moqe_tile_zeros(stage, bits, 0)[row]);
-            if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
-            else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), a_taddr);
-            else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), a_taddr);
+            if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
+            else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), lane_taddr + a * 64);
+            else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
             // the scale of a group that ends in this tile, for the epilogue thread of the same row
             if (ti.ends() && group != 0)
                 s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row] =
@@ -415,7 +419,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             fence_proxy_async();
             tmem_st_wait();
             tc_fence_before();
-            warrive(bar_afull + 8 * (t & (NA - 1)));
+            warrive(bar_afull + 8 * a);
+            stg += 4;
+            while (stg >= nstg) { stg -= nstg; wphase ^= 1u; }
+            a = a + 4 >= NA ? a + 4 - NA : a + 4;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp >= EP_WARP0 && warp < EP_WARP0 + 4) {
