@@ -54,7 +54,7 @@ WsLayout ws_layout(int M, int Np, int K, int E) {
 constexpr int AUTO_STREAM_MAX_ROWS = 128;
 constexpr int LAST_PATH = 5;
 
-bool g_auto_decode = false;   // whether the automatic choice takes the tcgen05 decode kernel where it applies
+bool g_auto_decode = true;   // whether the automatic choice takes the tcgen05 decode kernel where it applies
 
 // 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = tcgen05 decode kernel
 int pick_kernel(int path, int M, const moqe_expert* const* ex, int E) {
