@@ -29,8 +29,11 @@
 // Work split ("stream-K" over packed tiles): all tiles of the call form one sequence
 // [expert][channel tile nt][k-block kb]; tile (e, nt, kb) costs w[e].  CTA c of G owns the tiles
 // whose start cost lies in [c*C/G, (c+1)*C/G) -- equal work to within one tile, at most two partial
-// pieces per CTA.  Partial sums go to the workspace; the CTA that announces last for an (expert, nt)
-// segment adds them in CTA order (deterministic) and stores the rows.
+// pieces per CTA: a first one that starts inside its (expert, nt) segment and a last one that stops
+// inside its segment.  A first piece is parked in the workspace and flagged as soon as it is done,
+// early in the kernel; the CTA that holds the head of a segment -- its last piece -- keeps that sum in
+// registers, adds the parked pieces of the following CTAs in CTA order (deterministic) and stores
+// the rows.  All CTAs are resident (grid <= SM count), and the flag wait is bounded like every other.
 //
 // Takes experts that are per-channel or have groups of 128 k or more, and batches of at most 16
 // rows; the caller routes everything else to the other kernels.
@@ -94,8 +97,8 @@ struct DecParams {
     uint16_t* Y;
     const int32_t* perm;
     const int32_t* offsets;
-    float* partials;        // [CTA][slot 0/1][TOK][128]
-    uint32_t* counters;     // [expert][ntiles], zero on entry, left zero
+    float* partials;        // [CTA][TOK][128]: the partial sum of a CTA's first piece
+    uint32_t* flags;        // [CTA]: that partial sum is parked; zero on entry, left zero
     int* status;
     int M, N, K, KB, ntiles;
 };
@@ -120,6 +123,7 @@ __device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long 
 // The CTA's tiles, in order, as a table in shared memory (one 16-byte entry per tile), built once by the whole CTA
 // after the routing offsets are known: every role then reads its tile with one load instead of walking pieces.
 //   x = kb | nt << 16        y = flags | e << 8 | rows << 16 | row0 << 24        z = accumulation-group index g
+//   w = the last CTA that owns a tile of this tile's (expert, nt) segment
 // An accumulation group (one accumulator buffer handed to the epilogue) is: the whole piece for per-channel
 // experts; for groups of 128 k or more, the k-blocks of one quantization group inside the piece (the scale is
 // constant over the group, so a piece may cut it).
@@ -136,10 +140,10 @@ struct ExpertSm {            // per-expert facts of this CTA, in shared memory
 };
 
 struct Tile {
-    int kb, nt, flags, e, rows, row0, g;
+    int kb, nt, flags, e, rows, row0, g, c_last;
     __device__ __forceinline__ explicit Tile(const uint4& v)
         : kb((int)(v.x & 0xFFFFu)), nt((int)(v.x >> 16)), flags((int)(v.y & 0xFFu)), e((int)((v.y >> 8) & 0xFFu)),
-          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z) {}
+          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z), c_last((int)v.w) {}
     __device__ __forceinline__ bool first() const { return flags & TF_FIRST; }
     __device__ __forceinline__ bool last() const { return flags & TF_LAST; }
     __device__ __forceinline__ bool ends() const { return flags & TF_ENDS; }
@@ -323,7 +327,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         v.x = (uint32_t)kb | ((uint32_t)nt << 16);
         v.y = (uint32_t)flags | ((uint32_t)e << 8) | ((uint32_t)x.rows << 16) | ((uint32_t)x.row0 << 24);
         v.z = (uint32_t)(x.gbase + tile / x.gkb - x.tb / x.gkb);
-        v.w = 0;
+        // owner of the segment's last tile (needed where the head of a split segment ends)
+        v.w = (last && kb0 == 0 && kb1 != p.KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * p.KB + p.KB - 1) : 0u;
         *reinterpret_cast<uint4*>(smem + L::tile_off + 16 * i) = v;
     }
     __syncthreads();
@@ -430,14 +435,12 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         const int et = tid - EP_WARP0 * 32, row = (warp & 3) * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + D_COL0;
         uint32_t esync_phase = 0;
-        int n_pending = 0;
-        int pend_e[2], pend_nt[2], pend_j0[2], pend_rows[2];
-        float acc[TOK];
+        float acc[TOK], oth[TOK];
         float pc_s = 0.f;
         bool ok = true;
         for (int t = 0; ok && t < T; ++t) {
             const Tile ti(s_tile[t]);
-            if (!(ti.flags & (TF_FIRST | TF_ENDS))) continue;
+            if (!(ti.flags & (TF_FIRST | TF_ENDS | TF_LAST))) continue;
             const ExpertSm& ex = s_ex[ti.e];
             const int n = ti.nt * 128 + row, bits = ex.bits, group = ex.group;
             if (ti.first()) {
@@ -445,6 +448,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
                 if (group == 0) pc_s = __half2float(p.ex[ti.e].scales_pc[n]) * (bits == 8 ? W8_PRESCALE : 1.f);
             }
+            const bool head_last = ti.last() && !(ti.flags & (TF_WHOLE | TF_KB0NZ));
+            const int n_others = ti.c_last - (int)blockIdx.x;
             if (ti.ends()) {
                 const int d = ti.g & (ND - 1);
                 if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(ti.g >> 2) & 1u))) break;
@@ -467,63 +472,62 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                     for (int m = 0; m < TOK; ++m)
                         if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
                 }
-            } else {
-                // partial sum: park it in this CTA's slot (0: the piece starts inside its segment, 1: at its start)
-                float* dst = p.partials + ((size_t)(blockIdx.x * 2 + ((ti.flags & TF_KB0NZ) ? 0 : 1)) * TOK) * 128 + row;
+            } else if (ti.flags & TF_KB0NZ) {
+                // A piece that starts inside its segment -- always a CTA's FIRST piece, so it is ready early in the
+                // kernel: park the partial sum and raise this CTA's flag.  Nobody waits here.
+                float* dst = p.partials + (size_t)blockIdx.x * TOK * 128 + row;
 #pragma unroll
                 for (int m = 0; m < TOK; ++m)
                     if (m < rows) dst[m * 128] = acc[m];
-                if (n_pending < 2) {
-                    pend_e[n_pending] = ti.e; pend_nt[n_pending] = ti.nt; pend_j0[n_pending] = j0; pend_rows[n_pending] = rows;
-                    ++n_pending;
+                __threadfence();
+                mbar_arrive(bar_esync);
+                if (!(ok = wwait(bar_esync, esync_phase))) break;
+                esync_phase ^= 1u;
+                if (et == 0) {
+                    __threadfence();
+                    atomicExch(p.flags + blockIdx.x, 1u);
                 }
-            }
-        }
-        // ---- announce the parked pieces; whoever announces last for a segment adds its pieces up in CTA order
-        if (ok && n_pending > 0) {
-            __threadfence();
-            mbar_arrive(bar_esync);
-            ok = wwait(bar_esync, esync_phase);
-            esync_phase ^= 1u;
-            if (ok && et == 0) {
-                for (int i = 0; i < n_pending; ++i) {
-                    const long long base = dsched_base(sch, pend_e[i]);
-                    const int t0 = pend_nt[i] * p.KB;
-                    const int c_first = dsched_owner(sch, pend_e[i], base, t0);
-                    const int c_last = dsched_owner(sch, pend_e[i], base, t0 + p.KB - 1);
-                    unsigned* cnt = p.counters + (size_t)pend_e[i] * p.ntiles + pend_nt[i];
-                    const unsigned old = atomicAdd(cnt, 1u);
-                    const int last = old == (unsigned)(c_last - c_first) ? 1 : 0;
-                    if (last) *cnt = 0u;                               // leave the counters clear for the next call
-                    s_red[4 * i] = last; s_red[4 * i + 1] = c_first; s_red[4 * i + 2] = c_last - c_first + 1;
+            } else {
+                // The last tile of the head of a segment whose tail belongs to the following CTAs -- always a CTA's
+                // LAST piece, while the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as
+                // its first piece).  Fetch their sum in CTA order (deterministic) and add the own one (registers).
+                for (int i = et; i < n_others; i += 128) {
+                    volatile unsigned* f = p.flags + blockIdx.x + 1 + i;
+                    unsigned long long t_start = 0;
+                    for (unsigned it = 1; *f == 0u; ++it) {
+                        if ((it & 63u) == 0) {
+                            if (*s_abort) break;
+                            const unsigned long long now = global_ns();
+                            if (t_start == 0) t_start = now;
+                            else if (now - t_start > WAIT_LIMIT_NS) { *s_abort = 1; latch_status(p.status, (int)MOQE_ERR_TIMEOUT); break; }
+                        }
+                    }
                 }
                 __threadfence();
-            }
-            if (ok) {
                 mbar_arrive(bar_esync);
-                ok = wwait(bar_esync, esync_phase);
+                if (!(ok = wwait(bar_esync, esync_phase))) break;
                 esync_phase ^= 1u;
-            }
-            for (int i = 0; ok && i < n_pending; ++i) {
-                if (!s_red[4 * i]) continue;
-                const int c_first = s_red[4 * i + 1], n_contrib = s_red[4 * i + 2];
-                const int e = pend_e[i], nt = pend_nt[i], rows = pend_rows[i], n = nt * 128 + row;
-                const long long base = dsched_base(sch, e);
-                float sum[TOK];
+                if (*s_abort) { ok = false; break; }
 #pragma unroll
-                for (int m = 0; m < TOK; ++m) sum[m] = 0.f;
-                for (int ci = 0; ci < n_contrib; ++ci) {
-                    const int cc = c_first + ci;
-                    const int slot = dsched_tbegin(sch, cc, e, base) <= nt * p.KB ? 1 : 0;
-                    const float* src = p.partials + ((size_t)(cc * 2 + slot) * TOK) * 128 + row;
+                for (int m = 0; m < TOK; ++m) oth[m] = 0.f;
+                for (int c0 = 0; c0 < n_others; c0 += 2) {             // two contributors' loads in flight at a time
+                    float part[2][TOK];
 #pragma unroll
-                    for (int m = 0; m < TOK; ++m)
-                        if (m < rows) sum[m] += __ldcg(src + m * 128);
+                    for (int u = 0; u < 2; ++u) {
+                        const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0 + u) * TOK * 128 + row;
+#pragma unroll
+                        for (int m = 0; m < TOK; ++m) part[u][m] = (c0 + u < n_others && m < ti.rows) ? __ldcg(src + m * 128) : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+#pragma unroll
+                        for (int m = 0; m < TOK; ++m) oth[m] += part[u][m];
                 }
+                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
                 if (n < p.N) {
 #pragma unroll
                     for (int m = 0; m < TOK; ++m)
-                        if (m < rows) p.Y[(size_t)s_perm[pend_j0[i] + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(sum[m]));
+                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m] + oth[m]));
                 }
             }
         }
@@ -604,14 +608,15 @@ bool decode_supported(int M, const moqe_expert* const* ex, int E) {
 
 size_t decode_zero_bytes(int M, int Np) {
     if (M > DECODE_MAX_ROWS) return 0;
-    return (size_t)MOQE_MAX_EXPERTS * (Np / 128) * sizeof(uint32_t);
+    (void)Np;
+    return (size_t)DEC_MAX_GRID * sizeof(uint32_t);
 }
 
 size_t decode_workspace_bytes(int M, int Np, int E) {
     (void)E;
     if (M > DECODE_MAX_ROWS) return 0;
     const size_t counters = (decode_zero_bytes(M, Np) + 255) / 256 * 256;
-    const size_t partials = (size_t)DEC_MAX_GRID * 2 * TOK * 128 * sizeof(float);
+    const size_t partials = (size_t)DEC_MAX_GRID * TOK * 128 * sizeof(float);
     return counters + partials;
 }
 
@@ -627,7 +632,7 @@ moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_e
     if (!decode_plan(ex, E, s, grid)) return MOQE_ERR_UNSUPPORTED;
     for (int e = 0; e < E; ++e) p.ex[e] = ex[e]->dev();
     if (!ws || ws_bytes < decode_workspace_bytes(M, ex[0]->Np, E)) return MOQE_ERR_WORKSPACE;
-    p.counters = (uint32_t*)ws;
+    p.flags = (uint32_t*)ws;
     p.partials = (float*)((char*)ws + (decode_zero_bytes(M, ex[0]->Np) + 255) / 256 * 256);
     p.X = (const uint16_t*)X;
     p.Y = (uint16_t*)Y;
