@@ -57,7 +57,7 @@ constexpr int DEC_THREADS = 22 * 32;
 constexpr int RING_BYTES = 152 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
-constexpr int ND = 4;                                   // accumulator buffers (TOK columns each)
+constexpr int ND = 8;                                   // accumulator buffers (TOK columns each)
 constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
 constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             const int d = ti.g & (ND - 1);
             const bool ends = ti.ends();
             if (!wwait(bar_afull + 8 * a, aphase)) break;
-            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(ti.g >> 2) & 1u) ^ 1u)) break;
+            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(ti.g >> 3) & 1u) ^ 1u)) break;
             tc_fence_after();
             const uint32_t xs = sbase + L::x_off + xst * X_STAGE;
             const uint32_t dt = tmem_base + D_COL0 + d * TOK, a0 = tmem_base + a * 64;
@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             const int n_others = ti.c_last - (int)blockIdx.x;
             if (ti.ends()) {
                 const int d = ti.g & (ND - 1);
-                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(ti.g >> 2) & 1u))) break;
+                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(ti.g >> 3) & 1u))) break;
                 tc_fence_after();
                 const float s = group == 0 ? pc_s : s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row];
                 uint32_t v[16];
