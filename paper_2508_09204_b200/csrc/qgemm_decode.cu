@@ -189,7 +189,7 @@ template <int BITS>
 __device__ __forceinline__ void dequant_tile(const unsigned char* stage, int row, uint32_t zc, uint32_t a_taddr) {
     const unsigned char* blob = stage + (row >> 4) * moqe_blob_bytes(BITS);
     const int half = (row >> 3) & 1, r = row & 7;
-#pragma unroll
+#pragma unroll 1
     for (int q = 0; q < 4; ++q) {
         uint32_t w[PieceWords<BITS>::n];
         load_piece_smem<BITS>(blob, half, q * 8 + (r ^ (2 * q)), w);
