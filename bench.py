@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # proportion with the bytes streamed, so the ratio is applied to the average launch of the block.
 # None = no capture of the current kernel.
 TRAFFIC_RATIO = {
-    "llama7b_decode": 32.755 / 32.513,      # 32.73 MB read + 0.02 MB written vs 32.51 MB algorithmic
+    "llama7b_decode": 32.703 / 32.513,      # 32.70 MB read + 0 written (outputs stay in L2) vs 32.51 MB algorithmic
     "llama7b_prefill": 267.12 / 300.95,     # 158.4 MB read + 108.7 MB written (part of Y still in L2) vs 300.9 MB
 }
 
@@ -411,7 +411,8 @@ def main():
                     "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     "frac_of_nominal_8000": achieved / 8000.0}
     roofline.update({"peak_source": peaks["source"],
-                     "kernel": ("qgemm_tc_kernel" if tensor_time > hbm_time else "qgemm_stream_kernel") +
+                     "kernel": ("qgemm_tc_kernel" if tensor_time > hbm_time else
+                                ("qgemm_decode_kernel" if max(L["M"] for L in layers) <= 16 else "qgemm_stream_kernel")) +
                                f": average of the {n_launch} routed-GEMM launches of one block",
                      "launches_per_step": n_launch, "algorithmic_bytes_per_launch": sum(alg_bytes) / n_launch,
                      "traffic_unit": "bytes per launch",
