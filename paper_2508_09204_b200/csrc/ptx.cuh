@@ -37,9 +37,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
-// try_wait parks the thread in hardware until the phase completes or a short, system-defined time has passed,
-// so a waiting warp does not compete for issue slots the way a test_wait spin loop does.
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+// try_wait with a suspend-time hint parks the thread in hardware until the phase completes or the hint (1 ms)
+// has passed, so a waiting warp does not compete for issue slots; without the hint the wait returns after a short
+// system-defined time and a waiting warp spins, which costs the working warps of the same scheduler their slots.
+constexpr uint32_t TRY_WAIT_HINT_NS = 1000000u;
+// (kernels whose waits are short and on the critical path use the plain form: waking up from the hinted sleep is
+// slower than coming round a short spin)
+__device__ __forceinline__ bool mbar_try_short(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -48,15 +52,42 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(TRY_WAIT_HINT_NS) : "memory");
+    return ok != 0;
+}
 
-// Bounded wait.  Returns false if the CTA is aborting (someone's wait ran out).  The clock (%globaltimer is
-// slow to read) and the abort flag are only consulted every 256 failed tries, so the common path -- the phase
-// completes within a few tries -- costs nothing but the try_wait itself.
+// Bounded wait.  Returns false if the CTA is aborting (someone's wait ran out).  A failed try has already slept
+// for up to the hint, so the clock and the abort flag are consulted after every few of them.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
     if (mbar_try(bar, parity)) return true;
     unsigned long long t0 = 0;
     for (unsigned it = 1;; ++it) {
         if (mbar_try(bar, parity)) return true;
+        if ((it & 3u) == 0) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                latch_status(status, (int)MOQE_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// the same bounded wait on the plain try_wait: the clock is consulted every 256 failed tries
+__device__ __forceinline__ bool mbar_wait_short(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try_short(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (unsigned it = 1;; ++it) {
+        if (mbar_try_short(bar, parity)) return true;
         if ((it & 255u) == 0) {
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();

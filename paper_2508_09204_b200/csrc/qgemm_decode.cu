@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     const DecSched& sch = p.sched;
     // warp-uniform bounded wait: every lane polls, the warp agrees on the verdict
     auto wwait = [&](uint32_t bar, uint32_t parity) -> bool {
-        return __all_sync(0xffffffffu, mbar_wait(bar, parity, s_abort, p.status));
+        return __all_sync(0xffffffffu, mbar_wait_short(bar, parity, s_abort, p.status));
     };
     // one arrival per warp, after all its lanes are done with what the barrier hands over
     auto warrive = [&](uint32_t bar) {
