@@ -183,8 +183,9 @@ MOQE_API moqe_status moqe_permute_static(const void* X_bf16, const int32_t* row_
  * invalid id are written as zeros).  M == 0 is valid.  workspace:
  * moqe_routed_qgemm_workspace(M, N, K, E) bytes, contents irrelevant on entry;
  * calls that share a workspace must not overlap on the device.
- * Small batches stream each touched expert's packed weights once (split-K
- * dequant-MMA kernel); large batches run the persistent tcgen05 grouped GEMM.
+ * Decode batches (at most 16 rows, experts per-channel or with groups of 128 k or more) stream each touched
+ * expert's packed weights once through the tcgen05 decode kernel (TMEM-operand MMAs, stream-K split); other
+ * small batches take the split-K mma.sync streaming kernel; large batches run the persistent tcgen05 grouped GEMM.
  * ------------------------------------------------------------------------- */
 MOQE_API size_t moqe_routed_qgemm_workspace(int M, int N, int K, int E);
 MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_ids, int M,
@@ -193,7 +194,8 @@ MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_id
 
 /* Same, with the kernel chosen by the caller (testing / measurement):
  * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM (automatic
- * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles. */
+ * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles, 5 = tcgen05 decode kernel
+ * (MOQE_ERR_UNSUPPORTED if the batch has more than 16 rows or an expert has groups narrower than 128 k). */
 MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
                                    const moqe_expert* const* h_experts, int E, void* Y_bf16,
                                    void* workspace, size_t workspace_bytes, void* stream, int path);
@@ -222,6 +224,9 @@ MOQE_API const char* moqe_status_str(moqe_status s);
  *   "stream_tile_cost_w8" / "_w4" / "_w3" : relative cost of one packed 128x128 tile of
  *                            that bit-width in the streaming kernel's work split
  *                            (defaults 8 / 8 / 8).
+ *   "decode_tile_cost_w8" / "_w4" / "_w3" : the same for the tcgen05 decode kernel
+ *                            (defaults 8 / 10 / 11; 0 = the tile's bytes).
+ *   "auto_decode"          : whether path 0 takes the decode kernel where it applies (default 1).
  * Unknown key: MOQE_ERR_UNSUPPORTED. */
 MOQE_API moqe_status moqe_tune(const char* key, int value);
 
