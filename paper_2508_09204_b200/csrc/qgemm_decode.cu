@@ -54,14 +54,13 @@ namespace {
 constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
 constexpr int DQ_WARPS = 16, EP_WARP0 = 16, MMA_WARP = 20, W_WARP = 21;
 constexpr int DEC_THREADS = 22 * 32;
-constexpr int RING_BYTES = 152 * 1024;                  // packed-weight ring
+constexpr int RING_BYTES = 150 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
-constexpr int ND = 8;                                   // accumulator buffers (TOK columns each)
+constexpr int ND = 8;                                   // accumulator buffers (TOK columns each), group g -> g % 8
 constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
 constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
-constexpr int SCALE_SLOTS = 16;                         // group scales handed from the dequant to the epilogue threads
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL0 = NA * 64;
 constexpr int MAX_TILES = 512;                          // tiles one CTA can take (its tile table)
@@ -69,18 +68,19 @@ constexpr int MAX_TILES = 512;                          // tiles one CTA can tak
 struct DecSmem {
     static constexpr int ring_off = 0;
     static constexpr int x_off = RING_BYTES;
-    static constexpr int scale_off = x_off + NXS * X_STAGE;
-    static constexpr int bar_off = scale_off + SCALE_SLOTS * 512;
-    // wfull[16] wempty[16] afull[NA] done[8] accfull[ND] accempty[ND] esync
-    static constexpr int n_bars = 2 * MAX_STAGES + NA + DONE_RING + 2 * ND + 1;
+    static constexpr int out_off = x_off + NXS * X_STAGE;             // float[TOK][128]: a piece's sum, warpgroup by warpgroup
+    static constexpr int bar_off = out_off + TOK * 512;
+    // wfull[16] wempty[16] afull[NA] done[8] turn[4] flush_free esync
+    static constexpr int n_bars = 2 * MAX_STAGES + NA + DONE_RING + 4 + 1 + 1;
     static constexpr int misc_off = bar_off + n_bars * 8;              // tmem address, abort flag, ring geometry
     static constexpr int off_off = misc_off + 32;
     static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;   // perm of the batch's rows
     static constexpr int rng_off = perm_off + TOK * 4;
     static constexpr int red_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // reduction verdicts
     static constexpr int ex_off = red_off + 32;                        // ExpertSm[MOQE_MAX_EXPERTS]
-    static constexpr int tile_off = ex_off + MOQE_MAX_EXPERTS * 48;    // uint4[MAX_TILES]
-    static constexpr int total = tile_off + MAX_TILES * 16;
+    static constexpr int tile_off = (ex_off + MOQE_MAX_EXPERTS * 48 + 15) & ~15;   // uint4[MAX_TILES]
+    static constexpr int piece_off = tile_off + MAX_TILES * 16;        // int[MAX_TILES]: last tile of each piece
+    static constexpr int total = piece_off + MAX_TILES * 4;
     static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
 };
 
@@ -123,11 +123,13 @@ __device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long 
 // The CTA's tiles, in order, as a table in shared memory (one 16-byte entry per tile), built once by the whole CTA
 // after the routing offsets are known: every role then reads its tile with one load instead of walking pieces.
 //   x = kb | nt << 16        y = flags | e << 8 | rows << 16 | row0 << 24        z = accumulation-group index g
-//   w = the last CTA that owns a tile of this tile's (expert, nt) segment
+//   w = piece index | (the last CTA that owns a tile of this tile's (expert, nt) segment) << 16
+// flags: first / last tile of its piece, ends / starts an accumulation group, piece = whole segment, piece starts
+// inside its segment
 // An accumulation group (one accumulator buffer handed to the epilogue) is: the whole piece for per-channel
 // experts; for groups of 128 k or more, the k-blocks of one quantization group inside the piece (the scale is
 // constant over the group, so a piece may cut it).
-constexpr int TF_FIRST = 1, TF_LAST = 2, TF_ENDS = 4, TF_WHOLE = 8, TF_KB0NZ = 16;
+constexpr int TF_FIRST = 1, TF_LAST = 2, TF_ENDS = 4, TF_WHOLE = 8, TF_KB0NZ = 16, TF_GSTART = 32;
 
 struct ExpertSm {            // per-expert facts of this CTA, in shared memory
     int tb, te;              // the CTA's tile range inside the expert ([nt][kb] order); empty if the expert has no rows
@@ -136,14 +138,14 @@ struct ExpertSm {            // per-expert facts of this CTA, in shared memory
     int gkb;                 // k-blocks per accumulation group (KB for per-channel experts)
     int row0, rows;
     int bits, group, has_zeros, stride;
-    int pad;
+    int pbase;               // pieces of earlier experts
 };
 
 struct Tile {
-    int kb, nt, flags, e, rows, row0, g, c_last;
+    int kb, nt, flags, e, rows, row0, g, piece, c_last;
     __device__ __forceinline__ explicit Tile(const uint4& v)
         : kb((int)(v.x & 0xFFFFu)), nt((int)(v.x >> 16)), flags((int)(v.y & 0xFFu)), e((int)((v.y >> 8) & 0xFFu)),
-          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z), c_last((int)v.w) {}
+          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z), piece((int)(v.w & 0xFFFFu)), c_last((int)(v.w >> 16)) {}
     __device__ __forceinline__ bool first() const { return flags & TF_FIRST; }
     __device__ __forceinline__ bool last() const { return flags & TF_LAST; }
     __device__ __forceinline__ bool ends() const { return flags & TF_ENDS; }
@@ -232,8 +234,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + L::bar_off;
     const uint32_t bar_wfull = bar0, bar_wempty = bar0 + 8 * MAX_STAGES, bar_afull = bar_wempty + 8 * MAX_STAGES;
-    const uint32_t bar_done = bar_afull + 8 * NA, bar_accfull = bar_done + 8 * DONE_RING;
-    const uint32_t bar_accempty = bar_accfull + 8 * ND, bar_esync = bar_accempty + 8 * ND;
+    const uint32_t bar_done = bar_afull + 8 * NA, bar_turn = bar_done + 8 * DONE_RING;
+    const uint32_t bar_flushfree = bar_turn + 8 * 4, bar_esync = bar_flushfree + 8;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::misc_off);
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
     volatile int* s_geom = reinterpret_cast<volatile int*>(smem + L::misc_off + 8);    // {stages, stage bytes, tiles}
@@ -243,7 +245,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     volatile int* s_red = reinterpret_cast<volatile int*>(smem + L::red_off);
     ExpertSm* s_ex = reinterpret_cast<ExpertSm*>(smem + L::ex_off);
     const uint4* s_tile = reinterpret_cast<const uint4*>(smem + L::tile_off);
-    float* s_scale = reinterpret_cast<float*>(smem + L::scale_off);
+    float* s_out = reinterpret_cast<float*>(smem + L::out_off);
+    volatile int* s_piece = reinterpret_cast<volatile int*>(smem + L::piece_off);
     const DecSched& sch = p.sched;
     // warp-uniform bounded wait: every lane polls, the warp agrees on the verdict
     auto wwait = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -264,7 +267,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         for (int i = 0; i < MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, 4); }
         for (int i = 0; i < NA; ++i) mbar_init(bar_afull + 8 * i, 4);
         for (int i = 0; i < DONE_RING; ++i) mbar_init(bar_done + 8 * i, 1);
-        for (int i = 0; i < ND; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accempty + 8 * i, 4); }
+        for (int i = 0; i < 4; ++i) mbar_init(bar_turn + 8 * i, 4);
+        mbar_init(bar_flushfree, 4);
         mbar_init(bar_esync, 128);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -286,7 +290,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     tc_fence_after();
     if (tid == 0) {
         // per-expert facts, the ring geometry (stage = the largest packed tile this CTA will see) and the tile count
-        int cum = 0, gbase = 0, wmax = 0;
+        int cum = 0, gbase = 0, wmax = 0, pbase = 0;
         for (int e = 0; e < sch.E; ++e) {
             ExpertSm x;
             x.row0 = s_off[e];
@@ -297,10 +301,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             x.gkb = x.group == 0 ? p.KB : x.group / 128;
             x.cum = cum;
             x.gbase = gbase;
-            x.pad = 0;
+            x.pbase = pbase;
             if (x.te > x.tb) {
                 cum += x.te - x.tb;
                 gbase += x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
+                pbase += (x.te - 1) / p.KB - x.tb / p.KB + 1;
                 wmax = max(wmax, x.stride);
             }
             s_ex[e] = x;
@@ -309,10 +314,11 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
         s_geom[1] = stage_bytes;
         s_geom[2] = min(cum, MAX_TILES);
+        s_geom[3] = pbase;
     }
     __syncthreads();
     const uint32_t tmem_base = *s_tmem;
-    const int nstg = s_geom[0], stage_bytes = s_geom[1], T = s_geom[2];
+    const int nstg = s_geom[0], stage_bytes = s_geom[1], T = s_geom[2], NP = s_geom[3];
     for (int i = tid; i < T; i += DEC_THREADS) {            // the tile table, one thread per tile
         int e = 0;
         while (e + 1 < sch.E && s_ex[e + 1].cum <= i) ++e;
@@ -322,13 +328,17 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         const int kb0 = max(x.tb - nt * p.KB, 0), kb1 = min(x.te - nt * p.KB, p.KB);
         const bool last = kb + 1 == kb1;
         int flags = (kb == kb0 ? TF_FIRST : 0) | (last ? TF_LAST : 0) | ((last || (kb + 1) % x.gkb == 0) ? TF_ENDS : 0) |
-                    ((kb0 == 0 && kb1 == p.KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0);
+                    ((kb0 == 0 && kb1 == p.KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0) |
+                    ((kb == kb0 || kb % x.gkb == 0) ? TF_GSTART : 0);
+        const int piece = x.pbase + nt - x.tb / p.KB;
         uint4 v;
         v.x = (uint32_t)kb | ((uint32_t)nt << 16);
         v.y = (uint32_t)flags | ((uint32_t)e << 8) | ((uint32_t)x.rows << 16) | ((uint32_t)x.row0 << 24);
         v.z = (uint32_t)(x.gbase + tile / x.gkb - x.tb / x.gkb);
         // owner of the segment's last tile (needed where the head of a split segment ends)
-        v.w = (last && kb0 == 0 && kb1 != p.KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * p.KB + p.KB - 1) : 0u;
+        v.w = (uint32_t)piece |
+              ((last && kb0 == 0 && kb1 != p.KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * p.KB + p.KB - 1) << 16 : 0u);
+        if (last) s_piece[piece] = i;
         *reinterpret_cast<uint4*>(smem + L::tile_off + 16 * i) = v;
     }
     __syncthreads();
@@ -350,23 +360,22 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         }
     } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------------ MMA issuer
-        // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.
+        // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.  No accumulator
+        // hand-shake is needed: buffer g % 8 is drained by the warpgroup that unpacked the group's last tile j before
+        // it hands over its next tile j + 4, and the group that reuses the buffer starts at tile j + 8 or later.
         const uint32_t idesc = umma_idesc(TOK);
-        bool fresh = true;                           // the next MMA starts a group
         int a = 0, xst = 0;
         uint32_t aphase = 0;
         for (int t = 0; t < T; ++t) {
             const Tile ti(s_tile[t]);
-            const int d = ti.g & (ND - 1);
-            const bool ends = ti.ends();
             if (!wwait(bar_afull + 8 * a, aphase)) break;
-            if (fresh && !wwait(bar_accempty + 8 * d, ((uint32_t)(ti.g >> 3) & 1u) ^ 1u)) break;
             tc_fence_after();
             const uint32_t xs = sbase + L::x_off + xst * X_STAGE;
-            const uint32_t dt = tmem_base + D_COL0 + d * TOK, a0 = tmem_base + a * 64;
+            const uint32_t dt = tmem_base + D_COL0 + (ti.g & (ND - 1)) * TOK, a0 = tmem_base + a * 64;
             const uint64_t b0 = umma_desc_sw128(xs), b1 = umma_desc_sw128(xs + TOK * 128);
+            const uint32_t acc0 = (ti.flags & TF_GSTART) ? 0u : 1u;
             if (elect_one()) {
-                umma_bf16_ts(dt, a0, b0, idesc, fresh ? 0u : 1u);
+                umma_bf16_ts(dt, a0, b0, idesc, acc0);
                 umma_bf16_ts(dt, a0 + 8, b0 + 2, idesc, 1u);
                 umma_bf16_ts(dt, a0 + 16, b0 + 4, idesc, 1u);
                 umma_bf16_ts(dt, a0 + 24, b0 + 6, idesc, 1u);
@@ -374,11 +383,9 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 umma_bf16_ts(dt, a0 + 40, b1 + 2, idesc, 1u);
                 umma_bf16_ts(dt, a0 + 48, b1 + 4, idesc, 1u);
                 umma_bf16_ts(dt, a0 + 56, b1 + 6, idesc, 1u);
-                if (ends) umma_commit(bar_accfull + 8 * d);
                 umma_commit(bar_done + 8 * (t & (DONE_RING - 1)));
             }
             __syncwarp();
-            fresh = ends;
             if (++a == NA) { a = 0; aphase ^= 1u; }
             if (++xst == NXS) xst = 0;
         }
@@ -394,16 +401,63 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 asm volatile("cp.async.commit_group;" ::: "memory");
             }
         };
+        float acc[TOK];                              // this warpgroup's share of the current piece, channel `row`
+#pragma unroll
+        for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
+        int flushed = 0;                             // pieces this warpgroup has handed to the finalizer
+        int prev_t = -1, prev_g = 0, prev_piece = -1;   // its previous tile, if that ended an accumulation group
+        float prev_s = 0.f;
+        bool ok = true;
+        // the group that ended with the warpgroup's previous tile: scale and add (its MMAs finished long ago)
+        auto drain_prev = [&]() -> bool {
+            if (prev_t < 0) return true;
+            if (!wait_done(prev_t)) return false;
+            tc_fence_after();
+            uint32_t v[16];
+            tmem_ld16(lane_taddr + D_COL0 + (prev_g & (ND - 1)) * TOK, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < TOK; ++i) acc[i] = fmaf(prev_s, __uint_as_float(v[i]), acc[i]);
+            tc_fence_before();
+            prev_t = -1;
+            return true;
+        };
+        // Pieces before `upto` are complete as far as this warpgroup goes: add its share to the piece's sum in
+        // shared memory, warpgroup 0 first (it writes), then 1, 2, 3 (they add) -- a fixed order, so the result does
+        // not depend on timing -- and pass the turn on; the finalizer takes the sum after warpgroup 3.
+        auto flush_to = [&](int upto) -> bool {
+            for (; flushed < upto; ++flushed) {
+                const uint32_t par = (uint32_t)flushed & 1u;
+                if (wg == 0) { if (!wwait(bar_flushfree, par ^ 1u)) return false; }
+                else if (!wwait(bar_turn + 8 * (wg - 1), par)) return false;
+                const bool mine = prev_piece == flushed;
+                if (wg == 0) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] = mine ? acc[m] : 0.f;
+                } else if (mine) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] += acc[m];
+                }
+                if (mine) {
+#pragma unroll
+                    for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
+                }
+                warrive(bar_turn + 8 * wg);
+            }
+            return true;
+        };
         x_load(wg);
         int stg = wg % nstg, a = wg;                 // ring stage and A buffer of tile t, kept incrementally
         uint32_t wphase = (uint32_t)(wg / nstg) & 1u;
-        for (int t = wg; t < T; t += 4) {
+        for (int t = wg; ok && t < T; t += 4) {
             const Tile ti(s_tile[t]);
             const ExpertSm& ex = s_ex[ti.e];
             // tile t - 6 is done: A buffer t % 6 and token-tile stage (t + 4) % 10 are free
-            if (!wait_done(t - NA)) break;
+            if (!(ok = wait_done(t - NA))) break;
             x_load(t + 4);
-            if (!wwait(bar_wfull + 8 * stg, wphase)) break;
+            if (!(ok = drain_prev())) break;
+            if (!(ok = flush_to(ti.piece))) break;
+            if (!(ok = wwait(bar_wfull + 8 * stg, wphase))) break;
             tc_fence_after();
             const unsigned char* stage = smem + L::ring_off + stg * stage_bytes;
             const int bits = ex.bits, group = ex.group, has_zeros = ex.has_zeros;
@@ -415,10 +469,15 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
             else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), lane_taddr + a * 64);
             else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
-            // the scale of a group that ends in this tile, for the epilogue thread of the same row
-            if (ti.ends() && group != 0)
-                s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row] =
-                    __half2float(moqe_tile_scales(stage, bits, has_zeros, 0)[row]) * (bits == 8 ? W8_PRESCALE : 1.f);
+            prev_piece = ti.piece;
+            if (ti.ends()) {
+                // the scale of the group that ends with this tile; its accumulator is drained on the next round
+                prev_t = t;
+                prev_g = ti.g;
+                prev_s = (group == 0 ? __half2float(p.ex[ti.e].scales_pc[ti.nt * 128 + row])
+                                     : __half2float(moqe_tile_scales(stage, bits, has_zeros, 0)[row])) *
+                         (bits == 8 ? W8_PRESCALE : 1.f);
+            }
             warrive(bar_wempty + 8 * stg);
             asm volatile("cp.async.wait_group 1;" ::: "memory");      // this tile's token rows have landed
             fence_proxy_async();
@@ -429,42 +488,24 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             while (stg >= nstg) { stg -= nstg; wphase ^= 1u; }
             a = a + 4 >= NA ? a + 4 - NA : a + 4;
         }
+        if (ok) ok = drain_prev();
+        if (ok) flush_to(NP);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp >= EP_WARP0 && warp < EP_WARP0 + 4) {
-        // ------------------------------------------------------------------ epilogue warpgroup
+        // ------------------------------------------------------------------ finalizer warpgroup
+        // Takes each piece's sum once the four dequant warpgroups have added their shares, then stores the rows at
+        // their original positions (fused un-permutation), parks the sum, or adds the parked sums of other CTAs.
         const int et = tid - EP_WARP0 * 32, row = (warp & 3) * 32 + lane;
-        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + D_COL0;
         uint32_t esync_phase = 0;
-        float acc[TOK], oth[TOK];
-        float pc_s = 0.f;
         bool ok = true;
-        for (int t = 0; ok && t < T; ++t) {
-            const Tile ti(s_tile[t]);
-            if (!(ti.flags & (TF_FIRST | TF_ENDS | TF_LAST))) continue;
-            const ExpertSm& ex = s_ex[ti.e];
-            const int n = ti.nt * 128 + row, bits = ex.bits, group = ex.group;
-            if (ti.first()) {
+        for (int q = 0; ok && q < NP; ++q) {
+            const Tile ti(s_tile[s_piece[q]]);       // the piece's last tile carries its facts
+            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows;
+            if (!(ok = wwait(bar_turn + 8 * 3, (uint32_t)q & 1u))) break;
+            float acc[TOK];
 #pragma unroll
-                for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
-                if (group == 0) pc_s = __half2float(p.ex[ti.e].scales_pc[n]) * (bits == 8 ? W8_PRESCALE : 1.f);
-            }
-            const bool head_last = ti.last() && !(ti.flags & (TF_WHOLE | TF_KB0NZ));
-            const int n_others = ti.c_last - (int)blockIdx.x;
-            if (ti.ends()) {
-                const int d = ti.g & (ND - 1);
-                if (!(ok = wwait(bar_accfull + 8 * d, (uint32_t)(ti.g >> 3) & 1u))) break;
-                tc_fence_after();
-                const float s = group == 0 ? pc_s : s_scale[(ti.g & (SCALE_SLOTS - 1)) * 128 + row];
-                uint32_t v[16];
-                tmem_ld16(lane_base + d * TOK, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) acc[i] = fmaf(s, __uint_as_float(v[i]), acc[i]);
-                tc_fence_before();
-                warrive(bar_accempty + 8 * d);
-            }
-            if (!ti.last()) continue;
-            const int j0 = ti.row0, rows = ti.rows;
+            for (int m = 0; m < TOK; ++m) acc[m] = s_out[m * 128 + row];
+            warrive(bar_flushfree);
             if (ti.flags & TF_WHOLE) {
                 // the whole K of this segment was ours: round and store rows at their original positions
                 if (n < p.N) {
@@ -488,9 +529,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                     atomicExch(p.flags + blockIdx.x, 1u);
                 }
             } else {
-                // The last tile of the head of a segment whose tail belongs to the following CTAs -- always a CTA's
-                // LAST piece, while the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as
-                // its first piece).  Fetch their sum in CTA order (deterministic) and add the own one (registers).
+                // The head of a segment whose tail belongs to the following CTAs -- always a CTA's LAST piece, while
+                // the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as its first piece).
+                // Wait for their flags (bounded), add their sums in CTA order (deterministic), store.
+                const int n_others = ti.c_last - (int)blockIdx.x;
                 for (int i = et; i < n_others; i += 128) {
                     volatile unsigned* f = p.flags + blockIdx.x + 1 + i;
                     unsigned long long t_start = 0;
@@ -508,26 +550,24 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 if (!(ok = wwait(bar_esync, esync_phase))) break;
                 esync_phase ^= 1u;
                 if (*s_abort) { ok = false; break; }
-#pragma unroll
-                for (int m = 0; m < TOK; ++m) oth[m] = 0.f;
                 for (int c0 = 0; c0 < n_others; c0 += 2) {             // two contributors' loads in flight at a time
                     float part[2][TOK];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0 + u) * TOK * 128 + row;
 #pragma unroll
-                        for (int m = 0; m < TOK; ++m) part[u][m] = (c0 + u < n_others && m < ti.rows) ? __ldcg(src + m * 128) : 0.f;
+                        for (int m = 0; m < TOK; ++m) part[u][m] = (c0 + u < n_others && m < rows) ? __ldcg(src + m * 128) : 0.f;
                     }
 #pragma unroll
                     for (int u = 0; u < 2; ++u)
 #pragma unroll
-                        for (int m = 0; m < TOK; ++m) oth[m] += part[u][m];
+                        for (int m = 0; m < TOK; ++m) acc[m] += part[u][m];
                 }
                 for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
                 if (n < p.N) {
 #pragma unroll
                     for (int m = 0; m < TOK; ++m)
-                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m] + oth[m]));
+                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
                 }
             }
         }
