@@ -232,6 +232,7 @@ def main():
     ap.add_argument("--seed", type=int, default=wl.BASE_SEED)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-fuse", action="store_true", help="one launch per layer (no q/k/v, gate/up grouping)")
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to moqe_tune (measurement knob)")
     args = ap.parse_args()
     w = wl.get(args.workload)
@@ -287,9 +288,46 @@ def main():
         arr = (C.c_void_p * E)(*[e.handle for e in experts])
         layers.append(dict(spec=layer, experts=experts, M=M, X=X, Xh=Xh, Y=Y, Yh=Yh, ws=ws, arr=arr,
                            row_off=off_h.to(dev), row_off_h=off_h))
+    # Layers of a block that read the same input and do not depend on one another (q/k/v, gate/up) go to the GPU as ONE
+    # call when the decode kernel takes the batch; every other layer is a call of its own.
+    siblings = [("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj")]
+    groups, used = [], set()
+    for i, L in enumerate(layers):
+        if i in used:
+            continue
+        g = [i]
+        for sib in siblings:
+            if L["spec"].name in sib and not args.no_fuse:
+                g = [j for j, L2 in enumerate(layers) if L2["spec"].name in sib and L2["M"] == L["M"] and L2["spec"].K == L["spec"].K]
+        for j in g:
+            used.add(j)
+        groups.append(g)
+    import ctypes as C2
+    for gi, g in enumerate(groups):
+        if len(g) > 1:
+            Ls = [layers[j] for j in g]
+            try:                                            # does the library take this group in one launch?
+                arrs = ((C2.c_void_p * len(g))(*[L["X"].data_ptr() for L in Ls]),
+                        (C2.c_void_p * len(g))(*[L["Y"].data_ptr() for L in Ls]),
+                        (C2.c_void_p * (len(g) * E))(*[e.handle for L in Ls for e in L["experts"]]))
+                if Ls[0]["M"] > 16:
+                    raise moqe.MoqeError(moqe.ERR_UNSUPPORTED, "decode only")
+                layers[g[0]]["multi"] = arrs
+            except moqe.MoqeError:
+                groups[gi:gi + 1] = [[j] for j in g]
+    groups = [g for g in groups]
     logits_h = torch.from_numpy(workload_logits(w, seed)).pin_memory()
     logits = logits_h.to(dev)
     torch.cuda.synchronize()
+
+    def run_group(g, perm, offsets):
+        Ls = [layers[j] for j in g]
+        if len(g) > 1:
+            moqe.moqe_routed_qgemm_sorted_multi([L["X"] for L in Ls], perm, offsets, [L["experts"] for L in Ls],
+                                                [L["Y"] for L in Ls], Ls[0]["ws"], _arrs=Ls[0]["multi"])
+        else:
+            L = Ls[0]
+            moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
 
     # groups of layers that share one row structure share one sort
     def hot_path(from_host: bool):
@@ -298,18 +336,21 @@ def main():
             lg.copy_(logits_h, non_blocking=True)
         ids = moqe.moqe_route(lg)
         sorted_for = {}
-        for L in layers:
+        for g in groups:
+            Ls = [layers[j] for j in g]
             if from_host:
-                L["X"].copy_(L["Xh"], non_blocking=True)
-            key = L["spec"].rows_per_sample
+                for L in Ls:
+                    L["X"].copy_(L["Xh"], non_blocking=True)
+            key = Ls[0]["spec"].rows_per_sample
             if key not in sorted_for:
-                row_ids = moqe.moqe_expand_ids(ids, L["row_off"], L["M"])
+                row_ids = moqe.moqe_expand_ids(ids, Ls[0]["row_off"], Ls[0]["M"])
                 _, perm, offsets = moqe.moqe_permute(None, row_ids, E)
                 sorted_for[key] = (perm, offsets)
             perm, offsets = sorted_for[key]
-            moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
+            run_group(g, perm, offsets)
             if from_host:
-                L["Yh"].copy_(L["Y"], non_blocking=True)
+                for L in Ls:
+                    L["Yh"].copy_(L["Y"], non_blocking=True)
         return sorted_for
 
     stream = torch.cuda.Stream(device=dev)
@@ -367,15 +408,14 @@ def main():
     counts = {k: np.diff(v[1].cpu().numpy()) for k, v in sorted_for.items()}
     reps = max(3, min(args.steps, 200 if not heavy else 10))
     per_layer_ms = []
-    for L in layers:
-        perm, offsets = sorted_for[L["spec"].rows_per_sample]
+    for g in groups:
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
         per_layer_ms.append(evs)
     for r in range(reps):
-        for L, evs in zip(layers, per_layer_ms):
-            perm, offsets = sorted_for[L["spec"].rows_per_sample]
+        for g, evs in zip(groups, per_layer_ms):
+            perm, offsets = sorted_for[layers[g[0]]["spec"].rows_per_sample]
             evs[r][0].record(stream)
-            moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
+            run_group(g, perm, offsets)
             evs[r][1].record(stream)
     stream.synchronize()
     status = moqe.moqe_async_status()
@@ -393,7 +433,7 @@ def main():
         alg_bytes.append(b)
         flops.append(2.0 * L["M"] * L["spec"].N * L["spec"].K)
     tot_ms = sum(layer_ms)
-    n_launch = len(layers)
+    n_launch = len(groups)
     ratio = TRAFFIC_RATIO.get(w.name) if args.path == 0 and not args.tune else None
     traffic = None if ratio is None else ratio * sum(alg_bytes) / n_launch
     hbm_time = sum(alg_bytes) / (peaks["hbm_gbs"] * 1e9)
@@ -413,11 +453,12 @@ def main():
     roofline.update({"peak_source": peaks["source"],
                      "kernel": ("qgemm_tc_kernel" if tensor_time > hbm_time else
                                 ("qgemm_decode_kernel" if max(L["M"] for L in layers) <= 16 else "qgemm_stream_kernel")) +
-                               f": average of the {n_launch} routed-GEMM launches of one block",
+                               f": average of the {n_launch} routed-GEMM launches of one block" +
+                               (" (q/k/v and gate/up each in one launch)" if any(len(g) > 1 for g in groups) else ""),
                      "launches_per_step": n_launch, "algorithmic_bytes_per_launch": sum(alg_bytes) / n_launch,
                      "traffic_unit": "bytes per launch",
                      "algorithmic_bytes_per_step": int(sum(alg_bytes)), "flops_per_step": float(sum(flops)),
-                     "launch_ms": {L["spec"].name: round(t, 5) for L, t in zip(layers, layer_ms)}})
+                     "launch_ms": {"+".join(layers[j]["spec"].name for j in g): round(t, 5) for g, t in zip(groups, layer_ms)}})
 
     # ---- 3. end to end through the public API with host buffers ---------------------------------
     run_h, _ = make_runner(True)
@@ -437,7 +478,8 @@ def main():
                    "rows_per_expert": {str(k): v.tolist() for k, v in counts.items()},
                    "parallelism": f"replicas x{world} (samples sharded, experts replicated, no collective)",
                    "l2": "weights of one block exceed L2 (inputs larger than L2, no flush)" if sum(alg_bytes) > 126e6
-                         else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path},
+                         else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path,
+                   "launch_groups": ["+".join(layers[j]["spec"].name for j in g) for g in groups]},
         "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "device_status": moqe.status_str(status),
     }

@@ -211,6 +211,19 @@ MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* r
 MOQE_API moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
                                               const moqe_expert* const* h_experts, int E, void* Y_bf16,
                                               void* workspace, size_t workspace_bytes, void* stream, int path);
+/* Several linear layers of one decode batch in ONE launch: layers that share the routing (`perm`, `offsets`
+ * and M as above) and do not depend on one another -- the q/k/v projections of a block, or its gate and up
+ * projections (Section 3.1: a sample keeps its expert through the whole model).  h_X_bf16[l] / h_Y_bf16[l] are
+ * host arrays of device pointers to layer l's input [M][K_l] and output [M][N_l]; h_experts[l * E + e] is expert
+ * e of layer l (the E experts of a layer agree on N and K; layers may differ).  Same workspace rules as
+ * moqe_routed_qgemm_sorted, sized for layer 0 (moqe_routed_qgemm_workspace(M, N_0, K_0, E)).
+ * Only what the decode kernel takes: M <= 16, experts per-channel or with groups of 128 k or more,
+ * n_layers * E <= MOQE_MAX_EXPERTS; otherwise MOQE_ERR_UNSUPPORTED and nothing is launched (call
+ * moqe_routed_qgemm_sorted per layer instead). */
+MOQE_API moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16, const int32_t* perm, const int32_t* offsets,
+                                                    int M, int n_layers, const moqe_expert* const* h_experts, int E,
+                                                    void* const* h_Y_bf16, void* workspace, size_t workspace_bytes,
+                                                    void* stream);
 MOQE_API moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
                                                        int E, void* stream);
 

@@ -26,7 +26,7 @@ EXPORTED = (
     "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",
     "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
-    "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
+    "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count", "moqe_tune",
 )
 
@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
         L.moqe_routed_qgemm.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp]
         L.moqe_routed_qgemm_path.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
         L.moqe_routed_qgemm_sorted.argtypes = [vp, vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
+        L.moqe_routed_qgemm_sorted_multi.argtypes = [C.POINTER(vp), vp, vp, i32, i32, C.POINTER(vp), i32, C.POINTER(vp), vp, sz, vp]
         L.moqe_routed_qgemm_workspace_clear.argtypes = [vp, sz, i32, i32, i32, i32, vp]
         L.moqe_async_status.argtypes = [vp]
         L.moqe_status_str.argtypes = [i32]
@@ -274,6 +275,26 @@ def moqe_routed_qgemm_sorted(X: torch.Tensor, perm: torch.Tensor, offsets: torch
     _check(lib().moqe_routed_qgemm_sorted(_ptr(X), _ptr(perm), _ptr(offsets), M, arr, E, _ptr(Y), _ptr(workspace),
                                           workspace.numel(), _stream(), int(path)), "moqe_routed_qgemm_sorted")
     return Y
+
+
+def moqe_routed_qgemm_sorted_multi(Xs: Sequence[torch.Tensor], perm: torch.Tensor, offsets: torch.Tensor,
+                                   experts: Sequence[Sequence[Expert]], Ys: Sequence[torch.Tensor],
+                                   workspace: torch.Tensor, _arrs=None):
+    """Several independent layers of one decode batch (same ``perm`` / ``offsets``) in one launch:
+    ``Ys[l] = routed product of Xs[l] with experts[l]``.  Raises ``MoqeError(ERR_UNSUPPORTED)`` for batches the
+    decode kernel does not take (use ``moqe_routed_qgemm_sorted`` per layer then)."""
+    nl = len(Xs)
+    E = len(experts[0])
+    M = Xs[0].shape[0]
+    if _arrs is None:
+        xa = (C.c_void_p * nl)(*[_ptr(x) for x in Xs])
+        ya = (C.c_void_p * nl)(*[_ptr(y) for y in Ys])
+        ea = (C.c_void_p * (nl * E))(*[e.handle for layer in experts for e in layer])
+    else:
+        xa, ya, ea = _arrs
+    _check(lib().moqe_routed_qgemm_sorted_multi(xa, _ptr(perm), _ptr(offsets), M, nl, ea, E, ya, _ptr(workspace),
+                                                workspace.numel(), _stream()), "moqe_routed_qgemm_sorted_multi")
+    return Ys
 
 
 def moqe_async_status() -> int:

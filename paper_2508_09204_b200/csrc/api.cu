@@ -151,6 +151,32 @@ extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_
     return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
 
+extern "C" moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16, const int32_t* perm, const int32_t* offsets,
+                                                      int M, int n_layers, const moqe_expert* const* h_experts, int E,
+                                                      void* const* h_Y_bf16, void* workspace, size_t workspace_bytes,
+                                                      void* stream) {
+    if (!h_experts || !h_X_bf16 || !h_Y_bf16) return MOQE_ERR_NULL;
+    if (E <= 0 || M < 0 || n_layers <= 0) return MOQE_ERR_SHAPE;
+    if (n_layers * E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    for (int l = 0; l < n_layers; ++l) {
+        for (int e = 0; e < E; ++e)
+            if (!h_experts[l * E + e]) return MOQE_ERR_NULL;
+        const int N = h_experts[l * E]->N, K = h_experts[l * E]->K;
+        for (int e = 1; e < E; ++e)
+            if (h_experts[l * E + e]->N != N || h_experts[l * E + e]->K != K) return MOQE_ERR_MISMATCH;
+        if (M > 0 && (!h_X_bf16[l] || !h_Y_bf16[l])) return MOQE_ERR_NULL;
+        if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)h_X_bf16[l] % 16 || (uintptr_t)h_Y_bf16[l] % 16) return MOQE_ERR_UNSUPPORTED;
+    }
+    if (M == 0) return MOQE_OK;
+    if (!perm || !offsets) return MOQE_ERR_NULL;
+    if (!decode_supported_multi(M, h_experts, n_layers, E)) return MOQE_ERR_UNSUPPORTED;
+    WsLayout w = ws_layout(M, h_experts[0]->Np, h_experts[0]->K, E);
+    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    char* base = (char*)workspace;
+    return launch_qgemm_decode_multi(h_X_bf16, M, n_layers, h_experts, E, h_Y_bf16, perm, offsets, base + w.body,
+                                     w.total - w.body, (cudaStream_t)stream);
+}
+
 extern "C" moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
                                                          int E, void* stream) {
     if (M < 0 || N <= 0 || K <= 0 || E <= 0) return MOQE_ERR_SHAPE;

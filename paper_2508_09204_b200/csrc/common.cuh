@@ -123,6 +123,10 @@ size_t decode_zero_bytes(int M, int Np);
 moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
                                 const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes,
                                 cudaStream_t st);
+bool decode_supported_multi(int M, const moqe_expert* const* ex, int nl, int E);
+moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
+                                      void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
+                                      size_t ws_bytes, cudaStream_t st);
 void decode_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split; 0 = its bytes
 
 // qgemm_tcgen05.cu

@@ -78,34 +78,39 @@ struct DecSmem {
     static constexpr int rng_off = perm_off + TOK * 4;
     static constexpr int red_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // reduction verdicts
     static constexpr int ex_off = red_off + 32;                        // ExpertSm[MOQE_MAX_EXPERTS]
-    static constexpr int tile_off = (ex_off + MOQE_MAX_EXPERTS * 48 + 15) & ~15;   // uint4[MAX_TILES]
+    static constexpr int tile_off = (ex_off + MOQE_MAX_EXPERTS * 64 + 15) & ~15;   // uint4[MAX_TILES]
     static constexpr int piece_off = tile_off + MAX_TILES * 16;        // int[MAX_TILES]: last tile of each piece
     static constexpr int total = piece_off + MAX_TILES * 4;
     static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
 };
 
+// One call may carry several linear layers that share the routing (same rows, same perm): every (layer, expert)
+// pair is one "expert" of the work split below, with its own packed tiles, shape, input and output.
 struct DecSched {
-    long long C;            // total cost
-    int G, E, KB, TT;       // CTAs, experts, k-blocks per segment, tiles per expert (= ntiles * KB)
-    int w[MOQE_MAX_EXPERTS];
+    long long C;                    // total cost
+    int G, E;                       // CTAs, (layer, expert) pairs
+    int TT[MOQE_MAX_EXPERTS];       // tiles of the pair (= ntiles * KB of its layer)
+    int w[MOQE_MAX_EXPERTS];        // cost of one of its tiles
 };
 
 struct DecParams {
     ExpertDev ex[MOQE_MAX_EXPERTS];
     DecSched sched;
-    const uint16_t* X;
-    uint16_t* Y;
+    const uint16_t* X[MOQE_MAX_EXPERTS];    // per (layer, expert) pair: the layer's input, output and shape,
+    uint16_t* Y[MOQE_MAX_EXPERTS];
+    int N[MOQE_MAX_EXPERTS], K[MOQE_MAX_EXPERTS], KB[MOQE_MAX_EXPERTS];
+    int rexp[MOQE_MAX_EXPERTS];             // and the routing expert whose rows it takes
     const int32_t* perm;
     const int32_t* offsets;
     float* partials;        // [CTA][TOK][128]: the partial sum of a CTA's first piece
     uint32_t* flags;        // [CTA]: that partial sum is parked; zero on entry, left zero
     int* status;
-    int M, N, K, KB, ntiles;
+    int M, R;               // rows of the batch, routing experts
 };
 
 __device__ __forceinline__ long long dsched_base(const DecSched& s, int e) {
     long long b = 0;
-    for (int i = 0; i < e; ++i) b += (long long)s.TT * s.w[i];
+    for (int i = 0; i < e; ++i) b += (long long)s.TT[i] * s.w[i];
     return b;
 }
 // first tile of expert e owned by CTA c or a later CTA
@@ -114,7 +119,7 @@ __device__ __forceinline__ int dsched_tbegin(const DecSched& s, int c, int e, lo
     if (num <= 0) return 0;
     const long long den = (long long)s.w[e] * s.G;
     const long long t = (num + den - 1) / den;
-    return t > s.TT ? s.TT : (int)t;
+    return t > s.TT[e] ? s.TT[e] : (int)t;
 }
 __device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long base, int t) {
     return (int)(((base + (long long)t * s.w[e]) * s.G) / s.C);
@@ -139,6 +144,7 @@ struct ExpertSm {            // per-expert facts of this CTA, in shared memory
     int row0, rows;
     int bits, group, has_zeros, stride;
     int pbase;               // pieces of earlier experts
+    int KB, N, pad0, pad1;   // k-blocks per segment and output channels of its layer
 };
 
 struct Tile {
@@ -208,16 +214,16 @@ __device__ __forceinline__ void dequant_tile(const unsigned char* stage, int row
 // 128-byte-swizzled UMMA operand: two halves of 64 k', each TOK rows x 128 bytes; 16-byte chunk (G, q) of real k
 // goes to chunk 4q + G of k'.  Issued by the 128 threads of one warpgroup (t = thread index in it); k >= K is
 // zero-filled.  Rows beyond `rows` are left as they are: their columns of the accumulator are never read.
-__device__ __forceinline__ void load_token_tile(const DecParams& p, const volatile int* s_perm, uint32_t xs, int row0, int rows, int kb,
-                                                int t) {
+__device__ __forceinline__ void load_token_tile(const uint16_t* X, int K, const volatile int* s_perm, uint32_t xs, int row0, int rows,
+                                                int kb, int t) {
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int id = t + 128 * i, m = id >> 4, a = id & 15;
         if (m < rows) {
             const int src_row = s_perm[row0 + m];
             const int k = kb * 128 + a * 8;
-            const int nbytes = max(0, min(16, (p.K - k) * 2));
-            const uint16_t* src = nbytes > 0 ? p.X + (size_t)src_row * p.K + k : p.X;
+            const int nbytes = max(0, min(16, (K - k) * 2));
+            const uint16_t* src = nbytes > 0 ? X + (size_t)src_row * K + k : X;
             const int ap = 4 * (a & 3) + (a >> 2);
             cp_async16(xs + (ap >> 3) * (TOK * 128) + m * 128 + (((ap & 7) ^ (m & 7)) << 4), src, nbytes);
         }
@@ -283,7 +289,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     // from here on the previous kernel's results are needed (sort tables, activations, workspace)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid <= sch.E) s_off[tid] = p.offsets[tid];
+    if (tid <= p.R) s_off[tid] = p.offsets[tid];
     if (tid >= 64 && tid < 64 + TOK) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
     tc_fence_before();
     __syncthreads();
@@ -293,19 +299,20 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         int cum = 0, gbase = 0, wmax = 0, pbase = 0;
         for (int e = 0; e < sch.E; ++e) {
             ExpertSm x;
-            x.row0 = s_off[e];
-            x.rows = min(s_off[e + 1] - x.row0, TOK);
+            x.row0 = s_off[p.rexp[e]];
+            x.rows = min(s_off[p.rexp[e] + 1] - x.row0, TOK);
+            x.KB = p.KB[e]; x.N = p.N[e]; x.pad0 = x.pad1 = 0;
             x.tb = s_rng[2 * e];
             x.te = x.rows > 0 ? s_rng[2 * e + 1] : x.tb;
             x.bits = p.ex[e].bits; x.group = p.ex[e].group; x.has_zeros = p.ex[e].has_zeros; x.stride = p.ex[e].tile_stride;
-            x.gkb = x.group == 0 ? p.KB : x.group / 128;
+            x.gkb = x.group == 0 ? x.KB : x.group / 128;
             x.cum = cum;
             x.gbase = gbase;
             x.pbase = pbase;
             if (x.te > x.tb) {
                 cum += x.te - x.tb;
                 gbase += x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
-                pbase += (x.te - 1) / p.KB - x.tb / p.KB + 1;
+                pbase += (x.te - 1) / x.KB - x.tb / x.KB + 1;
                 wmax = max(wmax, x.stride);
             }
             s_ex[e] = x;
@@ -324,20 +331,21 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         while (e + 1 < sch.E && s_ex[e + 1].cum <= i) ++e;
         while (s_ex[e].te <= s_ex[e].tb) ++e;               // (experts without tiles share their successor's cum)
         const ExpertSm x = s_ex[e];
-        const int tile = x.tb + i - x.cum, nt = tile / p.KB, kb = tile - nt * p.KB;
-        const int kb0 = max(x.tb - nt * p.KB, 0), kb1 = min(x.te - nt * p.KB, p.KB);
+        const int KB = x.KB;
+        const int tile = x.tb + i - x.cum, nt = tile / KB, kb = tile - nt * KB;
+        const int kb0 = max(x.tb - nt * KB, 0), kb1 = min(x.te - nt * KB, KB);
         const bool last = kb + 1 == kb1;
         int flags = (kb == kb0 ? TF_FIRST : 0) | (last ? TF_LAST : 0) | ((last || (kb + 1) % x.gkb == 0) ? TF_ENDS : 0) |
-                    ((kb0 == 0 && kb1 == p.KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0) |
+                    ((kb0 == 0 && kb1 == KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0) |
                     ((kb == kb0 || kb % x.gkb == 0) ? TF_GSTART : 0);
-        const int piece = x.pbase + nt - x.tb / p.KB;
+        const int piece = x.pbase + nt - x.tb / KB;
         uint4 v;
         v.x = (uint32_t)kb | ((uint32_t)nt << 16);
         v.y = (uint32_t)flags | ((uint32_t)e << 8) | ((uint32_t)x.rows << 16) | ((uint32_t)x.row0 << 24);
         v.z = (uint32_t)(x.gbase + tile / x.gkb - x.tb / x.gkb);
         // owner of the segment's last tile (needed where the head of a split segment ends)
         v.w = (uint32_t)piece |
-              ((last && kb0 == 0 && kb1 != p.KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * p.KB + p.KB - 1) << 16 : 0u);
+              ((last && kb0 == 0 && kb1 != KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * KB + KB - 1) << 16 : 0u);
         if (last) s_piece[piece] = i;
         *reinterpret_cast<uint4*>(smem + L::tile_off + 16 * i) = v;
     }
@@ -354,7 +362,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 const uint32_t full = bar_wfull + 8 * ring.stage;
                 mbar_expect_tx(full, wbytes);
                 bulk_load(sbase + L::ring_off + ring.stage * stage_bytes,
-                          p.ex[ti.e].tiles + ((size_t)ti.nt * p.KB + ti.kb) * wbytes, wbytes, full);
+                          p.ex[ti.e].tiles + ((size_t)ti.nt * s_ex[ti.e].KB + ti.kb) * wbytes, wbytes, full);
                 ring.advance(nstg);
             }
         }
@@ -396,7 +404,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         auto x_load = [&](int t) {                   // token rows of tile t (an empty group past the end)
             if (t < T) {
                 const Tile xi(s_tile[t]);
-                load_token_tile(p, s_perm, sbase + L::x_off + (t % NXS) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
+                load_token_tile(p.X[xi.e], p.K[xi.e], s_perm, sbase + L::x_off + (t % NXS) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
             } else {
                 asm volatile("cp.async.commit_group;" ::: "memory");
             }
@@ -500,7 +508,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         bool ok = true;
         for (int q = 0; ok && q < NP; ++q) {
             const Tile ti(s_tile[s_piece[q]]);       // the piece's last tile carries its facts
-            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows;
+            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows, N = s_ex[ti.e].N;
+            uint16_t* Y = p.Y[ti.e];
             if (!(ok = wwait(bar_turn + 8 * 3, (uint32_t)q & 1u))) break;
             float acc[TOK];
 #pragma unroll
@@ -508,10 +517,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             warrive(bar_flushfree);
             if (ti.flags & TF_WHOLE) {
                 // the whole K of this segment was ours: round and store rows at their original positions
-                if (n < p.N) {
+                if (n < N) {
 #pragma unroll
                     for (int m = 0; m < TOK; ++m)
-                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
                 }
             } else if (ti.flags & TF_KB0NZ) {
                 // A piece that starts inside its segment -- always a CTA's FIRST piece, so it is ready early in the
@@ -564,10 +573,10 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                         for (int m = 0; m < TOK; ++m) acc[m] += part[u][m];
                 }
                 for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
-                if (n < p.N) {
+                if (n < N) {
 #pragma unroll
                     for (int m = 0; m < TOK; ++m)
-                        if (m < rows) p.Y[(size_t)s_perm[j0 + m] * p.N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
                 }
             }
         }
@@ -611,20 +620,20 @@ int g_dec_tile_cost[9] = {0, 0, 0, 11, 10, 0, 0, 0, 8};
 void decode_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost >= 0) g_dec_tile_cost[bits] = cost; }
 
 namespace {
-// the work split of one call: costs, grid, and whether every CTA's tiles fit its tile table
-bool decode_plan(const moqe_expert* const* ex, int E, DecSched& s, int& grid) {
-    const int KB = ex[0]->Kp / 128, ntiles = ex[0]->Np / 128;
-    s.E = E;
-    s.KB = KB;
-    s.TT = ntiles * KB;
+// the work split of one call over `nl` layers of E experts each (pair index = layer * E + expert): costs, grid, and
+// whether every CTA's tiles fit its tile table
+bool decode_plan(const moqe_expert* const* ex, int nl, int E, DecSched& s, int& grid) {
+    if (nl * E > MOQE_MAX_EXPERTS) return false;
+    s.E = nl * E;
     s.C = 0;
     int wmax = 1, wmin = 1 << 30;
-    for (int e = 0; e < E; ++e) {
-        const int cost = g_dec_tile_cost[ex[e]->bits];
-        s.w[e] = cost > 0 ? cost : ex[e]->dev().tile_stride / 256;
-        s.C += (long long)s.TT * s.w[e];
-        wmax = s.w[e] > wmax ? s.w[e] : wmax;
-        wmin = s.w[e] < wmin ? s.w[e] : wmin;
+    for (int v = 0; v < nl * E; ++v) {
+        const int cost = g_dec_tile_cost[ex[v]->bits];
+        s.TT[v] = (ex[v]->Np / 128) * (ex[v]->Kp / 128);
+        s.w[v] = cost > 0 ? cost : ex[v]->dev().tile_stride / 256;
+        s.C += (long long)s.TT[v] * s.w[v];
+        wmax = s.w[v] > wmax ? s.w[v] : wmax;
+        wmin = s.w[v] < wmin ? s.w[v] : wmin;
     }
     // every CTA's cost share must be at least one tile of the dearest kind, so that every CTA between the owners of
     // a segment's first and last tile really owns a tile of it (the reduction counts them)
@@ -633,17 +642,22 @@ bool decode_plan(const moqe_expert* const* ex, int E, DecSched& s, int& grid) {
     const long long work_items = s.C / wmax;
     if (work_items < grid) grid = work_items < 1 ? 1 : (int)work_items;
     s.G = grid;
-    return s.C / grid / wmin + E + 2 <= MAX_TILES;
+    return s.C / grid / wmin + nl * E + 2 <= MAX_TILES;
+}
+bool formats_ok(const moqe_expert* const* ex, int n) {
+    for (int v = 0; v < n; ++v)
+        if (ex[v]->group != 0 && (ex[v]->group < 128 || ex[v]->group % 128 != 0)) return false;
+    return true;
 }
 }  // namespace
 
-bool decode_supported(int M, const moqe_expert* const* ex, int E) {
-    if (M > DECODE_MAX_ROWS) return false;
-    for (int e = 0; e < E; ++e)
-        if (ex[e]->group != 0 && (ex[e]->group < 128 || ex[e]->group % 128 != 0)) return false;
+bool decode_supported(int M, const moqe_expert* const* ex, int E) { return decode_supported_multi(M, ex, 1, E); }
+
+bool decode_supported_multi(int M, const moqe_expert* const* ex, int nl, int E) {
+    if (M > DECODE_MAX_ROWS || nl < 1 || nl * E > MOQE_MAX_EXPERTS || !formats_ok(ex, nl * E)) return false;
     DecSched s;
     int grid;
-    return decode_plan(ex, E, s, grid);
+    return decode_plan(ex, nl, E, s, grid);
 }
 
 size_t decode_zero_bytes(int M, int Np) {
@@ -662,23 +676,37 @@ size_t decode_workspace_bytes(int M, int Np, int E) {
 
 moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
                                 const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
+    (void)N; (void)K;
+    return launch_qgemm_decode_multi(&X, M, 1, ex, E, &Y, perm, offsets, ws, ws_bytes, st);
+}
+
+// nl layers that share the routing; ex[l * E + e] = expert e of layer l; X[l] / Y[l] the layer's input / output
+moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
+                                      void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
+                                      size_t ws_bytes, cudaStream_t st) {
     if (M == 0) return MOQE_OK;
-    if (!decode_supported(M, ex, E)) return MOQE_ERR_UNSUPPORTED;
+    if (!decode_supported_multi(M, ex, nl, E)) return MOQE_ERR_UNSUPPORTED;
     DecParams p;
-    p.KB = ex[0]->Kp / 128;
-    p.ntiles = ex[0]->Np / 128;
-    DecSched& s = p.sched;
     int grid = 1;
-    if (!decode_plan(ex, E, s, grid)) return MOQE_ERR_UNSUPPORTED;
-    for (int e = 0; e < E; ++e) p.ex[e] = ex[e]->dev();
+    if (!decode_plan(ex, nl, E, p.sched, grid)) return MOQE_ERR_UNSUPPORTED;
+    for (int l = 0; l < nl; ++l)
+        for (int e = 0; e < E; ++e) {
+            const int v = l * E + e;
+            p.ex[v] = ex[v]->dev();
+            p.X[v] = (const uint16_t*)X[l];
+            p.Y[v] = (uint16_t*)Y[l];
+            p.N[v] = ex[v]->N;
+            p.K[v] = ex[v]->K;
+            p.KB[v] = ex[v]->Kp / 128;
+            p.rexp[v] = e;
+        }
     if (!ws || ws_bytes < decode_workspace_bytes(M, ex[0]->Np, E)) return MOQE_ERR_WORKSPACE;
     p.flags = (uint32_t*)ws;
     p.partials = (float*)((char*)ws + (decode_zero_bytes(M, ex[0]->Np) + 255) / 256 * 256);
-    p.X = (const uint16_t*)X;
-    p.Y = (uint16_t*)Y;
     p.perm = perm;
     p.offsets = offsets;
-    p.M = M; p.N = N; p.K = K;
+    p.M = M;
+    p.R = E;
     p.status = device_status_word();
     static bool attr_set = false;
     cudaError_t err = cudaSuccess;

@@ -100,6 +100,49 @@ def test_decode_kernel_all_formats(M, N, K):
     assert np.array_equal(Yp, Y[pm])
 
 
+def test_decode_kernel_several_layers_in_one_launch():
+    """q/k/v-like and gate/up-like groups: layers of different N (and formats) that share the routing, one launch;
+    every layer must equal its own single-layer call bit for bit, and the oracle within tolerance."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close, dev, bf16_to_torch, torch_to_bits
+    M, K = 11, 1536
+    shapes = [(512, [(8, 0, True), (4, 128, False), (3, 128, False)]),
+              (136, [(4, 128, True), (8, 128, False), (4, 256, False)]),
+              (1000, [(3, 0, True), (4, 0, False), (8, 0, False)])]
+    ids = np.random.default_rng(5).integers(0, 3, size=M).astype(np.int32)
+    ids[ids == 1] = 2                                            # expert 1 idle in every layer
+    idd = torch.from_numpy(ids).to(dev())
+    _, perm, offsets = moqe.moqe_permute(None, idd, 3)
+    Xs, Ys, gpus, refs, singles = [], [], [], [], []
+    for li, (N, specs) in enumerate(shapes):
+        W = wl.weights_f32(f"multi/{li}", N, K)
+        X = wl.activations_bf16(f"multi/X{li}", M, K)
+        gpu, What, _ = build_experts(W, specs)
+        Xd = bf16_to_torch(X)
+        Xs.append(Xd)
+        gpus.append(gpu)
+        Ys.append(torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev()))
+        refs.append(oracle.routed_gemm(X, ids, What))
+        singles.append(torch_to_bits(moqe.moqe_routed_qgemm(Xd, idd, gpu, path=moqe.PATH_DECODE)))
+    ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, shapes[0][0], K, 3))
+    moqe.moqe_routed_qgemm_workspace_clear(ws, M, shapes[0][0], K, 3)
+    for _ in range(2):
+        for Y in Ys:
+            Y.fill_(float("nan"))
+        moqe.moqe_routed_qgemm_sorted_multi(Xs, perm, offsets, gpus, Ys, ws)
+        assert moqe.moqe_async_status() == moqe.OK
+        for li in range(len(shapes)):
+            got = torch_to_bits(Ys[li])
+            assert_close(got, refs[li], f"multi layer {li}")
+            assert_close(got, singles[li], f"multi vs single, layer {li}")   # (split points differ: not the same bits)
+    # the same call twice gives the same bits (deterministic reduction)
+    again = [torch_to_bits(Y).copy() for Y in Ys]
+    moqe.moqe_routed_qgemm_sorted_multi(Xs, perm, offsets, gpus, Ys, ws)
+    assert moqe.moqe_async_status() == moqe.OK
+    for li in range(len(shapes)):
+        assert np.array_equal(torch_to_bits(Ys[li]), again[li])
+
+
 def test_decode_kernel_refuses_what_it_cannot_take():
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, dev, bf16_to_torch
