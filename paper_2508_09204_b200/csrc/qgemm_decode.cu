@@ -52,13 +52,14 @@ namespace moqe {
 namespace {
 
 constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
-constexpr int DQ_WARPS = 16, EP_WARP0 = 16, MMA_WARP = 20, W_WARP = 21;
+constexpr int NWG = 5;                                  // dequant warpgroups; warpgroup w takes tiles t = w (mod 5)
+constexpr int DQ_WARPS = 4 * NWG, MMA_WARP = 20, W_WARP = 21;
 constexpr int DEC_THREADS = 22 * 32;
-constexpr int RING_BYTES = 150 * 1024;                  // packed-weight ring
+constexpr int RING_BYTES = 142 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
 constexpr int ND = 8;                                   // accumulator buffers (TOK columns each), group g -> g % 8
-constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
+constexpr int NXS = 12;                                 // token-tile stages, tile t -> t % 12
 constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
 constexpr int TMEM_COLS = 512;
@@ -370,7 +371,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.  No accumulator
         // hand-shake is needed: buffer g % 8 is drained by the warpgroup that unpacked the group's last tile j before
-        // it hands over its next tile j + 4, and the group that reuses the buffer starts at tile j + 8 or later.
+        // it hands over its next tile j + 5, and the group that reuses the buffer starts at tile j + 8 or later.
         const uint32_t idesc = umma_idesc(TOK);
         int a = 0, xst = 0;
         uint32_t aphase = 0;
@@ -430,6 +431,76 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             prev_t = -1;
             return true;
         };
+        // The last warpgroup of the chain also finishes the piece: with the sum of all five shares in registers it
+        // stores the rows at their original positions (fused un-permutation), parks the sum, or adds the parked sums
+        // of other CTAs.
+        uint32_t esync_phase = 0;
+        const int et = twg;
+        auto finalize = [&](int q, float (&acc)[TOK]) -> bool {
+            const Tile ti(s_tile[s_piece[q]]);       // the piece's last tile carries its facts
+            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows, N = s_ex[ti.e].N;
+            uint16_t* Y = p.Y[ti.e];
+            if (ti.flags & TF_WHOLE) {
+                // the whole K of this segment was ours: round and store rows at their original positions
+                if (n < N) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m)
+                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                }
+            } else if (ti.flags & TF_KB0NZ) {
+                // A piece that starts inside its segment -- always a CTA's FIRST piece, so it is ready early in the
+                // kernel: park the partial sum and raise this CTA's flag.  Nobody waits here.
+                float* dst = p.partials + (size_t)blockIdx.x * TOK * 128 + row;
+#pragma unroll
+                for (int m = 0; m < TOK; ++m)
+                    if (m < rows) dst[m * 128] = acc[m];
+                __threadfence();
+                mbar_arrive(bar_esync);
+                if (!wwait(bar_esync, esync_phase)) return false;
+                esync_phase ^= 1u;
+                if (et == 0) {
+                    __threadfence();
+                    atomicExch(p.flags + blockIdx.x, 1u);
+                }
+            } else {
+                // The head of a segment whose tail belongs to the following CTAs -- always a CTA's LAST piece, while
+                // the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as its first piece).
+                // Wait for their flags (bounded), add their sums in CTA order (deterministic), store.
+                const int n_others = ti.c_last - (int)blockIdx.x;
+                for (int i = et; i < n_others; i += 128) {
+                    volatile unsigned* f = p.flags + blockIdx.x + 1 + i;
+                    unsigned long long t_start = 0;
+                    for (unsigned it = 1; *f == 0u; ++it) {
+                        if ((it & 63u) == 0) {
+                            if (*s_abort) break;
+                            const unsigned long long now = global_ns();
+                            if (t_start == 0) t_start = now;
+                            else if (now - t_start > WAIT_LIMIT_NS) { *s_abort = 1; latch_status(p.status, (int)MOQE_ERR_TIMEOUT); break; }
+                        }
+                    }
+                }
+                __threadfence();
+                mbar_arrive(bar_esync);
+                if (!wwait(bar_esync, esync_phase)) return false;
+                esync_phase ^= 1u;
+                if (*s_abort) return false;
+                for (int c0 = 0; c0 < n_others; ++c0) {
+                    const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0) * TOK * 128 + row;
+                    float part[TOK];
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m) part[m] = m < rows ? __ldcg(src + m * 128) : 0.f;
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m) acc[m] += part[m];
+                }
+                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
+                if (n < N) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m)
+                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                }
+            }
+            return true;
+        };
         // Pieces before `upto` are complete as far as this warpgroup goes: add its share to the piece's sum in
         // shared memory, warpgroup 0 first (it writes), then 1, 2, 3 (they add) -- a fixed order, so the result does
         // not depend on timing -- and pass the turn on; the finalizer takes the sum after warpgroup 3.
@@ -439,30 +510,38 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 if (wg == 0) { if (!wwait(bar_flushfree, par ^ 1u)) return false; }
                 else if (!wwait(bar_turn + 8 * (wg - 1), par)) return false;
                 const bool mine = prev_piece == flushed;
-                if (wg == 0) {
+                if (wg == NWG - 1) {
+                    float total[TOK];
 #pragma unroll
-                    for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] = mine ? acc[m] : 0.f;
-                } else if (mine) {
+                    for (int m = 0; m < TOK; ++m) total[m] = s_out[m * 128 + row] + (mine ? acc[m] : 0.f);
+                    warrive(bar_flushfree);
+                    if (!finalize(flushed, total)) return false;
+                } else {
+                    if (wg == 0) {
 #pragma unroll
-                    for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] += acc[m];
+                        for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] = mine ? acc[m] : 0.f;
+                    } else if (mine) {
+#pragma unroll
+                        for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] += acc[m];
+                    }
+                    warrive(bar_turn + 8 * wg);
                 }
                 if (mine) {
 #pragma unroll
                     for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
                 }
-                warrive(bar_turn + 8 * wg);
             }
             return true;
         };
         x_load(wg);
         int stg = wg % nstg, a = wg;                 // ring stage and A buffer of tile t, kept incrementally
         uint32_t wphase = (uint32_t)(wg / nstg) & 1u;
-        for (int t = wg; ok && t < T; t += 4) {
+        for (int t = wg; ok && t < T; t += NWG) {
             const Tile ti(s_tile[t]);
             const ExpertSm& ex = s_ex[ti.e];
-            // tile t - 6 is done: A buffer t % 6 and token-tile stage (t + 4) % 10 are free
+            // tile t - 6 is done (and so are all before it): A buffer t % 6 and token-tile stage (t + 5) % 12 are free
             if (!(ok = wait_done(t - NA))) break;
-            x_load(t + 4);
+            x_load(t + NWG);
             if (!(ok = drain_prev())) break;
             if (!(ok = flush_to(ti.piece))) break;
             if (!(ok = wwait(bar_wfull + 8 * stg, wphase))) break;
@@ -492,94 +571,13 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             tmem_st_wait();
             tc_fence_before();
             warrive(bar_afull + 8 * a);
-            stg += 4;
+            stg += NWG;
             while (stg >= nstg) { stg -= nstg; wphase ^= 1u; }
-            a = a + 4 >= NA ? a + 4 - NA : a + 4;
+            a = a + NWG >= NA ? a + NWG - NA : a + NWG;
         }
         if (ok) ok = drain_prev();
         if (ok) flush_to(NP);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
-    } else if (warp >= EP_WARP0 && warp < EP_WARP0 + 4) {
-        // ------------------------------------------------------------------ finalizer warpgroup
-        // Takes each piece's sum once the four dequant warpgroups have added their shares, then stores the rows at
-        // their original positions (fused un-permutation), parks the sum, or adds the parked sums of other CTAs.
-        const int et = tid - EP_WARP0 * 32, row = (warp & 3) * 32 + lane;
-        uint32_t esync_phase = 0;
-        bool ok = true;
-        for (int q = 0; ok && q < NP; ++q) {
-            const Tile ti(s_tile[s_piece[q]]);       // the piece's last tile carries its facts
-            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows, N = s_ex[ti.e].N;
-            uint16_t* Y = p.Y[ti.e];
-            if (!(ok = wwait(bar_turn + 8 * 3, (uint32_t)q & 1u))) break;
-            float acc[TOK];
-#pragma unroll
-            for (int m = 0; m < TOK; ++m) acc[m] = s_out[m * 128 + row];
-            warrive(bar_flushfree);
-            if (ti.flags & TF_WHOLE) {
-                // the whole K of this segment was ours: round and store rows at their original positions
-                if (n < N) {
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m)
-                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
-                }
-            } else if (ti.flags & TF_KB0NZ) {
-                // A piece that starts inside its segment -- always a CTA's FIRST piece, so it is ready early in the
-                // kernel: park the partial sum and raise this CTA's flag.  Nobody waits here.
-                float* dst = p.partials + (size_t)blockIdx.x * TOK * 128 + row;
-#pragma unroll
-                for (int m = 0; m < TOK; ++m)
-                    if (m < rows) dst[m * 128] = acc[m];
-                __threadfence();
-                mbar_arrive(bar_esync);
-                if (!(ok = wwait(bar_esync, esync_phase))) break;
-                esync_phase ^= 1u;
-                if (et == 0) {
-                    __threadfence();
-                    atomicExch(p.flags + blockIdx.x, 1u);
-                }
-            } else {
-                // The head of a segment whose tail belongs to the following CTAs -- always a CTA's LAST piece, while
-                // the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as its first piece).
-                // Wait for their flags (bounded), add their sums in CTA order (deterministic), store.
-                const int n_others = ti.c_last - (int)blockIdx.x;
-                for (int i = et; i < n_others; i += 128) {
-                    volatile unsigned* f = p.flags + blockIdx.x + 1 + i;
-                    unsigned long long t_start = 0;
-                    for (unsigned it = 1; *f == 0u; ++it) {
-                        if ((it & 63u) == 0) {
-                            if (*s_abort) break;
-                            const unsigned long long now = global_ns();
-                            if (t_start == 0) t_start = now;
-                            else if (now - t_start > WAIT_LIMIT_NS) { *s_abort = 1; latch_status(p.status, (int)MOQE_ERR_TIMEOUT); break; }
-                        }
-                    }
-                }
-                __threadfence();
-                mbar_arrive(bar_esync);
-                if (!(ok = wwait(bar_esync, esync_phase))) break;
-                esync_phase ^= 1u;
-                if (*s_abort) { ok = false; break; }
-                for (int c0 = 0; c0 < n_others; c0 += 2) {             // two contributors' loads in flight at a time
-                    float part[2][TOK];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0 + u) * TOK * 128 + row;
-#pragma unroll
-                        for (int m = 0; m < TOK; ++m) part[u][m] = (c0 + u < n_others && m < rows) ? __ldcg(src + m * 128) : 0.f;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u)
-#pragma unroll
-                        for (int m = 0; m < TOK; ++m) acc[m] += part[u][m];
-                }
-                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
-                if (n < N) {
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m)
-                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
-                }
-            }
-        }
     }
 
     // ---------------------------------------------------------------------- teardown
