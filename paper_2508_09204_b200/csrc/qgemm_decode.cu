@@ -52,9 +52,9 @@ namespace moqe {
 namespace {
 
 constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
-constexpr int NWG = 5;                                  // dequant warpgroups; warpgroup w takes tiles t = w (mod 5)
-constexpr int DQ_WARPS = 4 * NWG, MMA_WARP = 20, W_WARP = 21;
-constexpr int DEC_THREADS = 22 * 32;
+constexpr int NWG = 4;                                  // dequant warpgroups; warpgroup w takes tiles t = w (mod 4)
+constexpr int DQ_WARPS = 4 * NWG, MMA_WARP = DQ_WARPS, W_WARP = DQ_WARPS + 1;
+constexpr int DEC_THREADS = (DQ_WARPS + 2) * 32;
 constexpr int RING_BYTES = 142 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
@@ -64,6 +64,7 @@ constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
 constexpr int TMEM_COLS = 512;
 constexpr int D_COL0 = NA * 64;
+static_assert(NA > NWG && ND >= 2 * NWG && D_COL0 + ND * TOK <= TMEM_COLS, "buffers: a warpgroup must not wait for the previous round");
 constexpr int MAX_TILES = 512;                          // tiles one CTA can take (its tile table)
 
 struct DecSmem {
@@ -371,7 +372,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.  No accumulator
         // hand-shake is needed: buffer g % 8 is drained by the warpgroup that unpacked the group's last tile j before
-        // it hands over its next tile j + 5, and the group that reuses the buffer starts at tile j + 8 or later.
+        // it hands over its tile j + 8, and the group that reuses the buffer starts at tile j + 8 or later.
         const uint32_t idesc = umma_idesc(TOK);
         int a = 0, xst = 0;
         uint32_t aphase = 0;
@@ -414,24 +415,28 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
 #pragma unroll
         for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
         int flushed = 0;                             // pieces this warpgroup has handed to the finalizer
-        int prev_t = -1, prev_g = 0, prev_piece = -1;   // its previous tile, if that ended an accumulation group
-        float prev_s = 0.f;
+        // Accumulation groups that ended with this warpgroup's last two tiles and are not drained yet.  A group is
+        // drained TWO rounds after its last tile was handed over: one round later its MMAs may still be queued behind
+        // the other warpgroups' tiles, and waiting for them would put the MMA round trip into every round.
+        struct Rec { int t, g, piece; float s; };
+        Rec r0{-1, 0, 0, 0.f}, r1{-1, 0, 0, 0.f};    // two rounds back, previous round
+        int acc_piece = -1;                          // the piece `acc` belongs to
+        int last_t = -1, ph0 = 0, ph1 = 0;                        // pieces of this warpgroup's tiles of two rounds / one round ago
         bool ok = true;
-        // the group that ended with the warpgroup's previous tile: scale and add (its MMAs finished long ago)
-        auto drain_prev = [&]() -> bool {
-            if (prev_t < 0) return true;
-            if (!wait_done(prev_t)) return false;
+        // scale and add a finished group (the caller knows that its MMAs have completed)
+        auto drain = [&](Rec& r) {
+            if (r.t < 0) return;
             tc_fence_after();
             uint32_t v[16];
-            tmem_ld16(lane_taddr + D_COL0 + (prev_g & (ND - 1)) * TOK, v);
+            tmem_ld16(lane_taddr + D_COL0 + (r.g & (ND - 1)) * TOK, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < TOK; ++i) acc[i] = fmaf(prev_s, __uint_as_float(v[i]), acc[i]);
+            for (int i = 0; i < TOK; ++i) acc[i] = fmaf(r.s, __uint_as_float(v[i]), acc[i]);
             tc_fence_before();
-            prev_t = -1;
-            return true;
+            acc_piece = r.piece;
+            r.t = -1;
         };
-        // The last warpgroup of the chain also finishes the piece: with the sum of all five shares in registers it
+        // The last warpgroup of the chain also finishes the piece: with the sum of all four shares in registers it
         // stores the rows at their original positions (fused un-permutation), parks the sum, or adds the parked sums
         // of other CTAs.
         uint32_t esync_phase = 0;
@@ -509,7 +514,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                 const uint32_t par = (uint32_t)flushed & 1u;
                 if (wg == 0) { if (!wwait(bar_flushfree, par ^ 1u)) return false; }
                 else if (!wwait(bar_turn + 8 * (wg - 1), par)) return false;
-                const bool mine = prev_piece == flushed;
+                const bool mine = acc_piece == flushed;
                 if (wg == NWG - 1) {
                     float total[TOK];
 #pragma unroll
@@ -534,16 +539,24 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             return true;
         };
         x_load(wg);
-        int stg = wg % nstg, a = wg;                 // ring stage and A buffer of tile t, kept incrementally
+        int stg = wg % nstg, a = wg % NA;            // ring stage and A buffer of tile t, kept incrementally
         uint32_t wphase = (uint32_t)(wg / nstg) & 1u;
         for (int t = wg; ok && t < T; t += NWG) {
             const Tile ti(s_tile[t]);
             const ExpertSm& ex = s_ex[ti.e];
-            // tile t - 6 is done (and so are all before it): A buffer t % 6 and token-tile stage (t + 5) % 12 are free
+            // tile t - 6 is done, and so are all before it (MMAs are issued in tile order and a commit covers every
+            // earlier one): A buffer t % 6 and token-tile stage (t + 4) % 12 are free, and the group that ended two
+            // rounds ago (tile t - 8) can be drained without a wait of its own
+            // First of all the warpgroup takes its turn for the pieces before the one its tile of two rounds ago
+            // belongs to: all four warpgroups do this at the same distance behind their tiles and before they wait
+            // for anything else, so none of them can be waiting for a tile that another holds back while it waits
+            // for its turn.
+            if (!(ok = flush_to(ph0))) break;
             if (!(ok = wait_done(t - NA))) break;
             x_load(t + NWG);
-            if (!(ok = drain_prev())) break;
-            if (!(ok = flush_to(ti.piece))) break;
+            drain(r0);
+            r0 = r1;
+            r1.t = -1;
             if (!(ok = wwait(bar_wfull + 8 * stg, wphase))) break;
             tc_fence_after();
             const unsigned char* stage = smem + L::ring_off + stg * stage_bytes;
@@ -556,12 +569,12 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
             else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), lane_taddr + a * 64);
             else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
-            prev_piece = ti.piece;
             if (ti.ends()) {
-                // the scale of the group that ends with this tile; its accumulator is drained on the next round
-                prev_t = t;
-                prev_g = ti.g;
-                prev_s = (group == 0 ? __half2float(p.ex[ti.e].scales_pc[ti.nt * 128 + row])
+                // the scale of the group that ends with this tile; its accumulator is drained two rounds later
+                r1.t = t;
+                r1.g = ti.g;
+                r1.piece = ti.piece;
+                r1.s = (group == 0 ? __half2float(p.ex[ti.e].scales_pc[ti.nt * 128 + row])
                                      : __half2float(moqe_tile_scales(stage, bits, has_zeros, 0)[row])) *
                          (bits == 8 ? W8_PRESCALE : 1.f);
             }
@@ -571,12 +584,26 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             tmem_st_wait();
             tc_fence_before();
             warrive(bar_afull + 8 * a);
+            ph0 = ph1;
+            ph1 = ti.piece;
+            last_t = t;
             stg += NWG;
             while (stg >= nstg) { stg -= nstg; wphase ^= 1u; }
-            a = a + NWG >= NA ? a + NWG - NA : a + NWG;
+            a += NWG;
+            while (a >= NA) a -= NA;
         }
-        if (ok) ok = drain_prev();
-        if (ok) flush_to(NP);
+        if (ok) ok = flush_to(ph0);
+        // the MMAs of this warpgroup's last tile (hence of all earlier ones) -- not of an older tile: a barrier of the
+        // ring tells apart only tiles that are less than 8 apart
+        if (ok && last_t >= 0) ok = wait_done(last_t);
+        if (ok) {
+            drain(r0);
+            ok = flush_to(ph1);
+        }
+        if (ok) {
+            drain(r1);
+            flush_to(NP);
+        }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
 
