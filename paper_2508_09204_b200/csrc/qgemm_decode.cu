@@ -55,11 +55,11 @@ constexpr int TOK = 16;                                 // token columns of the 
 constexpr int NWG = 4;                                  // dequant warpgroups; warpgroup w takes tiles t = w (mod 4)
 constexpr int DQ_WARPS = 4 * NWG, MMA_WARP = DQ_WARPS, W_WARP = DQ_WARPS + 1;
 constexpr int DEC_THREADS = (DQ_WARPS + 2) * 32;
-constexpr int RING_BYTES = 142 * 1024;                  // packed-weight ring
+constexpr int RING_BYTES = 134 * 1024;                  // packed-weight ring
 constexpr int MAX_STAGES = 16;
 constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
 constexpr int ND = 8;                                   // accumulator buffers (TOK columns each), group g -> g % 8
-constexpr int NXS = 12;                                 // token-tile stages, tile t -> t % 12
+constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
 constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
 constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
 constexpr int TMEM_COLS = 512;
@@ -70,8 +70,8 @@ constexpr int MAX_TILES = 512;                          // tiles one CTA can tak
 struct DecSmem {
     static constexpr int ring_off = 0;
     static constexpr int x_off = RING_BYTES;
-    static constexpr int out_off = x_off + NXS * X_STAGE;             // float[TOK][128]: a piece's sum, warpgroup by warpgroup
-    static constexpr int bar_off = out_off + TOK * 512;
+    static constexpr int out_off = x_off + NXS * X_STAGE;             // float[NWG - 1][TOK][128]: a piece's shares
+    static constexpr int bar_off = out_off + (NWG - 1) * TOK * 512;
     // wfull[16] wempty[16] afull[NA] done[8] turn[4] flush_free esync
     static constexpr int n_bars = 2 * MAX_STAGES + NA + DONE_RING + 4 + 1 + 1;
     static constexpr int misc_off = bar_off + n_bars * 8;              // tmem address, abort flag, ring geometry
@@ -275,7 +275,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         for (int i = 0; i < MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, 4); }
         for (int i = 0; i < NA; ++i) mbar_init(bar_afull + 8 * i, 4);
         for (int i = 0; i < DONE_RING; ++i) mbar_init(bar_done + 8 * i, 1);
-        for (int i = 0; i < 4; ++i) mbar_init(bar_turn + 8 * i, 4);
+        mbar_init(bar_turn, DQ_WARPS);                  // every dequant warp, once per piece
         mbar_init(bar_flushfree, 4);
         mbar_init(bar_esync, 128);
         *s_abort = 0;
@@ -506,30 +506,33 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             }
             return true;
         };
-        // Pieces before `upto` are complete as far as this warpgroup goes: add its share to the piece's sum in
-        // shared memory, warpgroup 0 first (it writes), then 1, 2, 3 (they add) -- a fixed order, so the result does
-        // not depend on timing -- and pass the turn on; the finalizer takes the sum after warpgroup 3.
+        // Pieces before `upto` are complete as far as this warpgroup goes: hand its share over.
         auto flush_to = [&](int upto) -> bool {
             for (; flushed < upto; ++flushed) {
                 const uint32_t par = (uint32_t)flushed & 1u;
-                if (wg == 0) { if (!wwait(bar_flushfree, par ^ 1u)) return false; }
-                else if (!wwait(bar_turn + 8 * (wg - 1), par)) return false;
+                // every warpgroup has a slot of its own for its share, so none waits for another here -- only for the
+                // last warpgroup to have read the previous piece's slots
+                if (!wwait(bar_flushfree, par ^ 1u)) return false;
                 const bool mine = acc_piece == flushed;
+                float* slot = s_out + wg * (TOK * 128);
+                if (wg != NWG - 1) {
+#pragma unroll
+                    for (int m = 0; m < TOK; ++m) slot[m * 128 + row] = mine ? acc[m] : 0.f;
+                }
+                warrive(bar_turn);
                 if (wg == NWG - 1) {
+                    // the last warpgroup adds the shares in warpgroup order (deterministic) once all have arrived
+                    if (!wwait(bar_turn, par)) return false;
                     float total[TOK];
 #pragma unroll
-                    for (int m = 0; m < TOK; ++m) total[m] = s_out[m * 128 + row] + (mine ? acc[m] : 0.f);
+                    for (int m = 0; m < TOK; ++m) {
+                        float v = s_out[m * 128 + row];
+#pragma unroll
+                        for (int u = 1; u < NWG - 1; ++u) v += s_out[u * (TOK * 128) + m * 128 + row];
+                        total[m] = v + (mine ? acc[m] : 0.f);
+                    }
                     warrive(bar_flushfree);
                     if (!finalize(flushed, total)) return false;
-                } else {
-                    if (wg == 0) {
-#pragma unroll
-                        for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] = mine ? acc[m] : 0.f;
-                    } else if (mine) {
-#pragma unroll
-                        for (int m = 0; m < TOK; ++m) s_out[m * 128 + row] += acc[m];
-                    }
-                    warrive(bar_turn + 8 * wg);
                 }
                 if (mine) {
 #pragma unroll
@@ -545,7 +548,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
             const Tile ti(s_tile[t]);
             const ExpertSm& ex = s_ex[ti.e];
             // tile t - 6 is done, and so are all before it (MMAs are issued in tile order and a commit covers every
-            // earlier one): A buffer t % 6 and token-tile stage (t + 4) % 12 are free, and the group that ended two
+            // earlier one): A buffer t % 6 and token-tile stage (t + 4) % 10 are free, and the group that ended two
             // rounds ago (tile t - 8) can be drained without a wait of its own
             // First of all the warpgroup takes its turn for the pieces before the one its tile of two rounds ago
             // belongs to: all four warpgroups do this at the same distance behind their tiles and before they wait
