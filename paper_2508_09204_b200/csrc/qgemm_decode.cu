@@ -296,34 +296,49 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (tid == 0) {
-        // per-expert facts, the ring geometry (stage = the largest packed tile this CTA will see) and the tile count
-        int cum = 0, gbase = 0, wmax = 0, pbase = 0;
-        for (int e = 0; e < sch.E; ++e) {
-            ExpertSm x;
+    if (warp == 0) {
+        // Per-expert facts, the ring geometry (stage = the largest packed tile this CTA will see) and the tile count:
+        // lane e works out expert e (E <= 32), the running totals come from a warp scan -- one thread doing all
+        // experts in turn costs the better part of a microsecond at every launch.
+        const int e = lane;
+        ExpertSm x = {};
+        int cnt = 0, ng = 0, np = 0, str = 0;
+        if (e < sch.E) {
             x.row0 = s_off[p.rexp[e]];
             x.rows = min(s_off[p.rexp[e] + 1] - x.row0, TOK);
-            x.KB = p.KB[e]; x.N = p.N[e]; x.pad0 = x.pad1 = 0;
+            x.KB = p.KB[e]; x.N = p.N[e];
             x.tb = s_rng[2 * e];
             x.te = x.rows > 0 ? s_rng[2 * e + 1] : x.tb;
             x.bits = p.ex[e].bits; x.group = p.ex[e].group; x.has_zeros = p.ex[e].has_zeros; x.stride = p.ex[e].tile_stride;
             x.gkb = x.group == 0 ? x.KB : x.group / 128;
-            x.cum = cum;
-            x.gbase = gbase;
-            x.pbase = pbase;
             if (x.te > x.tb) {
-                cum += x.te - x.tb;
-                gbase += x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
-                pbase += (x.te - 1) / x.KB - x.tb / x.KB + 1;
-                wmax = max(wmax, x.stride);
+                cnt = x.te - x.tb;
+                ng = x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
+                np = (x.te - 1) / x.KB - x.tb / x.KB + 1;
+                str = x.stride;
             }
+        }
+        int c = cnt, g = ng, q = np, wmax = str;            // inclusive scans / maximum over the lanes
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int c2 = __shfl_up_sync(0xffffffffu, c, d), g2 = __shfl_up_sync(0xffffffffu, g, d),
+                      q2 = __shfl_up_sync(0xffffffffu, q, d);
+            if (lane >= d) { c += c2; g += g2; q += q2; }
+            wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, d));
+        }
+        if (e < sch.E) {
+            x.cum = c - cnt;
+            x.gbase = g - ng;
+            x.pbase = q - np;
             s_ex[e] = x;
         }
-        const int stage_bytes = (max(wmax, 128) + 127) & ~127;
-        s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
-        s_geom[1] = stage_bytes;
-        s_geom[2] = min(cum, MAX_TILES);
-        s_geom[3] = pbase;
+        if (lane == 31) {
+            const int stage_bytes = (max(wmax, 128) + 127) & ~127;
+            s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
+            s_geom[1] = stage_bytes;
+            s_geom[2] = min(c, MAX_TILES);
+            s_geom[3] = q;
+        }
     }
     __syncthreads();
     const uint32_t tmem_base = *s_tmem;
