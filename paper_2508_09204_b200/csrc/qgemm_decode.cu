@@ -78,8 +78,7 @@ struct DecSmem {
     static constexpr int off_off = misc_off + 32;
     static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;   // perm of the batch's rows
     static constexpr int rng_off = perm_off + TOK * 4;
-    static constexpr int red_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // reduction verdicts
-    static constexpr int ex_off = red_off + 32;                        // ExpertSm[MOQE_MAX_EXPERTS]
+    static constexpr int ex_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // ExpertSm[MOQE_MAX_EXPERTS]
     static constexpr int tile_off = (ex_off + MOQE_MAX_EXPERTS * 64 + 15) & ~15;   // uint4[MAX_TILES]
     static constexpr int piece_off = tile_off + MAX_TILES * 16;        // int[MAX_TILES]: last tile of each piece
     static constexpr int total = piece_off + MAX_TILES * 4;
@@ -250,7 +249,6 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
     volatile int* s_off = reinterpret_cast<volatile int*>(smem + L::off_off);
     volatile int* s_rng = reinterpret_cast<volatile int*>(smem + L::rng_off);
     volatile int* s_perm = reinterpret_cast<volatile int*>(smem + L::perm_off);
-    volatile int* s_red = reinterpret_cast<volatile int*>(smem + L::red_off);
     ExpertSm* s_ex = reinterpret_cast<ExpertSm*>(smem + L::ex_off);
     const uint4* s_tile = reinterpret_cast<const uint4*>(smem + L::tile_off);
     float* s_out = reinterpret_cast<float*>(smem + L::out_off);

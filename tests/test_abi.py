@@ -70,6 +70,13 @@ def test_host_side_argument_checks(moqe):
     assert L.moqe_routed_qgemm(fake, fake, 4, arr, 1, fake, fake, 0, None) == moqe.ERR_NULL
     assert L.moqe_routed_qgemm(fake, fake, 4, arr, 0, fake, fake, 0, None) == moqe.ERR_SHAPE
     assert L.moqe_expert_destroy(None) == moqe.ERR_NULL
+    # several layers in one launch: argument checks come before any device work
+    xs, ys = (C.c_void_p * 2)(0x1000, 0x2000), (C.c_void_p * 2)(0x3000, 0x4000)
+    assert L.moqe_routed_qgemm_sorted_multi(xs, fake, fake, 4, 2, None, 1, ys, fake, 0, None) == moqe.ERR_NULL
+    assert L.moqe_routed_qgemm_sorted_multi(xs, fake, fake, 4, 0, arr, 1, ys, fake, 0, None) == moqe.ERR_SHAPE
+    assert L.moqe_routed_qgemm_sorted_multi(xs, fake, fake, 4, 17, arr, 2, ys, fake, 0, None) == moqe.ERR_UNSUPPORTED
+    assert L.moqe_routed_qgemm_sorted_multi(xs, fake, fake, 4, 1, arr, 1, ys, fake, 0, None) == moqe.ERR_NULL
+    assert L.moqe_routed_qgemm_path(fake, fake, 4, arr, 1, fake, fake, 0, None, 6) == moqe.ERR_NULL
 
 
 def test_workspace_sizes(moqe):
