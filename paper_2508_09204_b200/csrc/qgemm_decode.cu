@@ -153,8 +153,6 @@ struct Tile {
     __device__ __forceinline__ explicit Tile(const uint4& v)
         : kb((int)(v.x & 0xFFFFu)), nt((int)(v.x >> 16)), flags((int)(v.y & 0xFFu)), e((int)((v.y >> 8) & 0xFFu)),
           rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z), piece((int)(v.w & 0xFFFFu)), c_last((int)(v.w >> 16)) {}
-    __device__ __forceinline__ bool first() const { return flags & TF_FIRST; }
-    __device__ __forceinline__ bool last() const { return flags & TF_LAST; }
     __device__ __forceinline__ bool ends() const { return flags & TF_ENDS; }
 };
 
