@@ -37,6 +37,18 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
+// A flag in global memory that one CTA raises and another polls.  The release orders every write that happens
+// before it -- the raising thread's own and, through a CTA barrier, those of the threads that arrived there before it
+// -- ahead of the flag; a thread that reads the flag with the acquire load sees them all afterwards.
+__device__ __forceinline__ void st_release_gpu(unsigned* p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // try_wait with a suspend-time hint parks the thread in hardware until the phase completes or the hint (1 ms)
 // has passed, so a waiting warp does not compete for issue slots; without the hint the wait returns after a short
 // system-defined time and a waiting warp spins, which costs the working warps of the same scheduler their slots.

@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         for (int i = 0; i < DONE_RING; ++i) mbar_init(bar_done + 8 * i, 1);
         mbar_init(bar_turn, DQ_WARPS);                  // every dequant warp, once per piece
         mbar_init(bar_flushfree, 4);
-        mbar_init(bar_esync, 128);
+        mbar_init(bar_esync, 4);                         // the four warps of the finalizing warpgroup
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -464,29 +464,27 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                         if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
                 }
             } else if (ti.flags & TF_KB0NZ) {
-                // A piece that starts inside its segment -- always a CTA's FIRST piece, so it is ready early in the
-                // kernel: park the partial sum and raise this CTA's flag.  Nobody waits here.
+                // A piece that starts inside its segment -- always a CTA's FIRST piece: park the partial sum and raise
+                // this CTA's flag.  Nobody waits here: the barrier puts the 128 threads' stores before thread 0's
+                // release, which publishes them together with the flag.
                 float* dst = p.partials + (size_t)blockIdx.x * TOK * 128 + row;
 #pragma unroll
                 for (int m = 0; m < TOK; ++m)
                     if (m < rows) dst[m * 128] = acc[m];
-                __threadfence();
-                mbar_arrive(bar_esync);
+                warrive(bar_esync);
                 if (!wwait(bar_esync, esync_phase)) return false;
                 esync_phase ^= 1u;
-                if (et == 0) {
-                    __threadfence();
-                    atomicExch(p.flags + blockIdx.x, 1u);
-                }
+                if (et == 0) st_release_gpu(p.flags + blockIdx.x, 1u);
             } else {
                 // The head of a segment whose tail belongs to the following CTAs -- always a CTA's LAST piece, while
-                // the later pieces were parked long ago by CTAs blockIdx.x + 1 .. c_last (each as its first piece).
-                // Wait for their flags (bounded), add their sums in CTA order (deterministic), store.
+                // the later pieces are parked by CTAs blockIdx.x + 1 .. c_last (each as its first piece).  Every thread
+                // waits for their flags itself (bounded; an acquire load, so its reads of the parked sums need no
+                // further fence), adds the sums in CTA order (deterministic) and stores.
                 const int n_others = ti.c_last - (int)blockIdx.x;
-                for (int i = et; i < n_others; i += 128) {
-                    volatile unsigned* f = p.flags + blockIdx.x + 1 + i;
+                for (int c0 = 0; c0 < n_others; ++c0) {
+                    const unsigned* f = p.flags + blockIdx.x + 1 + c0;
                     unsigned long long t_start = 0;
-                    for (unsigned it = 1; *f == 0u; ++it) {
+                    for (unsigned it = 1; ld_acquire_gpu(f) == 0u; ++it) {
                         if ((it & 63u) == 0) {
                             if (*s_abort) break;
                             const unsigned long long now = global_ns();
@@ -494,13 +492,6 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
                             else if (now - t_start > WAIT_LIMIT_NS) { *s_abort = 1; latch_status(p.status, (int)MOQE_ERR_TIMEOUT); break; }
                         }
                     }
-                }
-                __threadfence();
-                mbar_arrive(bar_esync);
-                if (!wwait(bar_esync, esync_phase)) return false;
-                esync_phase ^= 1u;
-                if (*s_abort) return false;
-                for (int c0 = 0; c0 < n_others; ++c0) {
                     const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0) * TOK * 128 + row;
                     float part[TOK];
 #pragma unroll
@@ -508,7 +499,12 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
 #pragma unroll
                     for (int m = 0; m < TOK; ++m) acc[m] += part[m];
                 }
-                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;   // clear for the next call
+                // all 128 threads have seen the flags before any of them is cleared for the next call
+                warrive(bar_esync);
+                if (!wwait(bar_esync, esync_phase)) return false;
+                esync_phase ^= 1u;
+                if (*s_abort) return false;
+                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;
                 if (n < N) {
 #pragma unroll
                     for (int m = 0; m < TOK; ++m)
