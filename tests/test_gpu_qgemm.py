@@ -75,11 +75,12 @@ DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True)
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (13, 136, 2304), (16, 1000, 640),
-                                   (7, 4096, 1024), (16, 512, 11008)])
+                                   (7, 4096, 1024), (16, 512, 11008), (9, 128, 32768)])
 def test_decode_kernel_all_formats(M, N, K):
     """The tcgen05 decode kernel (path 5: at most 16 rows, per-channel experts or groups of >= 128 k): every such
-    format as its own expert, ragged N, K not a multiple of 128, split K with several contributors per segment,
-    an expert that gets no rows."""
+    format as its own expert, ragged N, K not a multiple of 128, split K with several contributors per segment
+    (dozens in the last, one-tile-wide case, where most CTAs hold nothing but the middle of a segment), an expert
+    that gets no rows."""
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, assert_close
     specs = [f for f in DECODE_FORMATS if f[1] == 0 or K % f[1] == 0]
