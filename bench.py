@@ -41,7 +41,7 @@ UNIT = "tokens/s"
 # None = no capture of the current kernel.
 TRAFFIC_RATIO = {
     "llama7b_decode": 32.748 / 32.513,      # o_proj launch: 32.75 MB read + 0 written (outputs stay in L2) vs 32.51 MB algorithmic
-    "llama7b_prefill": 267.12 / 300.95,     # 158.4 MB read + 108.7 MB written (part of Y still in L2) vs 300.9 MB
+    "llama7b_prefill": 267.81 / 300.95,     # 158.3 MB read + 109.5 MB written (part of Y still in L2) vs 300.9 MB
 }
 
 
