@@ -368,14 +368,15 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __gr
         // ------------------------------------------------------------------ packed-weight producer
         if (lane == 0) {
             Ring ring;
+            const uint64_t once = l2_policy_evict_first();   // weights cross L2 once per call
             for (int t = 0; t < T; ++t) {
                 const Tile ti(s_tile[t]);
                 const uint32_t wbytes = (uint32_t)s_ex[ti.e].stride;
                 if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) break;
                 const uint32_t full = bar_wfull + 8 * ring.stage;
                 mbar_expect_tx(full, wbytes);
-                bulk_load(sbase + L::ring_off + ring.stage * stage_bytes,
-                          p.ex[ti.e].tiles + ((size_t)ti.nt * s_ex[ti.e].KB + ti.kb) * wbytes, wbytes, full);
+                bulk_load_once(sbase + L::ring_off + ring.stage * stage_bytes,
+                               p.ex[ti.e].tiles + ((size_t)ti.nt * s_ex[ti.e].KB + ti.kb) * wbytes, wbytes, full, once);
                 ring.advance(nstg);
             }
         }
