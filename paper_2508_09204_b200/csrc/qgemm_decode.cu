@@ -4,6 +4,7 @@
 //   producer (1 thread)     : cp.async.bulk copies of whole packed 128x128-code tiles (codes + the
 //                             tile's scales / zero-points, contiguous in HBM) into a shared-memory
 //                             ring guarded by full/empty mbarriers.
+//                             The copies carry an L2 evict-first policy: weights pass through L2 once.
 //   dequant (4 warpgroups)  : warpgroup w takes the CTA's tiles t = w (mod 4).  Thread r of a
 //                             warpgroup owns channel row r of the tile: it reads the row's packed
 //                             words with conflict-free 128-bit shared loads, unpacks them in registers
