@@ -129,6 +129,15 @@ moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const
                                       size_t ws_bytes, cudaStream_t st);
 void decode_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split; 0 = its bytes
 
+// qgemm_gemv.cu: the same decode shapes on warp-level MMAs, weights streamed by lane-private asynchronous copies
+bool gemv_supported_multi(int M, const moqe_expert* const* ex, int nl, int E);
+size_t gemv_workspace_bytes(int M);
+size_t gemv_zero_bytes(int M);
+moqe_status launch_qgemm_gemv_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
+                                    void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
+                                    size_t ws_bytes, cudaStream_t st);
+void gemv_set_tile_cost(int bits, int cost);
+
 // qgemm_tcgen05.cu
 void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)
 size_t tc_workspace_bytes(int M, int K, int E, int Np);

@@ -1,0 +1,709 @@
+// Routed dequant-GEMV for decode shapes (at most 16 token rows in the batch): every touched
+// expert's packed weights are streamed from HBM exactly once.
+//
+//   producer (1 thread)   : one bulk copy per packed 128x128-code tile (codes + the tile's scales / zero-points,
+//                           contiguous in HBM) into a shared-memory ring guarded by full/empty mbarriers.  A stage
+//                           holds a "super-tile": the tiles (nt, nt + 1) of one k-block.  The copies carry an L2
+//                           evict-first policy: weights pass through L2 once.
+//   16 consumer warps     : warp w owns one 16-channel blob of the super-tile.  A lane reads the codes of channel
+//                           rows g and g + 8, k quarter t (its share of an m16n8k16 A fragment) with conflict-free
+//                           128-bit shared loads, unpacks them in registers and issues warp-level tensor-core MMAs
+//                           (fp16 operands, fp32 accumulation) against the token fragments; it applies the group's
+//                           scale in fp32 once per k-block and keeps the running sums of its piece in registers.
+//   4 service warps       : stage the token rows one chunk of k-blocks ahead, double buffered: gathered through
+//                           `perm` (the fused permutation), converted from bf16 to scaled fp16 in MMA fragment order,
+//                           with their sums.  Chunk descriptors travel with the buffers, so the consumers follow the
+//                           work split without walking it themselves.
+//
+//   Unpacking costs 5 integer instructions per 8 four-bit codes (1 per 2 eight-bit codes, 23 per 32 three-bit
+//   codes): a masked code dropped into the mantissa of the fp16 number 1024 becomes 1024 + c, or 1024 + 16c
+//   for a code that sits four bits higher -- no shift, no subtraction.  The tensor core multiplies by token
+//   values that were pre-scaled by 1/16 at exactly those k, and what the constants 1024 and the zero-point
+//   contribute is removed in fp32 with per-(token, k-block) sums of the token values:
+//     Y[m][n] = sum_G s[n][G] * ( sum_{k in G} A[n][k] * B[m][k]  -  1024 * S1[m][G]  -  z[n][G] * S0[m][G] )
+//   A = 1024 + c / sigma_k,  B = sigma_k * x,  S1 = sum sigma_k x,  S0 = sum x.  All products are exact
+//   (11-bit x 8-bit significands).  bf16 token values beyond the fp16 range (|x| > 65504) are outside the
+//   kernel's domain: they turn into infinities.
+//
+// Work split ("stream-K" over super-tiles): the super-tiles of every (layer, expert) pair whose expert received
+// rows form one sequence [pair][channel-tile pair][k-block] with a per-format cost; CTA c of G owns the
+// super-tiles whose start cost lies in [c*C/G, (c+1)*C/G) -- the split follows the routing, so an expert
+// without rows costs nothing and a batch routed to one expert still uses every SM.  A warp that holds only
+// part of a segment parks its fp32 partial sums and bumps its arrival counter for that segment; whoever
+// arrives last adds the parked sums in CTA order (deterministic) and stores bf16 rows at their original
+// positions (the fused un-permutation).  Nobody waits for another CTA, so the kernel cannot stall whatever
+// else occupies the device.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, latches MOQE_ERR_TIMEOUT, and
+// every role leaves its loop.
+//
+// The operation is Section 3.1 of the paper (the selected quantization expert runs the sample); the paper
+// describes no kernel.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace moqe {
+namespace {
+
+constexpr int GV_CONS = 16;                                    // consumer warps
+constexpr int GV_SERV = 2;                                     // service warps
+constexpr int GV_THREADS = (GV_CONS + GV_SERV + 1) * 32;       // + the producer's warp
+constexpr int GV_MAX_STAGES = 12;
+constexpr int GV_RING_BYTES = 158 * 1024;
+constexpr int GV_XBUF = 32 * 1024;                             // one chunk of staged token rows
+constexpr int GV_CHUNK_KB = 16;                                // k-blocks per chunk for one token block (8 for two)
+constexpr int GV_SBUF = GV_CHUNK_KB * 8 * 2 * 4;               // the chunk's sums: [k-block][token block][t][4] floats
+constexpr int GV_SLOT_FLOATS = GV_CONS * 2 * 4 * 32;           // a parked partial sum: 256 channels x 16 tokens
+constexpr int GV_MAX_GRID = 256;
+
+struct GvSmem {
+    static constexpr int ring_off = 0;
+    static constexpr int x_off = GV_RING_BYTES;
+    static constexpr int s_off = x_off + 2 * GV_XBUF;
+    static constexpr int desc_off = s_off + 2 * GV_SBUF;                  // 2 chunk descriptors of 32 bytes
+    static constexpr int bar_off = desc_off + 2 * 32;                     // wfull[12] wempty[12] xfull[2] xempty[2]
+    static constexpr int off_off = bar_off + (2 * GV_MAX_STAGES + 4) * 8;
+    static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;
+    static constexpr int pair_off = perm_off + 16 * 4;                    // {tb, te} per pair
+    static constexpr int base_off = pair_off + MOQE_MAX_EXPERTS * 8;     // cost before each pair (long long)
+    static constexpr int misc_off = base_off + MOQE_MAX_EXPERTS * 8;     // C (long long), G, stages, stage bytes, abort
+    static constexpr int total = misc_off + 32;
+    static constexpr int dyn_bytes = total;
+};
+static_assert(GvSmem::dyn_bytes <= 227 * 1024, "shared memory budget");
+
+struct GvParams {
+    ExpertDev ex[MOQE_MAX_EXPERTS];         // per (layer, expert) pair
+    const uint16_t* X[MOQE_MAX_EXPERTS];    // the layer's input and output
+    uint16_t* Y[MOQE_MAX_EXPERTS];
+    int N[MOQE_MAX_EXPERTS], K[MOQE_MAX_EXPERTS], KB[MOQE_MAX_EXPERTS];
+    int NT1[MOQE_MAX_EXPERTS];              // 128-channel tiles of the layer
+    int rexp[MOQE_MAX_EXPERTS];             // the routing expert whose rows the pair takes
+    int w[MOQE_MAX_EXPERTS];                // cost of one super-tile
+    const int32_t* perm;
+    const int32_t* offsets;
+    float* partials;                        // [CTA][2][GV_SLOT_FLOATS]
+    uint32_t* counters;                     // [CTA][warp]: arrivals for the segment whose head that CTA holds; zero on entry, left zero
+    int* status;
+    int M, R, P;                            // rows of the batch, routing experts, pairs
+};
+
+// one chunk of work: k-blocks [kbc, kbc + nkb) of segment (pair v, channel-tile pair nt2), part of the piece [kb0, kb1)
+struct ChunkDesc { int v, nt2, kbc, nkb, kb0, kb1, valid, pad; };
+
+// a walk over the CTA's super-tiles in [pair][channel-tile pair][k-block] order, run by run (a run = the k-blocks of
+// one piece: contiguous in HBM)
+struct GvWalk {
+    int v, st, te, kb, KB, nt2;
+    __device__ __forceinline__ void start() { v = -1; st = te = kb = nt2 = 0; KB = 1; }
+    // opens the next run; returns false at the end.  `changed`: the run belongs to another pair than the last one
+    __device__ __forceinline__ bool next(const int* s_pair, const GvParams& p, bool& changed) {
+        changed = false;
+        if (v >= 0) st += run();
+        if (v < 0 || st >= te) {
+            do { ++v; } while (v < p.P && s_pair[2 * v + 1] <= s_pair[2 * v]);
+            if (v >= p.P) return false;
+            st = s_pair[2 * v]; te = s_pair[2 * v + 1]; KB = p.KB[v];
+            nt2 = st / KB; kb = st - nt2 * KB;
+            changed = true;
+        } else {
+            kb = 0; ++nt2;
+        }
+        return true;
+    }
+    __device__ __forceinline__ int run() const { return min(KB - kb, te - st); }
+};
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// (v & mask) | 0x6400 in both halves: the fp16 numbers 1024 + (field value), for a field inside the mantissa
+__device__ __forceinline__ uint32_t field_f16(uint32_t v, uint32_t mask) { return (v & mask) | 0x64006400u; }
+
+// pairs 0..3 of one 4-bit word (8 consecutive k): {1024 + c, 1024 + 16c, 1024 + c, 1024 + 16c}
+__device__ __forceinline__ void unpack_w4(uint32_t v, uint32_t (&o)[4]) {
+    o[0] = field_f16(v, 0x000F000Fu);
+    o[1] = field_f16(v, 0x00F000F0u);
+    const uint32_t u = v >> 8;
+    o[2] = field_f16(u, 0x000F000Fu);
+    o[3] = field_f16(u, 0x00F000F0u);
+}
+// pairs 0..3 of an 8-bit chunk held in two words: 1024 + c
+__device__ __forceinline__ void unpack_w8(uint32_t w0, uint32_t w1, uint32_t (&o)[4]) {
+    o[0] = __byte_perm(w0, 0x64646464u, 0x4140u);
+    o[1] = __byte_perm(w0, 0x64646464u, 0x4342u);
+    o[2] = __byte_perm(w1, 0x64646464u, 0x4140u);
+    o[3] = __byte_perm(w1, 0x64646464u, 0x4342u);
+}
+// the 16 pairs of a 3-bit piece (words A, B, C): pair p < 15 is field p % 5 of word p / 5 -> 1024 + {1, 8, 64, 1, 8} * c;
+// pair 15 is spread over bit 15 / 31 of the three words -> 1024 + 64c
+__device__ __forceinline__ void unpack_w3(uint32_t A, uint32_t B, uint32_t C, uint32_t (&o)[16]) {
+    const uint32_t w[3] = {A, B, C};
+    uint32_t s0 = 0;
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        const uint32_t u = w[i] >> 9;
+        if (i == 0) s0 = u;
+        o[5 * i + 0] = field_f16(w[i], 0x00070007u);
+        o[5 * i + 1] = field_f16(w[i], 0x00380038u);
+        o[5 * i + 2] = field_f16(w[i], 0x01C001C0u);
+        o[5 * i + 3] = field_f16(u, 0x00070007u);
+        o[5 * i + 4] = field_f16(u, 0x00380038u);
+    }
+    uint32_t r = field_f16(s0, 0x00400040u);            // bit 15 / 31 of A -> bit 6 / 22: 64 * (code bit 0)
+    r |= (B >> 8) & 0x00800080u;                        // of B -> bit 7 / 23
+    r |= (C >> 7) & 0x01000100u;                        // of C -> bit 8 / 24
+    o[15] = r;
+}
+// log2 of 1 / sigma for pair p (0..15) of a piece: how far the code sits above the mantissa's unit
+__device__ __forceinline__ int sigma_shift(int bits, int p) {
+    if (bits == 8) return 0;
+    if (bits == 4) return (p & 1) ? 4 : 0;
+    return p == 15 ? 6 : 3 * ((p % 5) % 3);
+}
+
+template <int BITS, int NT, bool GROUPED, bool ASYM>
+struct GvTag {
+    static constexpr int bits = BITS, nt = NT;
+    static constexpr bool grouped = GROUPED, asym = ASYM;
+};
+
+// The MMAs of one tile for one lane: `blob` is the shared-memory address of the warp's blob, `xb` that of the
+// lane's token fragments of this k-block.
+template <int BITS, int NT>
+__device__ __forceinline__ void tile_mma(uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
+    uint4 b[NT][4];
+#pragma unroll
+    for (int G = 0; G < 4; ++G)
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) b[tb][G] = lds128(xb + ((tb * 4 + G) << 9));
+    if constexpr (BITS == 4) {
+        const uint4 w0 = lds128(blob + slot16), w1 = lds128(blob + 512 + slot16);
+        const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+        for (int G = 0; G < 4; ++G) {
+            uint32_t ar[4], a8[4];
+            unpack_w4(a0[G], ar);
+            unpack_w4(a1[G], a8);
+#pragma unroll
+            for (int tb = 0; tb < NT; ++tb) {
+                mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][G].x, b[tb][G].y);
+                mma_f16(acc[tb], ar[2], a8[2], ar[3], a8[3], b[tb][G].z, b[tb][G].w);
+            }
+        }
+    } else if constexpr (BITS == 8) {
+        // 512-byte blocks of the blob: {row g: chunks 0,1}, {row g: chunks 2,3}, {row g + 8: chunks 0,1}, {row g + 8: chunks 2,3}
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint4 w0 = lds128(blob + u * 512 + slot16), w1 = lds128(blob + 1024 + u * 512 + slot16);
+            const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg) {
+                uint32_t ar[4], a8[4];
+                unpack_w8(a0[2 * gg], a0[2 * gg + 1], ar);
+                unpack_w8(a1[2 * gg], a1[2 * gg + 1], a8);
+#pragma unroll
+                for (int tb = 0; tb < NT; ++tb) {
+                    mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][2 * u + gg].x, b[tb][2 * u + gg].y);
+                    mma_f16(acc[tb], ar[2], a8[2], ar[3], a8[3], b[tb][2 * u + gg].z, b[tb][2 * u + gg].w);
+                }
+            }
+        }
+    } else {
+        const uint4 w0 = lds128(blob + slot16);
+        const uint2 w1 = lds64(blob + 512 + (slot16 >> 1));
+        uint32_t ar[16], a8[16];
+        unpack_w3(w0.x, w0.y, w0.z, ar);
+        unpack_w3(w0.w, w1.x, w1.y, a8);
+#pragma unroll
+        for (int G = 0; G < 4; ++G) {
+#pragma unroll
+            for (int tb = 0; tb < NT; ++tb) {
+                mma_f16(acc[tb], ar[4 * G], a8[4 * G], ar[4 * G + 1], a8[4 * G + 1], b[tb][G].x, b[tb][G].y);
+                mma_f16(acc[tb], ar[4 * G + 2], a8[4 * G + 2], ar[4 * G + 3], a8[4 * G + 3], b[tb][G].z, b[tb][G].w);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_constant__ GvParams p) {
+    using L = GvSmem;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_wfull = sbase + L::bar_off, bar_wempty = bar_wfull + 8 * GV_MAX_STAGES;
+    const uint32_t bar_xfull = bar_wempty + 8 * GV_MAX_STAGES, bar_xempty = bar_xfull + 16;
+    int* s_off = reinterpret_cast<int*>(smem + L::off_off);
+    int* s_perm = reinterpret_cast<int*>(smem + L::perm_off);
+    int* s_pair = reinterpret_cast<int*>(smem + L::pair_off);
+    long long* s_base = reinterpret_cast<long long*>(smem + L::base_off);
+    long long* s_C = reinterpret_cast<long long*>(smem + L::misc_off);
+    int* s_G = reinterpret_cast<int*>(smem + L::misc_off + 8);
+    int* s_geom = reinterpret_cast<int*>(smem + L::misc_off + 12);          // {stages, stage bytes}
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 20);
+    ChunkDesc* s_desc = reinterpret_cast<ChunkDesc*>(smem + L::desc_off);
+
+    // ---- prologue: nothing here depends on the previous kernel in the stream
+    if (tid == 0) {
+        for (int i = 0; i < GV_MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, GV_CONS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_xfull + 8 * i, GV_SERV * 32); mbar_init(bar_xempty + 8 * i, GV_CONS); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // from here on the previous kernel's results are needed (sort tables, activations, workspace)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid <= p.R) s_off[tid] = p.offsets[tid];
+    if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+    __syncthreads();
+
+    // ---- the work split, by warp 0: lane v works out pair v
+    if (warp == 0) {
+        const int v = lane;
+        long long cost = 0;
+        int TT = 0, wv = 1;
+        if (v < p.P) {
+            const int rows = s_off[p.rexp[v] + 1] - s_off[p.rexp[v]];
+            wv = p.w[v];
+            TT = rows > 0 ? ((p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
+            cost = (long long)TT * wv;
+        }
+        long long incl = cost;
+        int wmax = TT > 0 ? wv : 1;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const long long o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+            wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, d));
+        }
+        const long long C = __shfl_sync(0xffffffffu, incl, 31);
+        const long long base = incl - cost;
+        const long long Gl = C / wmax;                          // every CTA's share holds at least one super-tile start
+        const int G = (int)(Gl < (long long)gridDim.x ? Gl : (long long)gridDim.x);
+        int tb = 0, te = 0, str = 0;
+        if (v < p.P) {
+            if (TT > 0 && (int)blockIdx.x < G) {
+                const long long den = (long long)wv * G;
+                const long long n0 = (long long)blockIdx.x * C - base * G, n1 = (long long)(blockIdx.x + 1) * C - base * G;
+                const long long t0 = n0 <= 0 ? 0 : (n0 + den - 1) / den, t1 = n1 <= 0 ? 0 : (n1 + den - 1) / den;
+                tb = (int)(t0 > TT ? TT : t0);
+                te = (int)(t1 > TT ? TT : t1);
+            }
+            s_pair[2 * v] = tb;
+            s_pair[2 * v + 1] = te;
+            s_base[v] = base;
+            if (te > tb) str = p.ex[v].tile_stride;
+        }
+        // ring geometry: a stage holds two of the largest packed tiles this CTA will see
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) str = max(str, __shfl_xor_sync(0xffffffffu, str, d));
+        if (lane == 0) {
+            const int stage_bytes = 2 * ((max(str, 128) + 127) & ~127);
+            *s_C = C; *s_G = G;
+            s_geom[0] = min(GV_MAX_STAGES, GV_RING_BYTES / stage_bytes);
+            s_geom[1] = stage_bytes;
+        }
+    }
+    __syncthreads();
+    const int nstg = s_geom[0], stage_bytes = s_geom[1];
+
+    if (warp == GV_CONS + GV_SERV) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint64_t once = l2_policy_evict_first();
+            GvWalk wk;
+            wk.start();
+            Ring ring;
+            bool changed, ok = true;
+            while (ok && wk.next(s_pair, p, changed)) {
+                const int v = wk.v, n = wk.run();
+                const uint32_t stride = (uint32_t)p.ex[v].tile_stride;
+                const int nt = 2 * wk.nt2;
+                const bool two = nt + 1 < p.NT1[v];
+                const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * stride;
+                const uint8_t* b = a + (size_t)wk.KB * stride;
+                for (int i = 0; i < n; ++i) {
+                    if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) { ok = false; break; }
+                    const uint32_t full = bar_wfull + 8 * ring.stage;
+                    const uint32_t dst = sbase + L::ring_off + ring.stage * stage_bytes;
+                    mbar_expect_tx(full, two ? 2 * stride : stride);
+                    bulk_load_once(dst, a, stride, full, once);
+                    if (two) bulk_load_once(dst + (stage_bytes >> 1), b, stride, full, once);
+                    a += stride; b += stride;
+                    ring.advance(nstg);
+                }
+            }
+        }
+    } else if (warp >= GV_CONS) {
+        // ------------------------------------------------------------------ service warps: token rows, one chunk ahead
+        // Thread (m, a) = (st / 16, st % 16) converts the 8 values X[row 2r' + m ...][k-block's k = 8a .. 8a + 7]: a round
+        // is four token rows of one (k-block, token block) slab; four rounds are in flight.
+        const int st = tid - GV_CONS * 32;
+        const int a = st & 15, m4 = st >> 4, G = a >> 2, q = a & 3;
+        GvWalk wk;
+        wk.start();
+        bool changed, more = wk.next(s_pair, p, changed);
+        int kbc = more ? wk.kb : 0;                   // next k-block of the open run to stage
+        for (int n = 0;; ++n) {
+            const int buf = n & 1;
+            if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_xempty + 8 * buf, (uint32_t)((n >> 1) - 1) & 1u, s_abort, p.status))) break;
+            ChunkDesc* d = s_desc + buf;
+            if (!more) {
+                if (st == 0) d->valid = 0;
+                mbar_arrive(bar_xfull + 8 * buf);
+                break;
+            }
+            const int v = wk.v;
+            const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+            const int NT = rows > 8 ? 2 : 1;
+            const int kb1 = wk.kb + wk.run();
+            const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
+            if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
+            const int bits = p.ex[v].bits, K = p.K[v];
+            const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
+            float sig[4];
+            uint32_t sigh[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int e = sigma_shift(bits, 4 * G + i);
+                sig[i] = __int_as_float((127 - e) << 23);
+                sigh[i] = (uint32_t)((15 - e) << 10) * 0x00010001u;
+            }
+            // the thread's source rows: token m = 4j + m4 of the batch's sorted rows of this expert, j = 0..3
+            const uint16_t* rowp[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int m = 4 * j + m4;
+                rowp[j] = (j < 2 * NT && m < rows) ? p.X[v] + (size_t)s_perm[row0 + m] * K + a * 8 : nullptr;
+            }
+            // round r = (k-block kbl, token block tb, row half hh): r = (kbl * NT + tb) * 2 + hh
+            const int rounds = nkb * NT * 2;
+            const uint32_t xdst = sbase + L::x_off + buf * GV_XBUF + ((G * 32 + 4 * m4 + q) << 4);
+            float* sdst = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF) + (m4 >> 1) * 4 + (m4 & 1);
+            auto fetch = [&](int r) -> uint4 {
+                const int slab = r >> 1, hh = r & 1;
+                const int kbl = NT == 2 ? slab >> 1 : slab, tb = NT == 2 ? slab & 1 : 0;
+                const int k = (kbc + kbl) * 128;
+                const uint16_t* src = rowp[2 * tb + hh];
+                uint4 data = make_uint4(0, 0, 0, 0);
+                if (r < rounds && src != nullptr && k + a * 8 < K) data = __ldg(reinterpret_cast<const uint4*>(src + k));
+                return data;
+            };
+            auto convert = [&](int r, const uint4& data) {
+                const uint32_t w[4] = {data.x, data.y, data.z, data.w};
+                uint32_t o[4];
+                float S0 = 0.f, S1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+                    const float sum = lo + hi;
+                    S0 += sum;
+                    S1 = fmaf(sig[i], sum, S1);
+                    __half2 h = __floats2half2_rn(lo, hi);
+                    h = __hmul2(h, *reinterpret_cast<const __half2*>(&sigh[i]));
+                    o[i] = *reinterpret_cast<uint32_t*>(&h);
+                }
+#pragma unroll
+                for (int dlt = 1; dlt < 16; dlt <<= 1) {
+                    S0 += __shfl_xor_sync(0xffffffffu, S0, dlt);
+                    S1 += __shfl_xor_sync(0xffffffffu, S1, dlt);
+                }
+                // fragments at [slab][G][lane = 4 * (4 hh + m4) + q], sums at [slab][t = 2 hh + m4 / 2][4]
+                const int slab = r >> 1, hh = r & 1;
+                sts128(xdst + (slab << 11) + (hh << 8), o[0], o[1], o[2], o[3]);
+                if (a == 0) {
+                    sdst[slab * 16 + hh * 8] = fmaf(-1024.f, S1, -fold * S0);      // what the accumulator starts from
+                    sdst[slab * 16 + hh * 8 + 2] = S0;
+                }
+            };
+            for (int r0 = 0; r0 < rounds; r0 += 4) {
+                uint4 d0 = fetch(r0), d1 = fetch(r0 + 1), d2 = fetch(r0 + 2), d3 = fetch(r0 + 3);
+                convert(r0, d0);
+                if (r0 + 1 < rounds) convert(r0 + 1, d1);
+                if (r0 + 2 < rounds) convert(r0 + 2, d2);
+                if (r0 + 3 < rounds) convert(r0 + 3, d3);
+            }
+            mbar_arrive(bar_xfull + 8 * buf);
+            kbc += nkb;
+            if (kbc >= kb1) {
+                more = wk.next(s_pair, p, changed);
+                kbc = more ? wk.kb : 0;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        const int g = lane >> 2, t = lane & 3;
+        const int half = warp >> 3, blob = warp & 7;
+        const int slot16 = (t * 8 + (g ^ (2 * t))) * 16;          // this lane's 16-byte slot inside a 512-byte half blob
+        const uint32_t tile_base = sbase + L::ring_off + half * (stage_bytes >> 1);
+        Ring ring;
+        float fin[8];                                     // the running sums of the current piece: [token block][4]
+#pragma unroll
+        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+        float sc_r = 0.f, sc_r8 = 0.f, z_r = 0.f, z_r8 = 0.f;     // per-channel experts: scale / zero-point of rows g, g + 8
+        bool ok = true;
+
+        // One chunk of k-blocks of one piece, for a format fixed at compile time.
+        auto run_chunk = [&](auto tag, int nkb, int buf, bool active) {
+            constexpr int BITS = decltype(tag)::bits, NT = decltype(tag)::nt;
+            constexpr bool GROUPED = decltype(tag)::grouped, ASYM = decltype(tag)::asym;
+            const uint32_t xb0 = sbase + L::x_off + buf * GV_XBUF + lane * 16;
+            const float4* sS = reinterpret_cast<const float4*>(smem + L::s_off + buf * GV_SBUF) + t;
+            const uint32_t blob_off = blob * (BITS * 256);
+            const uint32_t meta_off = moqe_tile_bytes(BITS) + (blob * 16 + g) * 2;
+#pragma unroll 1
+            for (int kbl = 0; kbl < nkb; ++kbl) {
+                if (!__all_sync(0xffffffffu, mbar_wait_short(bar_wfull + 8 * ring.stage, ring.phase, s_abort, p.status))) { ok = false; return; }
+                if (active) {
+                    const uint32_t tile = tile_base + ring.stage * stage_bytes;
+                    float acc[NT][4], S0[NT][2];
+#pragma unroll
+                    for (int tb = 0; tb < NT; ++tb) {
+                        const float4 sv = sS[(kbl * NT + tb) * 4];
+                        acc[tb][0] = acc[tb][2] = sv.x;
+                        acc[tb][1] = acc[tb][3] = sv.y;
+                        S0[tb][0] = sv.z;
+                        S0[tb][1] = sv.w;
+                    }
+                    float s0 = sc_r, s8 = sc_r8, z0 = z_r, z8 = z_r8;
+                    if constexpr (GROUPED) {
+                        const uint32_t meta = tile + meta_off;
+                        s0 = __half2float(__ushort_as_half((unsigned short)lds16(meta)));
+                        s8 = __half2float(__ushort_as_half((unsigned short)lds16(meta + 16)));
+                        if constexpr (ASYM) {
+                            z0 = __uint_as_float(lds16(meta + 256) << 16);
+                            z8 = __uint_as_float(lds16(meta + 256 + 16) << 16);
+                        }
+                    }
+                    tile_mma<BITS, NT>(tile + blob_off, slot16, xb0 + ((kbl * NT * 4) << 9), acc);
+                    // the k-block is complete: scale and add
+#pragma unroll
+                    for (int tb = 0; tb < NT; ++tb) {
+                        if constexpr (ASYM) {
+                            fin[4 * tb + 0] = fmaf(s0, fmaf(-z0, S0[tb][0], acc[tb][0]), fin[4 * tb + 0]);
+                            fin[4 * tb + 1] = fmaf(s0, fmaf(-z0, S0[tb][1], acc[tb][1]), fin[4 * tb + 1]);
+                            fin[4 * tb + 2] = fmaf(s8, fmaf(-z8, S0[tb][0], acc[tb][2]), fin[4 * tb + 2]);
+                            fin[4 * tb + 3] = fmaf(s8, fmaf(-z8, S0[tb][1], acc[tb][3]), fin[4 * tb + 3]);
+                        } else {
+                            fin[4 * tb + 0] = fmaf(s0, acc[tb][0], fin[4 * tb + 0]);
+                            fin[4 * tb + 1] = fmaf(s0, acc[tb][1], fin[4 * tb + 1]);
+                            fin[4 * tb + 2] = fmaf(s8, acc[tb][2], fin[4 * tb + 2]);
+                            fin[4 * tb + 3] = fmaf(s8, acc[tb][3], fin[4 * tb + 3]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_wempty + 8 * ring.stage);
+                ring.advance(nstg);
+            }
+        };
+
+        for (int n = 0; ok; ++n) {
+            const int buf = n & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * buf, (uint32_t)(n >> 1) & 1u, s_abort, p.status))) break;
+            const ChunkDesc* d = s_desc + buf;
+            if (!d->valid) break;
+            const int v = d->v, nt2 = d->nt2, kbc = d->kbc, nkb = d->nkb, kb0 = d->kb0, kb1 = d->kb1;
+            const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+            const int bits = p.ex[v].bits, group = p.ex[v].group, has_zeros = p.ex[v].has_zeros;
+            const int nt = 2 * nt2 + half;
+            const bool active = nt < p.NT1[v];
+            const int n_r = nt * 128 + blob * 16 + g;
+            if (kbc == kb0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+                if (group == 0 && active) {
+                    sc_r = __half2float(p.ex[v].scales_pc[n_r]);
+                    sc_r8 = __half2float(p.ex[v].scales_pc[n_r + 8]);
+                    if (has_zeros) {
+                        z_r = __bfloat162float(p.ex[v].zeros_pc[n_r]);
+                        z_r8 = __bfloat162float(p.ex[v].zeros_pc[n_r + 8]);
+                    }
+                }
+            }
+            // dispatch on the format (uniform over the CTA)
+            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : 2)) * 8 + (rows > 8 ? 4 : 0) + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
+            switch (fmt) {
+#define GV_CASE(B, BI, NTV, GR, AS) \
+                case BI * 8 + (NTV - 1) * 4 + GR * 2 + AS: run_chunk(GvTag<B, NTV, GR != 0, AS != 0>{}, nkb, buf, active); break;
+#define GV_CASES(B, BI) GV_CASE(B, BI, 1, 0, 0) GV_CASE(B, BI, 1, 0, 1) GV_CASE(B, BI, 1, 1, 0) GV_CASE(B, BI, 1, 1, 1) \
+                        GV_CASE(B, BI, 2, 0, 0) GV_CASE(B, BI, 2, 0, 1) GV_CASE(B, BI, 2, 1, 0) GV_CASE(B, BI, 2, 1, 1)
+                GV_CASES(4, 0)
+                GV_CASES(8, 1)
+                GV_CASES(3, 2)
+#undef GV_CASES
+#undef GV_CASE
+                default: break;
+            }
+            if (!ok) break;
+
+            if (kbc + nkb == kb1 && active) {
+                // ---- the piece is complete
+                const int NT = rows > 8 ? 2 : 1;
+                const int KB = p.KB[v], N = p.N[v];
+                uint16_t* Y = p.Y[v];
+                auto store_rows = [&]() {
+#pragma unroll
+                    for (int tb = 0; tb < 2; ++tb) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int m = 8 * tb + 2 * t + (j & 1), nn = n_r + (j >> 1) * 8;
+                            if (tb < NT && m < rows && nn < N)
+                                Y[(size_t)s_perm[row0 + m] * N + nn] = __bfloat16_as_ushort(__float2bfloat16_rn(fin[4 * tb + j]));
+                        }
+                    }
+                };
+                if (kb0 == 0 && kb1 == KB) {
+                    store_rows();
+                } else {
+                    // part of a segment: park this warp's sums, announce, and add everything up if this was the last arrival
+                    const long long C = *s_C, base = s_base[v];
+                    const int G = *s_G, wv = p.w[v];
+                    const int c_a = (int)(((base + (long long)(nt2 * KB) * wv) * G) / C);
+                    const int c_b = (int)(((base + (long long)(nt2 * KB + KB - 1) * wv) * G) / C);
+                    float* slot = p.partials + (size_t)(2 * blockIdx.x + (kb0 == 0 ? 1 : 0)) * GV_SLOT_FLOATS;
+#pragma unroll
+                    for (int tb = 0; tb < 2; ++tb)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (tb < NT) __stcg(slot + ((warp * 2 + tb) * 4 + j) * 32 + lane, fin[4 * tb + j]);
+                    __syncwarp();
+                    unsigned arrived = 0;
+                    if (lane == 0) {
+                        __threadfence();
+                        arrived = atomicAdd(p.counters + c_a * GV_CONS + warp, 1u);
+                    }
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    if (arrived == (unsigned)(c_b - c_a)) {
+                        __threadfence();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+                        for (int c = c_a; c <= c_b; ++c) {
+                            const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
+#pragma unroll
+                            for (int tb = 0; tb < 2; ++tb)
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    if (tb < NT) fin[4 * tb + j] += __ldcg(src + ((warp * 2 + tb) * 4 + j) * 32 + lane);
+                        }
+                        store_rows();
+                        if (lane == 0) p.counters[c_a * GV_CONS + warp] = 0u;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_xempty + 8 * buf);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncthreads();
+    if (*s_abort) {
+        // let bulk copies that may still be in flight land before the shared memory is released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+}
+
+int gv_sm_count() {
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
+}
+
+// relative cost of one super-tile in the work split, by code width
+int g_gv_cost[9] = {0, 0, 0, 11, 10, 0, 0, 0, 16};
+
+bool gv_formats_ok(const moqe_expert* const* ex, int n) {
+    for (int v = 0; v < n; ++v) {
+        if (ex[v]->bits != 3 && ex[v]->bits != 4 && ex[v]->bits != 8) return false;
+        if (ex[v]->group != 0 && (ex[v]->group < 128 || ex[v]->group % 128 != 0)) return false;
+    }
+    return true;
+}
+
+}  // namespace
+
+void gemv_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost > 0) g_gv_cost[bits] = cost; }
+
+bool gemv_supported_multi(int M, const moqe_expert* const* ex, int nl, int E) {
+    return M <= DECODE_MAX_ROWS && nl >= 1 && nl * E <= MOQE_MAX_EXPERTS && gv_formats_ok(ex, nl * E);
+}
+
+size_t gemv_zero_bytes(int M) { return M > DECODE_MAX_ROWS ? 0 : (size_t)GV_MAX_GRID * GV_CONS * sizeof(uint32_t); }
+
+size_t gemv_workspace_bytes(int M) {
+    if (M > DECODE_MAX_ROWS) return 0;
+    return (gemv_zero_bytes(M) + 255) / 256 * 256 + (size_t)GV_MAX_GRID * 2 * GV_SLOT_FLOATS * sizeof(float);
+}
+
+// nl layers that share the routing; ex[l * E + e] = expert e of layer l; X[l] / Y[l] the layer's input / output
+moqe_status launch_qgemm_gemv_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
+                                    void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
+                                    size_t ws_bytes, cudaStream_t st) {
+    if (M == 0) return MOQE_OK;
+    if (!gemv_supported_multi(M, ex, nl, E)) return MOQE_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < gemv_workspace_bytes(M)) return MOQE_ERR_WORKSPACE;
+    GvParams p;
+    for (int l = 0; l < nl; ++l)
+        for (int e = 0; e < E; ++e) {
+            const int v = l * E + e;
+            p.ex[v] = ex[v]->dev();
+            p.X[v] = (const uint16_t*)X[l];
+            p.Y[v] = (uint16_t*)Y[l];
+            p.N[v] = ex[v]->N;
+            p.K[v] = ex[v]->K;
+            p.KB[v] = ex[v]->Kp / 128;
+            p.NT1[v] = ex[v]->Np / 128;
+            p.rexp[v] = e;
+            p.w[v] = g_gv_cost[ex[v]->bits];
+        }
+    p.counters = (uint32_t*)ws;
+    p.partials = (float*)((char*)ws + (gemv_zero_bytes(M) + 255) / 256 * 256);
+    p.perm = perm;
+    p.offsets = offsets;
+    p.M = M;
+    p.R = E;
+    p.P = nl * E;
+    p.status = device_status_word();
+    int grid = gv_sm_count();
+    if (grid > GV_MAX_GRID) grid = GV_MAX_GRID;
+    cudaError_t err = cudaFuncSetAttribute(qgemm_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GvSmem::dyn_bytes);
+    if (err == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GV_THREADS); cfg.dynamicSmemBytes = GvSmem::dyn_bytes; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, qgemm_gemv_kernel, p);
+    }
+    if (err != cudaSuccess) return MOQE_ERR_CUDA;
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace moqe
