@@ -138,16 +138,36 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// (v & mask) | 0x6400 in both halves: the fp16 numbers 1024 + (field value), for a field inside the mantissa
-__device__ __forceinline__ uint32_t field_f16(uint32_t v, uint32_t mask) { return (v & mask) | 0x64006400u; }
+// Constants of the unpacking, held in registers the compiler cannot see through: (v & mask) | 0x64006400 is ONE
+// three-input logic instruction when mask and constant are registers, two when they are immediates.
+struct GvConst {
+    uint32_t base, m4lo, m4hi, m3a, m3b, m3c, m3s0, m3s1, m3s2;
+    __device__ __forceinline__ void init() {
+        asm volatile("mov.u32 %0, 0x64006400;" : "=r"(base));
+        asm volatile("mov.u32 %0, 0x000F000F;" : "=r"(m4lo));
+        asm volatile("mov.u32 %0, 0x00F000F0;" : "=r"(m4hi));
+        asm volatile("mov.u32 %0, 0x00070007;" : "=r"(m3a));
+        asm volatile("mov.u32 %0, 0x00380038;" : "=r"(m3b));
+        asm volatile("mov.u32 %0, 0x01C001C0;" : "=r"(m3c));
+        asm volatile("mov.u32 %0, 0x00400040;" : "=r"(m3s0));
+        asm volatile("mov.u32 %0, 0x00800080;" : "=r"(m3s1));
+        asm volatile("mov.u32 %0, 0x01000100;" : "=r"(m3s2));
+    }
+};
+// (v & mask) | c: the fp16 numbers 1024 + (field value) in both halves, for a field inside the mantissa
+__device__ __forceinline__ uint32_t and_or(uint32_t v, uint32_t mask, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(v), "r"(mask), "r"(c));
+    return d;
+}
 
 // pairs 0..3 of one 4-bit word (8 consecutive k): {1024 + c, 1024 + 16c, 1024 + c, 1024 + 16c}
-__device__ __forceinline__ void unpack_w4(uint32_t v, uint32_t (&o)[4]) {
-    o[0] = field_f16(v, 0x000F000Fu);
-    o[1] = field_f16(v, 0x00F000F0u);
+__device__ __forceinline__ void unpack_w4(const GvConst& k, uint32_t v, uint32_t (&o)[4]) {
+    o[0] = and_or(v, k.m4lo, k.base);
+    o[1] = and_or(v, k.m4hi, k.base);
     const uint32_t u = v >> 8;
-    o[2] = field_f16(u, 0x000F000Fu);
-    o[3] = field_f16(u, 0x00F000F0u);
+    o[2] = and_or(u, k.m4lo, k.base);
+    o[3] = and_or(u, k.m4hi, k.base);
 }
 // pairs 0..3 of an 8-bit chunk held in two words: 1024 + c
 __device__ __forceinline__ void unpack_w8(uint32_t w0, uint32_t w1, uint32_t (&o)[4]) {
@@ -158,22 +178,22 @@ __device__ __forceinline__ void unpack_w8(uint32_t w0, uint32_t w1, uint32_t (&o
 }
 // the 16 pairs of a 3-bit piece (words A, B, C): pair p < 15 is field p % 5 of word p / 5 -> 1024 + {1, 8, 64, 1, 8} * c;
 // pair 15 is spread over bit 15 / 31 of the three words -> 1024 + 64c
-__device__ __forceinline__ void unpack_w3(uint32_t A, uint32_t B, uint32_t C, uint32_t (&o)[16]) {
+__device__ __forceinline__ void unpack_w3(const GvConst& k, uint32_t A, uint32_t B, uint32_t C, uint32_t (&o)[16]) {
     const uint32_t w[3] = {A, B, C};
     uint32_t s0 = 0;
 #pragma unroll
     for (int i = 0; i < 3; ++i) {
         const uint32_t u = w[i] >> 9;
         if (i == 0) s0 = u;
-        o[5 * i + 0] = field_f16(w[i], 0x00070007u);
-        o[5 * i + 1] = field_f16(w[i], 0x00380038u);
-        o[5 * i + 2] = field_f16(w[i], 0x01C001C0u);
-        o[5 * i + 3] = field_f16(u, 0x00070007u);
-        o[5 * i + 4] = field_f16(u, 0x00380038u);
+        o[5 * i + 0] = and_or(w[i], k.m3a, k.base);
+        o[5 * i + 1] = and_or(w[i], k.m3b, k.base);
+        o[5 * i + 2] = and_or(w[i], k.m3c, k.base);
+        o[5 * i + 3] = and_or(u, k.m3a, k.base);
+        o[5 * i + 4] = and_or(u, k.m3b, k.base);
     }
-    uint32_t r = field_f16(s0, 0x00400040u);            // bit 15 / 31 of A -> bit 6 / 22: 64 * (code bit 0)
-    r |= (B >> 8) & 0x00800080u;                        // of B -> bit 7 / 23
-    r |= (C >> 7) & 0x01000100u;                        // of C -> bit 8 / 24
+    uint32_t r = and_or(s0, k.m3s0, k.base);            // bit 15 / 31 of A -> bit 6 / 22: 64 * (code bit 0)
+    r = and_or(B >> 8, k.m3s1, r);                      // of B -> bit 7 / 23
+    r = and_or(C >> 7, k.m3s2, r);                      // of C -> bit 8 / 24
     o[15] = r;
 }
 // log2 of 1 / sigma for pair p (0..15) of a piece: how far the code sits above the mantissa's unit
@@ -192,7 +212,7 @@ struct GvTag {
 // The MMAs of one tile for one lane: `blob` is the shared-memory address of the warp's blob, `xb` that of the
 // lane's token fragments of this k-block.
 template <int BITS, int NT>
-__device__ __forceinline__ void tile_mma(uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
+__device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
     uint4 b[NT][4];
 #pragma unroll
     for (int G = 0; G < 4; ++G)
@@ -204,8 +224,8 @@ __device__ __forceinline__ void tile_mma(uint32_t blob, int slot16, uint32_t xb,
 #pragma unroll
         for (int G = 0; G < 4; ++G) {
             uint32_t ar[4], a8[4];
-            unpack_w4(a0[G], ar);
-            unpack_w4(a1[G], a8);
+            unpack_w4(kc, a0[G], ar);
+            unpack_w4(kc, a1[G], a8);
 #pragma unroll
             for (int tb = 0; tb < NT; ++tb) {
                 mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][G].x, b[tb][G].y);
@@ -234,8 +254,8 @@ __device__ __forceinline__ void tile_mma(uint32_t blob, int slot16, uint32_t xb,
         const uint4 w0 = lds128(blob + slot16);
         const uint2 w1 = lds64(blob + 512 + (slot16 >> 1));
         uint32_t ar[16], a8[16];
-        unpack_w3(w0.x, w0.y, w0.z, ar);
-        unpack_w3(w0.w, w1.x, w1.y, a8);
+        unpack_w3(kc, w0.x, w0.y, w0.z, ar);
+        unpack_w3(kc, w0.w, w1.x, w1.y, a8);
 #pragma unroll
         for (int G = 0; G < 4; ++G) {
 #pragma unroll
@@ -459,6 +479,8 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
         const int slot16 = (t * 8 + (g ^ (2 * t))) * 16;          // this lane's 16-byte slot inside a 512-byte half blob
         const uint32_t tile_base = sbase + L::ring_off + half * (stage_bytes >> 1);
         Ring ring;
+        GvConst kc;
+        kc.init();
         float fin[8];                                     // the running sums of the current piece: [token block][4]
 #pragma unroll
         for (int i = 0; i < 8; ++i) fin[i] = 0.f;
@@ -497,7 +519,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
                             z8 = __uint_as_float(lds16(meta + 256 + 16) << 16);
                         }
                     }
-                    tile_mma<BITS, NT>(tile + blob_off, slot16, xb0 + ((kbl * NT * 4) << 9), acc);
+                    tile_mma<BITS, NT>(kc, tile + blob_off, slot16, xb0 + ((kbl * NT * 4) << 9), acc);
                     // the k-block is complete: scale and add
 #pragma unroll
                     for (int tb = 0; tb < NT; ++tb) {
