@@ -39,6 +39,8 @@
 //
 // The operation is Section 3.1 of the paper (the selected quantization expert runs the sample); the paper
 // describes no kernel.
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -295,9 +297,8 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
     // from here on the previous kernel's results are needed (sort tables, activations, workspace)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid <= p.R) s_off[tid] = p.offsets[tid];
+    if (tid >= 32 && tid <= 32 + p.R) s_off[tid - 32] = p.offsets[tid - 32];
     if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
-    __syncthreads();
 
     // ---- the work split, by warp 0: lane v works out pair v
     if (warp == 0) {
@@ -305,7 +306,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
         long long cost = 0;
         int TT = 0, wv = 1;
         if (v < p.P) {
-            const int rows = s_off[p.rexp[v] + 1] - s_off[p.rexp[v]];
+            const int rows = p.offsets[p.rexp[v] + 1] - p.offsets[p.rexp[v]];
             wv = p.w[v];
             TT = rows > 0 ? ((p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
             cost = (long long)TT * wv;
@@ -349,6 +350,92 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
     __syncthreads();
     const int nstg = s_geom[0], stage_bytes = s_geom[1];
 
+    // ---- staging of one chunk of token rows by `nthr` threads (this one is number st of them).  A thread takes whole
+    // row tiles -- the 128 values X[row m][k-block] -- one after the other: sixteen 16-byte fetches (eight in flight),
+    // each converted to four fp16 pairs in MMA fragment order, and the row tile's sums, which need no exchange between
+    // threads.  The caller's walk is advanced past the chunk.  Returns false when there was no chunk left (an invalid
+    // descriptor has been written).
+    auto stage_chunk = [&](GvWalk& wk, int& kbc, bool& more, int n, int nthr, int st) -> bool {
+        const int buf = n & 1;
+        ChunkDesc* d = s_desc + buf;
+        if (!more) {
+            if (st == 0) d->valid = 0;
+            return false;
+        }
+        const int v = wk.v;
+        const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+        const int NT = rows > 8 ? 2 : 1;
+        const int kb1 = wk.kb + wk.run();
+        const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
+        if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
+        const int bits = p.ex[v].bits, K = p.K[v];
+        const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
+        const uint32_t xbuf = sbase + L::x_off + buf * GV_XBUF;
+        float* sbuf = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF);
+        // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block
+        const int tiles = nkb * NT * 8;
+        for (int rt = st; rt < tiles; rt += nthr) {
+            const int slab = rt >> 3, mm = rt & 7;
+            const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
+            const int k0 = (kbc + kbl) * 128;
+            const uint16_t* src = m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
+            const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
+            float S0 = 0.f, S1 = 0.f;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint4 data[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int a = 8 * h + i;
+                    data[i] = make_uint4(0, 0, 0, 0);
+                    if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int a = 8 * h + i, G = a >> 2, q = a & 3;       // chunk (G, q) of the k-block: k = 32G + 8q ..
+                    const uint32_t w[4] = {data[i].x, data[i].y, data[i].z, data[i].w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
+                        const int p16 = 4 * G + j;
+                        const int e = bits == 8 ? 0 : (bits == 4 ? ((j & 1) ? 4 : 0) : (p16 == 15 ? 6 : 3 * ((p16 % 5) % 3)));
+                        const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
+                        const float sum = lo + hi;
+                        S0 += sum;
+                        S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
+                        __half2 hh = __floats2half2_rn(lo, hi);
+                        const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
+                        hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
+                        o[j] = *reinterpret_cast<uint32_t*>(&hh);
+                    }
+                    // fragments at [slab][G][lane = 4 mm + q]
+                    sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
+                }
+            }
+            // sums at [slab][t = mm / 2][4]
+            float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
+            S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
+            S[2] = S0;
+        }
+        kbc += nkb;
+        if (kbc >= kb1) {
+            bool changed;
+            more = wk.next(s_pair, p, changed);
+            kbc = more ? wk.kb : 0;
+        }
+        return true;
+    };
+    // the first chunk is staged by the consumer and service warps together: one fetch latency instead of many
+    GvWalk swk;
+    swk.start();
+    bool s_changed, s_more = swk.next(s_pair, p, s_changed);
+    int s_kbc = s_more ? swk.kb : 0;
+    if (warp < GV_CONS + GV_SERV) {
+        stage_chunk(swk, s_kbc, s_more, 0, (GV_CONS + GV_SERV) * 32, tid);
+        asm volatile("bar.sync 1, %0;" ::"n"((GV_CONS + GV_SERV) * 32) : "memory");   // (the producer is already streaming)
+    }
+
     if (warp == GV_CONS + GV_SERV) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
@@ -357,6 +444,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
             wk.start();
             Ring ring;
             bool changed, ok = true;
+            int issued = 0;
             while (ok && wk.next(s_pair, p, changed)) {
                 const int v = wk.v, n = wk.run();
                 const uint32_t stride = (uint32_t)p.ex[v].tile_stride;
@@ -365,6 +453,10 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
                 const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * stride;
                 const uint8_t* b = a + (size_t)wk.KB * stride;
                 for (int i = 0; i < n; ++i) {
+                    // Ramp-up: when all CTAs ask for a full ring at once, a CTA's first tile queues behind everybody's
+                    // ninth; so the first two stages go out alone and the rest follows once the first has landed.
+                    if (issued == 2 && !mbar_wait(bar_wfull, 0u, s_abort, p.status)) { ok = false; break; }
+                    ++issued;
                     if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) { ok = false; break; }
                     const uint32_t full = bar_wfull + 8 * ring.stage;
                     const uint32_t dst = sbase + L::ring_off + ring.stage * stage_bytes;
@@ -378,99 +470,13 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
         }
     } else if (warp >= GV_CONS) {
         // ------------------------------------------------------------------ service warps: token rows, one chunk ahead
-        // Thread (m, a) = (st / 16, st % 16) converts the 8 values X[row 2r' + m ...][k-block's k = 8a .. 8a + 7]: a round
-        // is four token rows of one (k-block, token block) slab; four rounds are in flight.
         const int st = tid - GV_CONS * 32;
-        const int a = st & 15, m4 = st >> 4, G = a >> 2, q = a & 3;
-        GvWalk wk;
-        wk.start();
-        bool changed, more = wk.next(s_pair, p, changed);
-        int kbc = more ? wk.kb : 0;                   // next k-block of the open run to stage
-        for (int n = 0;; ++n) {
+        for (int n = 1;; ++n) {
             const int buf = n & 1;
             if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_xempty + 8 * buf, (uint32_t)((n >> 1) - 1) & 1u, s_abort, p.status))) break;
-            ChunkDesc* d = s_desc + buf;
-            if (!more) {
-                if (st == 0) d->valid = 0;
-                mbar_arrive(bar_xfull + 8 * buf);
-                break;
-            }
-            const int v = wk.v;
-            const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
-            const int NT = rows > 8 ? 2 : 1;
-            const int kb1 = wk.kb + wk.run();
-            const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
-            if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
-            const int bits = p.ex[v].bits, K = p.K[v];
-            const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
-            float sig[4];
-            uint32_t sigh[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int e = sigma_shift(bits, 4 * G + i);
-                sig[i] = __int_as_float((127 - e) << 23);
-                sigh[i] = (uint32_t)((15 - e) << 10) * 0x00010001u;
-            }
-            // the thread's source rows: token m = 4j + m4 of the batch's sorted rows of this expert, j = 0..3
-            const uint16_t* rowp[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int m = 4 * j + m4;
-                rowp[j] = (j < 2 * NT && m < rows) ? p.X[v] + (size_t)s_perm[row0 + m] * K + a * 8 : nullptr;
-            }
-            // round r = (k-block kbl, token block tb, row half hh): r = (kbl * NT + tb) * 2 + hh
-            const int rounds = nkb * NT * 2;
-            const uint32_t xdst = sbase + L::x_off + buf * GV_XBUF + ((G * 32 + 4 * m4 + q) << 4);
-            float* sdst = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF) + (m4 >> 1) * 4 + (m4 & 1);
-            auto fetch = [&](int r) -> uint4 {
-                const int slab = r >> 1, hh = r & 1;
-                const int kbl = NT == 2 ? slab >> 1 : slab, tb = NT == 2 ? slab & 1 : 0;
-                const int k = (kbc + kbl) * 128;
-                const uint16_t* src = rowp[2 * tb + hh];
-                uint4 data = make_uint4(0, 0, 0, 0);
-                if (r < rounds && src != nullptr && k + a * 8 < K) data = __ldg(reinterpret_cast<const uint4*>(src + k));
-                return data;
-            };
-            auto convert = [&](int r, const uint4& data) {
-                const uint32_t w[4] = {data.x, data.y, data.z, data.w};
-                uint32_t o[4];
-                float S0 = 0.f, S1 = 0.f;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-                    const float sum = lo + hi;
-                    S0 += sum;
-                    S1 = fmaf(sig[i], sum, S1);
-                    __half2 h = __floats2half2_rn(lo, hi);
-                    h = __hmul2(h, *reinterpret_cast<const __half2*>(&sigh[i]));
-                    o[i] = *reinterpret_cast<uint32_t*>(&h);
-                }
-#pragma unroll
-                for (int dlt = 1; dlt < 16; dlt <<= 1) {
-                    S0 += __shfl_xor_sync(0xffffffffu, S0, dlt);
-                    S1 += __shfl_xor_sync(0xffffffffu, S1, dlt);
-                }
-                // fragments at [slab][G][lane = 4 * (4 hh + m4) + q], sums at [slab][t = 2 hh + m4 / 2][4]
-                const int slab = r >> 1, hh = r & 1;
-                sts128(xdst + (slab << 11) + (hh << 8), o[0], o[1], o[2], o[3]);
-                if (a == 0) {
-                    sdst[slab * 16 + hh * 8] = fmaf(-1024.f, S1, -fold * S0);      // what the accumulator starts from
-                    sdst[slab * 16 + hh * 8 + 2] = S0;
-                }
-            };
-            for (int r0 = 0; r0 < rounds; r0 += 4) {
-                uint4 d0 = fetch(r0), d1 = fetch(r0 + 1), d2 = fetch(r0 + 2), d3 = fetch(r0 + 3);
-                convert(r0, d0);
-                if (r0 + 1 < rounds) convert(r0 + 1, d1);
-                if (r0 + 2 < rounds) convert(r0 + 2, d2);
-                if (r0 + 3 < rounds) convert(r0 + 3, d3);
-            }
+            const bool staged = stage_chunk(swk, s_kbc, s_more, n, GV_SERV * 32, st);
             mbar_arrive(bar_xfull + 8 * buf);
-            kbc += nkb;
-            if (kbc >= kb1) {
-                more = wk.next(s_pair, p, changed);
-                kbc = more ? wk.kb : 0;
-            }
+            if (!staged) break;
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
@@ -544,7 +550,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_gemv_kernel(const __grid_
 
         for (int n = 0; ok; ++n) {
             const int buf = n & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * buf, (uint32_t)(n >> 1) & 1u, s_abort, p.status))) break;
+            if (n > 0 && !__all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * buf, (uint32_t)((n - 1) >> 1) & 1u, s_abort, p.status))) break;
             const ChunkDesc* d = s_desc + buf;
             if (!d->valid) break;
             const int v = d->v, nt2 = d->nt2, kbc = d->kbc, nkb = d->nkb, kb0 = d->kb0, kb1 = d->kb1;
