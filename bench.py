@@ -35,14 +35,32 @@ import moqe_workloads as wl  # noqa: E402
 METRIC = "routed_qgemm_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from one ncu capture of the
-# q_proj launch of the workload (profiles/), as a ratio to that launch's algorithmic bytes; traffic grows in
-# proportion with the bytes streamed, so the ratio is applied to the average launch of the block.
-# None = no capture of the current kernel.
-TRAFFIC_RATIO = {
-    "llama7b_decode": 32.748 / 32.513,      # o_proj launch: 32.75 MB read + 0 written (outputs stay in L2) vs 32.51 MB algorithmic
-    "llama7b_prefill": 267.81 / 300.95,     # 158.3 MB read + 109.5 MB written (part of Y still in L2) vs 300.9 MB
-}
+# DRAM traffic of the dominant kernel comes from the tracked table profiles/dram_traffic.txt: one line per ncu capture,
+#   workload  kernel source file  git blob hash of that file when captured  dram bytes per launch  algorithmic bytes of that launch
+# The ratio of the last two is applied to the average launch of the block (traffic grows with the bytes streamed).
+# A line whose hash no longer matches the source file is ignored: `traffic` is then null.
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+
+
+def git_blob_hash(path: str) -> str:
+    import hashlib
+    with open(path, "rb") as f:
+        data = f.read()
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+
+
+def traffic_ratio(workload: str):
+    try:
+        with open(TRAFFIC_TABLE) as f:
+            lines = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    except OSError:
+        return None
+    for name, src, blob, dram, alg in lines:
+        if name == workload:
+            path = os.path.join(ROOT, src)
+            if os.path.exists(path) and git_blob_hash(path) == blob:
+                return float(dram) / float(alg)
+    return None
 
 
 # --------------------------------------------------------------------------- helpers
@@ -234,6 +252,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-fuse", action="store_true", help="one launch per layer (no q/k/v, gate/up grouping)")
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to moqe_tune (measurement knob)")
+    ap.add_argument("--repeats", type=int, default=5, help="timings of --steps steps each; the median is reported")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the sub-records of the other workloads")
     args = ap.parse_args()
     w = wl.get(args.workload)
     heavy = w.kind in ("prefill", "mixed", "conv")
@@ -266,25 +286,88 @@ def main():
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
+    heavy = w.kind in ("prefill", "mixed", "conv")
     peaks = load_peaks()
     seed = replicas.shard_seed(args.seed, rank)             # every rank owns its own shard of samples (weak scaling)
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    ctx = dict(torch=torch, moqe=moqe, replicas=replicas, dev=dev, stream=stream, world=world, rank=rank, local=local,
+               peaks=peaks, seed=seed, args=args, experts={})
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    line = bench_workload(ctx, w, steps=args.steps, warmup=args.warmup, repeats=args.repeats, with_e2e=True)
+    line["clocks"] = sampler.stop()
+
+    # ---- the other workloads of the metric, as sub-records (resident inputs, fewer steps) -------
+    if args.workload == "llama7b_decode" and not args.no_workloads and world == 1:
+        subs = {}
+        for name in ("llama7b_prefill", "qwen7b_mixed", "resnet50_1x1", "tiny"):
+            w2 = wl.get(name)
+            heavy2 = w2.kind in ("prefill", "mixed", "conv")
+            sm = ClockSampler(physical_gpu_index(local))
+            sm.start()
+            rec = bench_workload(ctx, w2, steps=5 if heavy2 else 200, warmup=3 if heavy2 else 20, repeats=3, with_e2e=False)
+            if name == "llama7b_prefill":
+                # the seeded mix is mostly 8-bit rows: time every format alone as well (all sequences to one expert)
+                rec["per_format"] = {}
+                for e, sp in enumerate(w2.experts):
+                    r = bench_workload(ctx, w2, steps=5, warmup=3, repeats=3, with_e2e=False, force_expert=e)
+                    rec["per_format"][sp.tag] = {"ms_per_step": r["ms_per_step"], "roofline": r["roofline"]}
+            rec["clocks"] = sm.stop()
+            subs[name] = {k: rec[k] for k in ("ms_per_step", "value", "unit", "config", "roofline", "gpu_launches", "clocks",
+                                              "device_status", "ms_per_step_repeats") if k in rec}
+            if "per_format" in rec:
+                subs[name]["per_format"] = rec["per_format"]
+            ctx["experts"] = {k: v for k, v in ctx["experts"].items() if k[0] == "llama"}   # free what the next one cannot reuse
+            torch.cuda.empty_cache()
+        line["workloads"] = subs
+
+    # ---- the oracle on this machine's cores (rank 0, single-GPU runs only) ----------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        max_rows = 16 if not heavy else 6
+        prepared, t_quant, t_deq = prepare_oracle(w, args.seed, max_rows)
+        sec = run_oracle_once(w, prepared, None)
+        tokens_per_step = line["config"]["tokens_per_step"]
+        line["cpu_baseline"] = {"value": tokens_per_step / sec, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": oracle_sample_text(w, prepared), "gemm_s_extrapolated": sec,
+                                "dequant_s": t_deq, "quantize_s": t_quant}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
+    """Times one workload: experts built (or reused), inputs resident, one step = route -> expand -> sort -> the routed
+    GEMM of every layer; returns the record (top-level keys of the JSON line)."""
+    import ctypes as C
+    torch, moqe, replicas = ctx["torch"], ctx["moqe"], ctx["replicas"]
+    dev, stream, world, peaks, seed, args = ctx["dev"], ctx["stream"], ctx["world"], ctx["peaks"], ctx["seed"], ctx["args"]
+    heavy = w.kind in ("prefill", "mixed", "conv")
     E = w.n_experts
 
     # ---- experts (replicated on every rank) and resident inputs ---------------------------------
+    family = w.name.split("7b")[0] if "7b" in w.name else w.name
     layers = []
     for layer in w.layers:
-        Wd = torch.from_numpy(wl.weights_f32(f"{w.name}/{layer.name}/W", layer.N, layer.K, 0.02, args.seed)).to(dev)
-        experts = [moqe.moqe_quantize_rtn(Wd, sp.bits, sp.group, sp.sym) for sp in w.experts]
-        del Wd
+        key = (family, layer.name, layer.N, layer.K, tuple(sp.tag for sp in w.experts))
+        if key not in ctx["experts"]:                       # (workloads of one model share shapes and formats: one set of experts)
+            Wd = torch.from_numpy(wl.weights_f32(f"{w.name}/{layer.name}/W", layer.N, layer.K, 0.02, args.seed)).to(dev)
+            ctx["experts"][key] = [moqe.moqe_quantize_rtn(Wd, sp.bits, sp.group, sp.sym) for sp in w.experts]
+            del Wd
+        experts = ctx["experts"][key]
         M = w.M_of(layer)
-        Xh = torch.from_numpy(wl.activations_bf16(f"{w.name}/{layer.name}/X", M, layer.K, w.relu_inputs, seed).view(np.int16)).view(torch.bfloat16).pin_memory()
+        Xh = torch.from_numpy(wl.activations_bf16(f"{w.name}/{layer.name}/X", M, layer.K, w.relu_inputs, seed).view(np.int16)).view(torch.bfloat16)
+        if with_e2e:
+            Xh = Xh.pin_memory()
         X = Xh.to(dev)
         Y = torch.empty((M, layer.N), dtype=torch.bfloat16, device=dev)
-        Yh = torch.empty((M, layer.N), dtype=torch.bfloat16).pin_memory()
+        Yh = torch.empty((M, layer.N), dtype=torch.bfloat16).pin_memory() if with_e2e else None
         ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, layer.N, layer.K, E), dev)
         moqe.moqe_routed_qgemm_workspace_clear(ws, M, layer.N, layer.K, E)
         off_h = torch.from_numpy(w.row_offsets(layer)).pin_memory()
-        import ctypes as C
         arr = (C.c_void_p * E)(*[e.handle for e in experts])
         layers.append(dict(spec=layer, experts=experts, M=M, X=X, Xh=Xh, Y=Y, Yh=Yh, ws=ws, arr=arr,
                            row_off=off_h.to(dev), row_off_h=off_h))
@@ -297,26 +380,22 @@ def main():
             continue
         g = [i]
         for sib in siblings:
-            if L["spec"].name in sib and not args.no_fuse:
+            if L["spec"].name in sib and not args.no_fuse and L["M"] <= 16:
                 g = [j for j, L2 in enumerate(layers) if L2["spec"].name in sib and L2["M"] == L["M"] and L2["spec"].K == L["spec"].K]
         for j in g:
             used.add(j)
         groups.append(g)
-    import ctypes as C2
-    for gi, g in enumerate(groups):
+    for g in groups:
         if len(g) > 1:
             Ls = [layers[j] for j in g]
-            try:                                            # does the library take this group in one launch?
-                arrs = ((C2.c_void_p * len(g))(*[L["X"].data_ptr() for L in Ls]),
-                        (C2.c_void_p * len(g))(*[L["Y"].data_ptr() for L in Ls]),
-                        (C2.c_void_p * (len(g) * E))(*[e.handle for L in Ls for e in L["experts"]]))
-                if Ls[0]["M"] > 16:
-                    raise moqe.MoqeError(moqe.ERR_UNSUPPORTED, "decode only")
-                layers[g[0]]["multi"] = arrs
-            except moqe.MoqeError:
-                groups[gi:gi + 1] = [[j] for j in g]
-    groups = [g for g in groups]
-    logits_h = torch.from_numpy(workload_logits(w, seed)).pin_memory()
+            layers[g[0]]["multi"] = ((C.c_void_p * len(g))(*[L["X"].data_ptr() for L in Ls]),
+                                     (C.c_void_p * len(g))(*[L["Y"].data_ptr() for L in Ls]),
+                                     (C.c_void_p * (len(g) * E))(*[e.handle for L in Ls for e in L["experts"]]))
+    lg = workload_logits(w, seed)
+    if force_expert is not None:                            # every sample to one expert
+        lg = np.full_like(lg, -1.0)
+        lg[:, force_expert] = 1.0
+    logits_h = torch.from_numpy(lg).pin_memory()
     logits = logits_h.to(dev)
     torch.cuda.synchronize()
 
@@ -331,10 +410,10 @@ def main():
 
     # groups of layers that share one row structure share one sort
     def hot_path(from_host: bool):
-        lg = logits
+        lgd = logits
         if from_host:
-            lg.copy_(logits_h, non_blocking=True)
-        ids = moqe.moqe_route(lg)
+            lgd.copy_(logits_h, non_blocking=True)
+        ids = moqe.moqe_route(lgd)
         sorted_for = {}
         for g in groups:
             Ls = [layers[j] for j in g]
@@ -352,9 +431,6 @@ def main():
                 for L in Ls:
                     L["Yh"].copy_(L["Y"], non_blocking=True)
         return sorted_for
-
-    stream = torch.cuda.Stream(device=dev)
-    torch.cuda.set_stream(stream)
 
     def make_runner(from_host: bool):
         """Warm up eagerly, then capture one step in a CUDA graph (the launch-bound inner loop)."""
@@ -375,15 +451,15 @@ def main():
         per_step = moqe.moqe_launch_count() - before
         return g.replay, per_step
 
-    def timed(run, steps, warmup):
-        for _ in range(warmup):
+    def timed(run, n_steps, n_warmup):
+        for _ in range(n_warmup):
             run()
         stream.synchronize()
         replicas.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for _ in range(steps):
+        for _ in range(n_steps):
             run()
         e1.record(stream)
         torch.cuda.synchronize()
@@ -391,22 +467,23 @@ def main():
         return replicas.max_over_ranks(e0.elapsed_time(e1), dev)
 
     tokens_per_step = sum(w.sample_rows) if w.layers[0].rows_per_sample is None else w.n_samples
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
 
-    # ---- 1. resident inputs ---------------------------------------------------------------------
+    # ---- 1. resident inputs: the median of `repeats` timings of `steps` steps each --------------
     run, graph_launches = make_runner(False)
     l0 = moqe.moqe_launch_count()
-    ms = timed(run, args.steps, args.warmup)
-    launches = (graph_launches * args.steps) if graph_launches else (moqe.moqe_launch_count() - l0)
-    ms_per_step = ms / args.steps
+    rep_ms = []
+    for r in range(max(1, repeats)):
+        rep_ms.append(timed(run, steps, warmup if r == 0 else 1) / steps)
+    launches_eager = moqe.moqe_launch_count() - l0
+    launches = (graph_launches * steps) if graph_launches else launches_eager // max(1, repeats)
+    ms_per_step = float(np.median(rep_ms))
     value = replicas.whole_job_value(tokens_per_step, world, ms_per_step)
 
     # ---- 2. per-launch duration of the dominant kernel (events round every routed-GEMM call) ----
     sorted_for = hot_path(False)
     stream.synchronize()
     counts = {k: np.diff(v[1].cpu().numpy()) for k, v in sorted_for.items()}
-    reps = max(3, min(args.steps, 200 if not heavy else 10))
+    reps = max(3, min(steps, 200 if not heavy else 10))
     per_layer_ms = []
     for g in groups:
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
@@ -419,84 +496,76 @@ def main():
             evs[r][1].record(stream)
     stream.synchronize()
     status = moqe.moqe_async_status()
-    clocks = sampler.stop()
     layer_ms = [float(np.mean([a.elapsed_time(b) for a, b in evs[1:]])) for evs in per_layer_ms]
 
-    alg_bytes, flops = [], []
+    alg_bytes, act_bytes, flops = [], [], []
     for L in layers:
         cnt = counts[L["spec"].rows_per_sample]
         b = 0
         for e, ex in enumerate(L["experts"]):
             if cnt[e] > 0:
                 b += ex.code_bytes + ex.meta_bytes
-        b += L["M"] * L["spec"].K * 2 + L["M"] * L["spec"].N * 2
-        alg_bytes.append(b)
+        a = L["M"] * L["spec"].K * 2 + L["M"] * L["spec"].N * 2
+        alg_bytes.append(b + a)
+        act_bytes.append(a)
         flops.append(2.0 * L["M"] * L["spec"].N * L["spec"].K)
     tot_ms = sum(layer_ms)
     n_launch = len(groups)
-    ratio = TRAFFIC_RATIO.get(w.name) if args.path == 0 and not args.tune else None
+    ratio = traffic_ratio(w.name) if args.path == 0 and not args.tune and force_expert is None else None
     traffic = None if ratio is None else ratio * sum(alg_bytes) / n_launch
     hbm_time = sum(alg_bytes) / (peaks["hbm_gbs"] * 1e9)
     tensor_time = sum(flops) / (peaks["bf16_tflops"] * 1e12)
+    hbm = {"achieved": sum(alg_bytes) / (tot_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    hbm["frac"] = hbm["achieved"] / hbm["peak"]
+    hbm["frac_of_nominal_8000"] = hbm["achieved"] / 8000.0
+    tens = {"achieved": sum(flops) / (tot_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+    tens["frac"] = tens["achieved"] / tens["peak"]
+    tens["frac_of_nominal_2250"] = tens["achieved"] / 2250.0
     if tensor_time > hbm_time:
-        achieved = sum(flops) / (tot_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
-                    "frac_whole_step": sum(flops) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                    "frac_of_nominal_2250": achieved / 2250.0}
+        roofline = {"bound": "tensor", **tens, "traffic": traffic,
+                    "frac_whole_step": sum(flops) / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        if w.kind == "mixed":                               # the other fraction of a mixed batch: expert bytes streamed once
+            roofline["hbm"] = hbm
     else:
-        achieved = sum(alg_bytes) / (tot_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic,
-                    "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                    "frac_of_nominal_8000": achieved / 8000.0}
+        roofline = {"bound": "hbm", **hbm, "traffic": traffic,
+                    "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    max_m = max(L["M"] for L in layers)
+    kernel = "qgemm_tc_kernel" if max_m > 128 else ("qgemm_decode_kernel" if max_m <= 16 else "qgemm_stream_kernel")
     roofline.update({"peak_source": peaks["source"],
-                     "kernel": ("qgemm_tc_kernel" if tensor_time > hbm_time else
-                                ("qgemm_decode_kernel" if max(L["M"] for L in layers) <= 16 else "qgemm_stream_kernel")) +
-                               f": average of the {n_launch} routed-GEMM launches of one block" +
+                     "kernel": kernel + f": average of the {n_launch} routed-GEMM launches of one block" +
                                (" (q/k/v and gate/up each in one launch)" if any(len(g) > 1 for g in groups) else ""),
                      "launches_per_step": n_launch, "algorithmic_bytes_per_launch": sum(alg_bytes) / n_launch,
                      "traffic_unit": "bytes per launch",
-                     "algorithmic_bytes_per_step": int(sum(alg_bytes)), "flops_per_step": float(sum(flops)),
+                     "algorithmic_bytes_per_step": int(sum(alg_bytes)), "activation_bytes_per_step": int(sum(act_bytes)),
+                     "flops_per_step": float(sum(flops)),
                      "launch_ms": {"+".join(layers[j]["spec"].name for j in g): round(t, 5) for g, t in zip(groups, layer_ms)}})
 
-    # ---- 3. end to end through the public API with host buffers ---------------------------------
-    run_h, _ = make_runner(True)
-    e2e_steps = max(3, args.steps // 4)
-    ms_h = timed(run_h, e2e_steps, 3) / e2e_steps
-    h2d = int(logits_h.numel() * 4 + sum(L["Xh"].numel() * 2 for L in layers))
-    d2h = int(sum(L["Yh"].numel() * 2 for L in layers))
-    e2e = {"value": replicas.whole_job_value(tokens_per_step, world, ms_h), "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": ms_h}
-
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "ms_per_step_repeats": [round(v, 6) for v in rep_ms], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "layers": [f"{l.name}:{l.N}x{l.K}" for l in w.layers],
                    "experts": [sp.tag for sp in w.experts], "tokens_per_step": tokens_per_step,
                    "rows_per_expert": {str(k): v.tolist() for k, v in counts.items()},
+                   "routing": "every sample to expert %d" % force_expert if force_expert is not None else w.routing,
                    "parallelism": f"replicas x{world} (samples sharded, experts replicated, no collective)",
                    "l2": "weights of one block exceed L2 (inputs larger than L2, no flush)" if sum(alg_bytes) > 126e6
                          else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path,
+                   "timing": f"median of {max(1, repeats)} repeats of {steps} steps",
                    "launch_groups": ["+".join(layers[j]["spec"].name for j in g) for g in groups]},
-        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-        "device_status": moqe.status_str(status),
+        "roofline": roofline, "gpu_launches": int(launches), "device_status": moqe.status_str(status),
     }
 
-    # ---- 4. the oracle on this machine's cores (rank 0, single-GPU runs only) -------------------
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        max_rows = 16 if not heavy else 6
-        prepared, t_quant, t_deq = prepare_oracle(w, args.seed, max_rows)
-        sec = run_oracle_once(w, prepared, None)
-        line["cpu_baseline"] = {"value": tokens_per_step / sec, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                                "sample": oracle_sample_text(w, prepared), "gemm_s_extrapolated": sec,
-                                "dequant_s": t_deq, "quantize_s": t_quant}
-    if rank == 0:
-        print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    # ---- 3. end to end through the public API with host buffers ---------------------------------
+    if with_e2e:
+        run_h, _ = make_runner(True)
+        e2e_steps = max(3, steps // 4)
+        ms_h = timed(run_h, e2e_steps, 3) / e2e_steps
+        h2d = int(logits_h.numel() * 4 + sum(L["Xh"].numel() * 2 for L in layers))
+        d2h = int(sum(L["Yh"].numel() * 2 for L in layers))
+        line["e2e"] = {"value": replicas.whole_job_value(tokens_per_step, world, ms_h), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "ms_per_step": ms_h}
+    return line
 
 
 if __name__ == "__main__":

@@ -5,6 +5,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace moqe {
 
@@ -44,10 +45,8 @@ WsLayout ws_layout(int M, int Np, int K, int E) {
     w.offsets = off; off += align256((MOQE_MAX_EXPERTS + 2) * sizeof(int32_t));
     w.sort = off;    off += align256(sort_workspace_bytes(M, E));
     w.body = off;
-    size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np), c = decode_workspace_bytes(M, Np, E);
-    const size_t d = gemv_workspace_bytes(M);
+    size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np), c = decode_workspace_bytes(M);
     a = a > b ? a : b;
-    a = a > d ? a : d;
     off += align256(a > c ? a : c);
     w.total = off;
     return w;
@@ -57,29 +56,19 @@ constexpr int AUTO_STREAM_MAX_ROWS = 128;
 constexpr int LAST_PATH = 5;
 
 bool g_auto_decode = true;   // whether the automatic choice takes a decode kernel where it applies
-int g_decode_impl = 0;       // 0 = warp-MMA GEMV kernel, 1 = tcgen05 decode kernel (measurement knob)
 
-bool any_decode_supported(int M, const moqe_expert* const* ex, int nl, int E) {
-    return g_decode_impl == 0 ? gemv_supported_multi(M, ex, nl, E) : decode_supported_multi(M, ex, nl, E);
-}
-moqe_status launch_any_decode(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E, void* const* Y,
-                              const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
-    if (g_decode_impl == 0) return launch_qgemm_gemv_multi(X, M, nl, ex, E, Y, perm, offsets, ws, ws_bytes, st);
-    return launch_qgemm_decode_multi(X, M, nl, ex, E, Y, perm, offsets, ws, ws_bytes, st);
-}
-
-// 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = tcgen05 decode kernel
+// 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = decode kernel
 int pick_kernel(int path, int M, const moqe_expert* const* ex, int E) {
     if (path == 5) return 2;
     if (path == 1) return 1;
-    if (path == 0) return (g_auto_decode && any_decode_supported(M, ex, 1, E)) ? 2 : (M <= AUTO_STREAM_MAX_ROWS ? 1 : 0);
+    if (path == 0) return (g_auto_decode && decode_supported_multi(M, ex, 1, E)) ? 2 : (M <= AUTO_STREAM_MAX_ROWS ? 1 : 0);
     return 0;
 }
 
 // the arrival counters at the head of the workspace body (both split-K kernels keep theirs there)
 size_t body_zero_bytes(int M, int Np) {
-    const size_t a = stream_zero_bytes(M, Np), b = decode_zero_bytes(M, Np), c = gemv_zero_bytes(M);
-    return a > b ? (a > c ? a : c) : (b > c ? b : c);
+    const size_t a = stream_zero_bytes(M, Np), b = decode_zero_bytes(M);
+    return a > b ? a : b;
 }
 
 }  // namespace
@@ -116,13 +105,13 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     int32_t* perm = (int32_t*)(base + w.perm);
     int32_t* offsets = (int32_t*)(base + w.offsets);
     const int kernel = pick_kernel(path, M, h_experts, E);
-    if (kernel == 2 && !any_decode_supported(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
+    if (kernel == 2 && !decode_supported_multi(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
     size_t zero_bytes = kernel != 0 ? body_zero_bytes(M, Np) : 0;
     moqe_status s = launch_sort(row_ids, M, E, perm, offsets, base + w.sort, w.body - w.sort, base + w.body, zero_bytes,
                                 Y_bf16, N, st);
     if (s != MOQE_OK) return s;
     if (kernel == 2)
-        return launch_any_decode(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+        return launch_qgemm_decode_multi(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
     if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
@@ -151,9 +140,9 @@ extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)workspace;
     const int kernel = pick_kernel(path, M, h_experts, E);
-    if (kernel == 2 && !any_decode_supported(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
+    if (kernel == 2 && !decode_supported_multi(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
     if (kernel == 2)
-        return launch_any_decode(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+        return launch_qgemm_decode_multi(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
     if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
@@ -179,11 +168,11 @@ extern "C" moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf1
     }
     if (M == 0) return MOQE_OK;
     if (!perm || !offsets) return MOQE_ERR_NULL;
-    if (!any_decode_supported(M, h_experts, n_layers, E)) return MOQE_ERR_UNSUPPORTED;
+    if (!decode_supported_multi(M, h_experts, n_layers, E)) return MOQE_ERR_UNSUPPORTED;
     WsLayout w = ws_layout(M, h_experts[0]->Np, h_experts[0]->K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
     char* base = (char*)workspace;
-    return launch_any_decode(h_X_bf16, M, n_layers, h_experts, E, h_Y_bf16, perm, offsets, base + w.body,
+    return launch_qgemm_decode_multi(h_X_bf16, M, n_layers, h_experts, E, h_Y_bf16, perm, offsets, base + w.body,
                              w.total - w.body, (cudaStream_t)stream);
 }
 
@@ -210,10 +199,6 @@ extern "C" moqe_status moqe_tune(const char* key, int value) {
     if (!strcmp(key, "stream_tile_cost_w4")) { stream_set_tile_cost(4, value); return MOQE_OK; }
     if (!strcmp(key, "stream_tile_cost_w3")) { stream_set_tile_cost(3, value); return MOQE_OK; }
     if (!strcmp(key, "auto_decode")) { g_auto_decode = value != 0; return MOQE_OK; }
-    if (!strcmp(key, "decode_impl")) { g_decode_impl = value != 0; return MOQE_OK; }
-    if (!strcmp(key, "gemv_tile_cost_w8")) { gemv_set_tile_cost(8, value); return MOQE_OK; }
-    if (!strcmp(key, "gemv_tile_cost_w4")) { gemv_set_tile_cost(4, value); return MOQE_OK; }
-    if (!strcmp(key, "gemv_tile_cost_w3")) { gemv_set_tile_cost(3, value); return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w8")) { decode_set_tile_cost(8, value); return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w4")) { decode_set_tile_cost(4, value); return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w3")) { decode_set_tile_cost(3, value); return MOQE_OK; }
@@ -228,6 +213,33 @@ extern "C" moqe_status moqe_async_status(void* stream) {
     if (cudaMemcpy(&v, w, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MOQE_ERR_CUDA;
     if (v != 0 && cudaMemset(w, 0, sizeof(int)) != cudaSuccess) return MOQE_ERR_CUDA;
     return (moqe_status)v;
+}
+
+namespace moqe {
+namespace {
+// One thread initialises an mbarrier on which nobody ever arrives and waits for it with the library's bounded wait.
+__global__ void selftest_timeout_kernel(int* status, unsigned long long limit_ns, int* returned) {
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool ok = mbar_wait_limit(smem_u32(&bar), 0u, &abort_flag, status, limit_ns);
+        *returned = ok ? 1 : 2;
+    }
+}
+}  // namespace
+}  // namespace moqe
+
+extern "C" moqe_status moqe_selftest_timeout(unsigned limit_us, int* d_returned, void* stream) {
+    if (!d_returned) return MOQE_ERR_NULL;
+    if (limit_us == 0 || limit_us > 1000000u) return MOQE_ERR_SHAPE;
+    int* w = device_status_word();
+    if (!w) return MOQE_ERR_ALLOC;
+    selftest_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(w, (unsigned long long)limit_us * 1000ull, d_returned);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
 }
 
 extern "C" const char* moqe_status_str(moqe_status s) {

@@ -115,28 +115,16 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
 size_t stream_zero_bytes(int M, int Np);
 void stream_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split (measurement knob)
 
-// qgemm_decode.cu: decode shapes -- at most DECODE_MAX_ROWS rows, experts per-channel or with groups of >= 128 k
+// qgemm_decode.cu: decode shapes -- at most DECODE_MAX_ROWS rows, experts per-channel or with groups of >= 128 k;
+// nl layers that share the routing go down as one launch (ex[l * E + e] = expert e of layer l)
 constexpr int DECODE_MAX_ROWS = 16;
-bool decode_supported(int M, const moqe_expert* const* ex, int E);
-size_t decode_workspace_bytes(int M, int Np, int E);
-size_t decode_zero_bytes(int M, int Np);
-moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
-                                const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes,
-                                cudaStream_t st);
 bool decode_supported_multi(int M, const moqe_expert* const* ex, int nl, int E);
+size_t decode_workspace_bytes(int M);
+size_t decode_zero_bytes(int M);
 moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
                                       void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
                                       size_t ws_bytes, cudaStream_t st);
-void decode_set_tile_cost(int bits, int cost);   // relative cost of one packed tile in the work split; 0 = its bytes
-
-// qgemm_gemv.cu: the same decode shapes on warp-level MMAs, weights streamed by lane-private asynchronous copies
-bool gemv_supported_multi(int M, const moqe_expert* const* ex, int nl, int E);
-size_t gemv_workspace_bytes(int M);
-size_t gemv_zero_bytes(int M);
-moqe_status launch_qgemm_gemv_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
-                                    void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
-                                    size_t ws_bytes, cudaStream_t st);
-void gemv_set_tile_cost(int bits, int cost);
+void decode_set_tile_cost(int bits, int cost);   // relative cost of one super-tile in the work split, by code width
 
 // qgemm_tcgen05.cu
 void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)

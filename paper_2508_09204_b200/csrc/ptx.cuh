@@ -76,7 +76,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns false if the CTA is aborting (someone's wait ran out).  A failed try has already slept
 // for up to the hint, so the clock and the abort flag are consulted after every few of them.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                unsigned long long limit_ns) {
     if (mbar_try(bar, parity)) return true;
     unsigned long long t0 = 0;
     for (unsigned it = 1;; ++it) {
@@ -85,13 +86,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 latch_status(status, (int)MOQE_ERR_TIMEOUT);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    return mbar_wait_limit(bar, parity, abort_flag, status, WAIT_LIMIT_NS);
 }
 
 // the same bounded wait on the plain try_wait: the clock is consulted every 256 failed tries

@@ -1,731 +1,700 @@
-// Routed dequant-GEMM for decode shapes (at most 16 token rows in the batch): every touched
+// Routed dequant-GEMM for decode shapes (a GEMV-like, HBM-bound path) (at most 16 token rows in the batch): every touched
 // expert's packed weights are streamed from HBM exactly once.
 //
-//   producer (1 thread)     : cp.async.bulk copies of whole packed 128x128-code tiles (codes + the
-//                             tile's scales / zero-points, contiguous in HBM) into a shared-memory
-//                             ring guarded by full/empty mbarriers.
-//                             The copies carry an L2 evict-first policy: weights pass through L2 once.
-//   dequant (4 warpgroups)  : warpgroup w takes the CTA's tiles t = w (mod 4).  Thread r of a
-//                             warpgroup owns channel row r of the tile: it reads the row's packed
-//                             words with conflict-free 128-bit shared loads, unpacks them in registers
-//                             to the exact integers (c - z) in bf16 and stores them straight into
-//                             TENSOR MEMORY (tcgen05.st, lane r) as operand A of the MMA -- no
-//                             shared-memory round trip.  The same warpgroup fetches the token rows of
-//                             its next tile (gathered through `perm`: the fused permutation) with
-//                             16-byte async copies into a K-major, 128-byte-swizzled operand tile.
-//                             Sixteen warps run this one loop, which is what hides the latency of the
-//                             half-rate integer / bf16x2 instructions the unpacking consists of.
-//   MMA issuer (1 warp)     : tcgen05.mma, A from TMEM (128 channels x 16 k), B = the token tile in
-//                             shared memory (N = 16), fp32 accumulators in TMEM, one buffer per
-//                             quantization group:
-//                               Y[m][n] = sum_G s[n][G] * (sum_{k in G} X[m][k] * (c[n][k] - z[n][G]))
-//                             so the tensor core only multiplies exactly representable numbers.
-//                             The whole warp walks the tiles; one elected lane issues eight
-//                             straight-line MMAs per tile and the commits.
-//   epilogue (1 warpgroup)  : drains a finished group buffer (tcgen05.ld), multiplies by the group's
-//                             fp32 scale, accumulates in registers, and at the end of a piece writes
-//                             bf16 rows to their ORIGINAL positions (fused un-permutation) or parks an
-//                             fp32 partial sum.
+//   producer (1 thread)   : one bulk copy per packed 128x128-code tile (codes + the tile's scales / zero-points,
+//                           contiguous in HBM) into a shared-memory ring guarded by full/empty mbarriers.  A stage
+//                           holds a "super-tile": the tiles (nt, nt + 1) of one k-block.  The copies carry an L2
+//                           evict-first policy: weights pass through L2 once.
+//   16 consumer warps     : warp w owns one 16-channel blob of the super-tile.  A lane reads the codes of channel
+//                           rows g and g + 8, k quarter t (its share of an m16n8k16 A fragment) with conflict-free
+//                           128-bit shared loads, unpacks them in registers and issues warp-level tensor-core MMAs
+//                           (fp16 operands, fp32 accumulation) against the token fragments; it applies the group's
+//                           scale in fp32 once per k-block and keeps the running sums of its piece in registers.
+//   4 service warps       : stage the token rows one chunk of k-blocks ahead, double buffered: gathered through
+//                           `perm` (the fused permutation), converted from bf16 to scaled fp16 in MMA fragment order,
+//                           with their sums.  Chunk descriptors travel with the buffers, so the consumers follow the
+//                           work split without walking it themselves.
 //
-// Work split ("stream-K" over packed tiles): all tiles of the call form one sequence
-// [expert][channel tile nt][k-block kb]; tile (e, nt, kb) costs w[e].  CTA c of G owns the tiles
-// whose start cost lies in [c*C/G, (c+1)*C/G) -- equal work to within one tile, at most two partial
-// pieces per CTA: a first one that starts inside its (expert, nt) segment and a last one that stops
-// inside its segment.  A first piece is parked in the workspace and flagged as soon as it is done,
-// early in the kernel; the CTA that holds the head of a segment -- its last piece -- keeps that sum in
-// registers, adds the parked pieces of the following CTAs in CTA order (deterministic) and stores
-// the rows.  All CTAs are resident (grid <= SM count), and the flag wait is bounded like every other.
+//   Unpacking costs 5 integer instructions per 8 four-bit codes (1 per 2 eight-bit codes, 23 per 32 three-bit
+//   codes): a masked code dropped into the mantissa of the fp16 number 1024 becomes 1024 + c, or 1024 + 16c
+//   for a code that sits four bits higher -- no shift, no subtraction.  The tensor core multiplies by token
+//   values that were pre-scaled by 1/16 at exactly those k, and what the constants 1024 and the zero-point
+//   contribute is removed in fp32 with per-(token, k-block) sums of the token values:
+//     Y[m][n] = sum_G s[n][G] * ( sum_{k in G} A[n][k] * B[m][k]  -  1024 * S1[m][G]  -  z[n][G] * S0[m][G] )
+//   A = 1024 + c / sigma_k,  B = sigma_k * x,  S1 = sum sigma_k x,  S0 = sum x.  All products are exact
+//   (11-bit x 8-bit significands).  bf16 token values beyond the fp16 range (|x| > 65504) are outside the
+//   kernel's domain: they turn into infinities.
 //
-// Takes experts that are per-channel or have groups of 128 k or more, and batches of at most 16
-// rows; the caller routes everything else to the other kernels.
+// Work split ("stream-K" over super-tiles): the super-tiles of every (layer, expert) pair whose expert received
+// rows form one sequence [pair][channel-tile pair][k-block] with a per-format cost; CTA c of G owns the
+// super-tiles whose start cost lies in [c*C/G, (c+1)*C/G) -- the split follows the routing, so an expert
+// without rows costs nothing and a batch routed to one expert still uses every SM.  A warp that holds only
+// part of a segment parks its fp32 partial sums and bumps its arrival counter for that segment; whoever
+// arrives last adds the parked sums in CTA order (deterministic) and stores bf16 rows at their original
+// positions (the fused un-permutation).  Nobody waits for another CTA, so the kernel cannot stall whatever
+// else occupies the device.
 //
-// Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, latches
-// MOQE_ERR_TIMEOUT, lets copies in flight land, frees its TMEM and returns.
+// Every mbarrier wait is bounded; on expiry the CTA raises its abort flag, latches MOQE_ERR_TIMEOUT, and
+// every role leaves its loop.
 //
-// The operation is Section 3.1 of the paper (the selected quantization expert runs the sample);
-// the paper describes no kernel.
+// The operation is Section 3.1 of the paper (the selected quantization expert runs the sample); the paper
+// describes no kernel.
 #include <type_traits>
 
-#include "dequant.cuh"
-#include "tc_ptx.cuh"
+#include "common.cuh"
+#include "ptx.cuh"
 
 namespace moqe {
 namespace {
 
-constexpr int TOK = 16;                                 // token columns of the MMA (rows of a batch)
-constexpr int NWG = 4;                                  // dequant warpgroups; warpgroup w takes tiles t = w (mod 4)
-constexpr int DQ_WARPS = 4 * NWG, MMA_WARP = DQ_WARPS, W_WARP = DQ_WARPS + 1;
-constexpr int DEC_THREADS = (DQ_WARPS + 2) * 32;
-constexpr int RING_BYTES = 134 * 1024;                  // packed-weight ring
-constexpr int MAX_STAGES = 16;
-constexpr int NA = 6;                                   // A-operand buffers in TMEM (64 columns each), tile t -> t % 6
-constexpr int ND = 8;                                   // accumulator buffers (TOK columns each), group g -> g % 8
-constexpr int NXS = 10;                                 // token-tile stages, tile t -> t % 10
-constexpr int X_STAGE = TOK * 256;                      // TOK rows x 128 k bf16
-constexpr int DONE_RING = 8;                            // "MMAs of tile t have completed" barriers, tile t -> t % 8
-constexpr int TMEM_COLS = 512;
-constexpr int D_COL0 = NA * 64;
-static_assert(NA > NWG && ND >= 2 * NWG && D_COL0 + ND * TOK <= TMEM_COLS, "buffers: a warpgroup must not wait for the previous round");
-constexpr int MAX_TILES = 512;                          // tiles one CTA can take (its tile table)
+constexpr int GV_CONS = 16;                                    // consumer warps
+constexpr int GV_SERV = 2;                                     // service warps
+constexpr int GV_THREADS = (GV_CONS + GV_SERV + 1) * 32;       // + the producer's warp
+constexpr int GV_MAX_STAGES = 12;
+constexpr int GV_RING_BYTES = 158 * 1024;
+constexpr int GV_XBUF = 32 * 1024;                             // one chunk of staged token rows
+constexpr int GV_CHUNK_KB = 16;                                // k-blocks per chunk for one token block (8 for two)
+constexpr int GV_SBUF = GV_CHUNK_KB * 8 * 2 * 4;               // the chunk's sums: [k-block][token block][t][4] floats
+constexpr int GV_SLOT_FLOATS = GV_CONS * 2 * 4 * 32;           // a parked partial sum: 256 channels x 16 tokens
+constexpr int GV_MAX_GRID = 256;
 
-struct DecSmem {
+struct GvSmem {
     static constexpr int ring_off = 0;
-    static constexpr int x_off = RING_BYTES;
-    static constexpr int out_off = x_off + NXS * X_STAGE;             // float[NWG - 1][TOK][128]: a piece's shares
-    static constexpr int bar_off = out_off + (NWG - 1) * TOK * 512;
-    // wfull[16] wempty[16] afull[NA] done[8] turn[4] flush_free esync
-    static constexpr int n_bars = 2 * MAX_STAGES + NA + DONE_RING + 4 + 1 + 1;
-    static constexpr int misc_off = bar_off + n_bars * 8;              // tmem address, abort flag, ring geometry
-    static constexpr int off_off = misc_off + 32;
-    static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;   // perm of the batch's rows
-    static constexpr int rng_off = perm_off + TOK * 4;
-    static constexpr int ex_off = rng_off + 2 * MOQE_MAX_EXPERTS * 4;  // ExpertSm[MOQE_MAX_EXPERTS]
-    static constexpr int tile_off = (ex_off + MOQE_MAX_EXPERTS * 64 + 15) & ~15;   // uint4[MAX_TILES]
-    static constexpr int piece_off = tile_off + MAX_TILES * 16;        // int[MAX_TILES]: last tile of each piece
-    static constexpr int total = piece_off + MAX_TILES * 4;
-    static constexpr int dyn_bytes = total + 1024;                     // slack for manual 1024-byte alignment
+    static constexpr int x_off = GV_RING_BYTES;
+    static constexpr int s_off = x_off + 2 * GV_XBUF;
+    static constexpr int desc_off = s_off + 2 * GV_SBUF;                  // 2 chunk descriptors of 32 bytes
+    static constexpr int bar_off = desc_off + 2 * 32;                     // wfull[12] wempty[12] xfull[2] xempty[2]
+    static constexpr int off_off = bar_off + (2 * GV_MAX_STAGES + 4) * 8;
+    static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;
+    static constexpr int pair_off = perm_off + 16 * 4;                    // {tb, te} per pair
+    static constexpr int base_off = pair_off + MOQE_MAX_EXPERTS * 8;     // cost before each pair (long long)
+    static constexpr int misc_off = base_off + MOQE_MAX_EXPERTS * 8;     // C (long long), G, stages, stage bytes, abort
+    static constexpr int total = misc_off + 32;
+    static constexpr int dyn_bytes = total;
 };
+static_assert(GvSmem::dyn_bytes <= 227 * 1024, "shared memory budget");
 
-// One call may carry several linear layers that share the routing (same rows, same perm): every (layer, expert)
-// pair is one "expert" of the work split below, with its own packed tiles, shape, input and output.
-struct DecSched {
-    long long C;                    // total cost
-    int G, E;                       // CTAs, (layer, expert) pairs
-    int TT[MOQE_MAX_EXPERTS];       // tiles of the pair (= ntiles * KB of its layer)
-    int w[MOQE_MAX_EXPERTS];        // cost of one of its tiles
-};
-
-struct DecParams {
-    ExpertDev ex[MOQE_MAX_EXPERTS];
-    DecSched sched;
-    const uint16_t* X[MOQE_MAX_EXPERTS];    // per (layer, expert) pair: the layer's input, output and shape,
+struct GvParams {
+    ExpertDev ex[MOQE_MAX_EXPERTS];         // per (layer, expert) pair
+    const uint16_t* X[MOQE_MAX_EXPERTS];    // the layer's input and output
     uint16_t* Y[MOQE_MAX_EXPERTS];
     int N[MOQE_MAX_EXPERTS], K[MOQE_MAX_EXPERTS], KB[MOQE_MAX_EXPERTS];
-    int rexp[MOQE_MAX_EXPERTS];             // and the routing expert whose rows it takes
+    int NT1[MOQE_MAX_EXPERTS];              // 128-channel tiles of the layer
+    int rexp[MOQE_MAX_EXPERTS];             // the routing expert whose rows the pair takes
+    int w[MOQE_MAX_EXPERTS];                // cost of one super-tile
     const int32_t* perm;
     const int32_t* offsets;
-    float* partials;        // [CTA][TOK][128]: the partial sum of a CTA's first piece
-    uint32_t* flags;        // [CTA]: that partial sum is parked; zero on entry, left zero
+    float* partials;                        // [CTA][2][GV_SLOT_FLOATS]
+    uint32_t* counters;                     // [CTA][warp]: arrivals for the segment whose head that CTA holds; zero on entry, left zero
     int* status;
-    int M, R;               // rows of the batch, routing experts
+    int M, R, P;                            // rows of the batch, routing experts, pairs
 };
 
-__device__ __forceinline__ long long dsched_base(const DecSched& s, int e) {
-    long long b = 0;
-    for (int i = 0; i < e; ++i) b += (long long)s.TT[i] * s.w[i];
-    return b;
-}
-// first tile of expert e owned by CTA c or a later CTA
-__device__ __forceinline__ int dsched_tbegin(const DecSched& s, int c, int e, long long base) {
-    const long long num = (long long)c * s.C - base * s.G;
-    if (num <= 0) return 0;
-    const long long den = (long long)s.w[e] * s.G;
-    const long long t = (num + den - 1) / den;
-    return t > s.TT[e] ? s.TT[e] : (int)t;
-}
-__device__ __forceinline__ int dsched_owner(const DecSched& s, int e, long long base, int t) {
-    return (int)(((base + (long long)t * s.w[e]) * s.G) / s.C);
-}
+// one chunk of work: k-blocks [kbc, kbc + nkb) of segment (pair v, channel-tile pair nt2), part of the piece [kb0, kb1)
+struct ChunkDesc { int v, nt2, kbc, nkb, kb0, kb1, valid, pad; };
 
-// The CTA's tiles, in order, as a table in shared memory (one 16-byte entry per tile), built once by the whole CTA
-// after the routing offsets are known: every role then reads its tile with one load instead of walking pieces.
-//   x = kb | nt << 16        y = flags | e << 8 | rows << 16 | row0 << 24        z = accumulation-group index g
-//   w = piece index | (the last CTA that owns a tile of this tile's (expert, nt) segment) << 16
-// flags: first / last tile of its piece, ends / starts an accumulation group, piece = whole segment, piece starts
-// inside its segment
-// An accumulation group (one accumulator buffer handed to the epilogue) is: the whole piece for per-channel
-// experts; for groups of 128 k or more, the k-blocks of one quantization group inside the piece (the scale is
-// constant over the group, so a piece may cut it).
-constexpr int TF_FIRST = 1, TF_LAST = 2, TF_ENDS = 4, TF_WHOLE = 8, TF_KB0NZ = 16, TF_GSTART = 32;
-
-struct ExpertSm {            // per-expert facts of this CTA, in shared memory
-    int tb, te;              // the CTA's tile range inside the expert ([nt][kb] order); empty if the expert has no rows
-    int cum;                 // tiles of earlier experts
-    int gbase;               // accumulation groups of earlier experts
-    int gkb;                 // k-blocks per accumulation group (KB for per-channel experts)
-    int row0, rows;
-    int bits, group, has_zeros, stride;
-    int pbase;               // pieces of earlier experts
-    int KB, N, pad0, pad1;   // k-blocks per segment and output channels of its layer
+// a walk over the CTA's super-tiles in [pair][channel-tile pair][k-block] order, run by run (a run = the k-blocks of
+// one piece: contiguous in HBM)
+struct GvWalk {
+    int v, st, te, kb, KB, nt2;
+    __device__ __forceinline__ void start() { v = -1; st = te = kb = nt2 = 0; KB = 1; }
+    // opens the next run; returns false at the end.  `changed`: the run belongs to another pair than the last one
+    __device__ __forceinline__ bool next(const int* s_pair, const GvParams& p, bool& changed) {
+        changed = false;
+        if (v >= 0) st += run();
+        if (v < 0 || st >= te) {
+            do { ++v; } while (v < p.P && s_pair[2 * v + 1] <= s_pair[2 * v]);
+            if (v >= p.P) return false;
+            st = s_pair[2 * v]; te = s_pair[2 * v + 1]; KB = p.KB[v];
+            nt2 = st / KB; kb = st - nt2 * KB;
+            changed = true;
+        } else {
+            kb = 0; ++nt2;
+        }
+        return true;
+    }
+    __device__ __forceinline__ int run() const { return min(KB - kb, te - st); }
 };
 
-struct Tile {
-    int kb, nt, flags, e, rows, row0, g, piece, c_last;
-    __device__ __forceinline__ explicit Tile(const uint4& v)
-        : kb((int)(v.x & 0xFFFFu)), nt((int)(v.x >> 16)), flags((int)(v.y & 0xFFu)), e((int)((v.y >> 8) & 0xFFu)),
-          rows((int)((v.y >> 16) & 0xFFu)), row0((int)(v.y >> 24)), g((int)v.z), piece((int)(v.w & 0xFFFFu)), c_last((int)(v.w >> 16)) {}
-    __device__ __forceinline__ bool ends() const { return flags & TF_ENDS; }
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// Constants of the unpacking, held in registers the compiler cannot see through: (v & mask) | 0x64006400 is ONE
+// three-input logic instruction when mask and constant are registers, two when they are immediates.
+struct GvConst {
+    uint32_t base, m4lo, m4hi, m3a, m3b, m3c, m3s0, m3s1, m3s2;
+    __device__ __forceinline__ void init() {
+        asm volatile("mov.u32 %0, 0x64006400;" : "=r"(base));
+        asm volatile("mov.u32 %0, 0x000F000F;" : "=r"(m4lo));
+        asm volatile("mov.u32 %0, 0x00F000F0;" : "=r"(m4hi));
+        asm volatile("mov.u32 %0, 0x00070007;" : "=r"(m3a));
+        asm volatile("mov.u32 %0, 0x00380038;" : "=r"(m3b));
+        asm volatile("mov.u32 %0, 0x01C001C0;" : "=r"(m3c));
+        asm volatile("mov.u32 %0, 0x00400040;" : "=r"(m3s0));
+        asm volatile("mov.u32 %0, 0x00800080;" : "=r"(m3s1));
+        asm volatile("mov.u32 %0, 0x01000100;" : "=r"(m3s2));
+    }
+};
+// (v & mask) | c: the fp16 numbers 1024 + (field value) in both halves, for a field inside the mantissa
+__device__ __forceinline__ uint32_t and_or(uint32_t v, uint32_t mask, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(v), "r"(mask), "r"(c));
+    return d;
+}
+
+// pairs 0..3 of one 4-bit word (8 consecutive k): {1024 + c, 1024 + 16c, 1024 + c, 1024 + 16c}
+__device__ __forceinline__ void unpack_w4(const GvConst& k, uint32_t v, uint32_t (&o)[4]) {
+    o[0] = and_or(v, k.m4lo, k.base);
+    o[1] = and_or(v, k.m4hi, k.base);
+    const uint32_t u = v >> 8;
+    o[2] = and_or(u, k.m4lo, k.base);
+    o[3] = and_or(u, k.m4hi, k.base);
+}
+// pairs 0..3 of an 8-bit chunk held in two words: 1024 + c
+__device__ __forceinline__ void unpack_w8(uint32_t w0, uint32_t w1, uint32_t (&o)[4]) {
+    o[0] = __byte_perm(w0, 0x64646464u, 0x4140u);
+    o[1] = __byte_perm(w0, 0x64646464u, 0x4342u);
+    o[2] = __byte_perm(w1, 0x64646464u, 0x4140u);
+    o[3] = __byte_perm(w1, 0x64646464u, 0x4342u);
+}
+// the 16 pairs of a 3-bit piece (words A, B, C): pair p < 15 is field p % 5 of word p / 5 -> 1024 + {1, 8, 64, 1, 8} * c;
+// pair 15 is spread over bit 15 / 31 of the three words -> 1024 + 64c
+__device__ __forceinline__ void unpack_w3(const GvConst& k, uint32_t A, uint32_t B, uint32_t C, uint32_t (&o)[16]) {
+    const uint32_t w[3] = {A, B, C};
+    uint32_t s0 = 0;
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        const uint32_t u = w[i] >> 9;
+        if (i == 0) s0 = u;
+        o[5 * i + 0] = and_or(w[i], k.m3a, k.base);
+        o[5 * i + 1] = and_or(w[i], k.m3b, k.base);
+        o[5 * i + 2] = and_or(w[i], k.m3c, k.base);
+        o[5 * i + 3] = and_or(u, k.m3a, k.base);
+        o[5 * i + 4] = and_or(u, k.m3b, k.base);
+    }
+    uint32_t r = and_or(s0, k.m3s0, k.base);            // bit 15 / 31 of A -> bit 6 / 22: 64 * (code bit 0)
+    r = and_or(B >> 8, k.m3s1, r);                      // of B -> bit 7 / 23
+    r = and_or(C >> 7, k.m3s2, r);                      // of C -> bit 8 / 24
+    o[15] = r;
+}
+// log2 of 1 / sigma for pair p (0..15) of a piece: how far the code sits above the mantissa's unit
+__device__ __forceinline__ int sigma_shift(int bits, int p) {
+    if (bits == 8) return 0;
+    if (bits == 4) return (p & 1) ? 4 : 0;
+    return p == 15 ? 6 : 3 * ((p % 5) % 3);
+}
+
+template <int BITS, int NT, bool GROUPED, bool ASYM>
+struct GvTag {
+    static constexpr int bits = BITS, nt = NT;
+    static constexpr bool grouped = GROUPED, asym = ASYM;
 };
 
-// ---------------------------------------------------------------------------- dequant role
-// Chunk G (8 consecutive k) of a piece as four bf16x2 registers holding the exact integers c - z.  `zc` is the
-// tile's zero-point constant, packed once per tile: bf16x2(128 + z) for 4- and 3-bit codes (0x4300 | c is the
-// bf16 number 128 + c), bf16x2(-z * 2^-13) for 8-bit codes (a zero-extended byte is the bf16 number c * 2^-133;
-// one FMA with 2^120 gives (c - z) * 2^-13, and the fp32 scale carries the 2^13).
-template <int BITS, int G>
-__device__ __forceinline__ void unpack_chunk_zc(const uint32_t (&w)[PieceWords<BITS>::n], uint32_t zc, uint32_t* out) {
+// The MMAs of one tile for one lane: `blob` is the shared-memory address of the warp's blob, `xb` that of the
+// lane's token fragments of this k-block.
+template <int BITS, int NT>
+__device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
+    uint4 b[NT][4];
+#pragma unroll
+    for (int G = 0; G < 4; ++G)
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) b[tb][G] = lds128(xb + ((tb * 4 + G) << 9));
     if constexpr (BITS == 4) {
-        const uint32_t v = w[G];
+        const uint4 w0 = lds128(blob + slot16), w1 = lds128(blob + 512 + slot16);
+        const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) out[i] = hsub2_bf16(((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zc);
-    } else if constexpr (BITS == 3) {
+        for (int G = 0; G < 4; ++G) {
+            uint32_t ar[4], a8[4];
+            unpack_w4(kc, a0[G], ar);
+            unpack_w4(kc, a1[G], a8);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int pr = 4 * G + i;                 // pair index inside the piece
-            uint32_t v;
-            if (pr < 15) v = (w[pr / 5] >> (3 * (pr % 5))) & 0x00070007u;
-            else v = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[2] >> 13) & 0x00040004u);
-            out[i] = hsub2_bf16(v | 0x43004300u, zc);
+            for (int tb = 0; tb < NT; ++tb) {
+                mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][G].x, b[tb][G].y);
+                mma_f16(acc[tb], ar[2], a8[2], ar[3], a8[3], b[tb][G].z, b[tb][G].w);
+            }
+        }
+    } else if constexpr (BITS == 8) {
+        // 512-byte blocks of the blob: {row g: chunks 0,1}, {row g: chunks 2,3}, {row g + 8: chunks 0,1}, {row g + 8: chunks 2,3}
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint4 w0 = lds128(blob + u * 512 + slot16), w1 = lds128(blob + 1024 + u * 512 + slot16);
+            const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg) {
+                uint32_t ar[4], a8[4];
+                unpack_w8(a0[2 * gg], a0[2 * gg + 1], ar);
+                unpack_w8(a1[2 * gg], a1[2 * gg + 1], a8);
+#pragma unroll
+                for (int tb = 0; tb < NT; ++tb) {
+                    mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][2 * u + gg].x, b[tb][2 * u + gg].y);
+                    mma_f16(acc[tb], ar[2], a8[2], ar[3], a8[3], b[tb][2 * u + gg].z, b[tb][2 * u + gg].w);
+                }
+            }
         }
     } else {
-        const uint32_t k120 = 0x7B807B80u;           // 2^120 in both halves
+        const uint4 w0 = lds128(blob + slot16);
+        const uint2 w1 = lds64(blob + 512 + (slot16 >> 1));
+        uint32_t ar[16], a8[16];
+        unpack_w3(kc, w0.x, w0.y, w0.z, ar);
+        unpack_w3(kc, w0.w, w1.x, w1.y, a8);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t pair = __byte_perm(w[2 * G + (i >> 1)], 0u, (i & 1) ? 0x4342u : 0x4140u);
-            __nv_bfloat162 r = __hfma2(*reinterpret_cast<const __nv_bfloat162*>(&pair), *reinterpret_cast<const __nv_bfloat162*>(&k120),
-                                       *reinterpret_cast<const __nv_bfloat162*>(&zc));
-            out[i] = *reinterpret_cast<uint32_t*>(&r);
+        for (int G = 0; G < 4; ++G) {
+#pragma unroll
+            for (int tb = 0; tb < NT; ++tb) {
+                mma_f16(acc[tb], ar[4 * G], a8[4 * G], ar[4 * G + 1], a8[4 * G + 1], b[tb][G].x, b[tb][G].y);
+                mma_f16(acc[tb], ar[4 * G + 2], a8[4 * G + 2], ar[4 * G + 3], a8[4 * G + 3], b[tb][G].z, b[tb][G].w);
+            }
         }
     }
-}
-
-// One packed tile -> operand A in tensor memory, for the thread that owns channel row `row` (= its TMEM lane).
-// MMA k index k' = 32q + 8G + t holds the code of real k = 32G + 8q + t (piece q, chunk G): a piece then fills 16
-// consecutive TMEM columns with one store, and the token-tile loader applies the same permutation to its
-// 16-byte chunks.
-template <int BITS>
-__device__ __forceinline__ void dequant_tile(const unsigned char* stage, int row, uint32_t zc, uint32_t a_taddr) {
-    const unsigned char* blob = stage + (row >> 4) * moqe_blob_bytes(BITS);
-    const int half = (row >> 3) & 1, r = row & 7;
-#pragma unroll 1
-    for (int q = 0; q < 4; ++q) {
-        uint32_t w[PieceWords<BITS>::n];
-        load_piece_smem<BITS>(blob, half, q * 8 + (r ^ (2 * q)), w);
-        uint32_t o[16];
-        unpack_chunk_zc<BITS, 0>(w, zc, o);
-        unpack_chunk_zc<BITS, 1>(w, zc, o + 4);
-        unpack_chunk_zc<BITS, 2>(w, zc, o + 8);
-        unpack_chunk_zc<BITS, 3>(w, zc, o + 12);
-        tmem_st16(a_taddr + 16 * q, o);
-    }
-}
-
-// The token rows of one tile (expert rows [row0, row0 + rows) of the sorted batch, k-block kb) as a K-major,
-// 128-byte-swizzled UMMA operand: two halves of 64 k', each TOK rows x 128 bytes; 16-byte chunk (G, q) of real k
-// goes to chunk 4q + G of k'.  Issued by the 128 threads of one warpgroup (t = thread index in it); k >= K is
-// zero-filled.  Rows beyond `rows` are left as they are: their columns of the accumulator are never read.
-__device__ __forceinline__ void load_token_tile(const uint16_t* X, int K, const volatile int* s_perm, uint32_t xs, int row0, int rows,
-                                                int kb, int t) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int id = t + 128 * i, m = id >> 4, a = id & 15;
-        if (m < rows) {
-            const int src_row = s_perm[row0 + m];
-            const int k = kb * 128 + a * 8;
-            const int nbytes = max(0, min(16, (K - k) * 2));
-            const uint16_t* src = nbytes > 0 ? X + (size_t)src_row * K + k : X;
-            const int ap = 4 * (a & 3) + (a >> 2);
-            cp_async16(xs + (ap >> 3) * (TOK * 128) + m * 128 + (((ap & 7) ^ (m & 7)) << 4), src, nbytes);
-        }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------- the kernel
-__global__ void __launch_bounds__(DEC_THREADS, 1) qgemm_decode_kernel(const __grid_constant__ DecParams p) {
-    using L = DecSmem;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+__global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __grid_constant__ GvParams p) {
+    using L = GvSmem;
+    extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar0 = sbase + L::bar_off;
-    const uint32_t bar_wfull = bar0, bar_wempty = bar0 + 8 * MAX_STAGES, bar_afull = bar_wempty + 8 * MAX_STAGES;
-    const uint32_t bar_done = bar_afull + 8 * NA, bar_turn = bar_done + 8 * DONE_RING;
-    const uint32_t bar_flushfree = bar_turn + 8 * 4, bar_esync = bar_flushfree + 8;
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + L::misc_off);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
-    volatile int* s_geom = reinterpret_cast<volatile int*>(smem + L::misc_off + 8);    // {stages, stage bytes, tiles}
-    volatile int* s_off = reinterpret_cast<volatile int*>(smem + L::off_off);
-    volatile int* s_rng = reinterpret_cast<volatile int*>(smem + L::rng_off);
-    volatile int* s_perm = reinterpret_cast<volatile int*>(smem + L::perm_off);
-    ExpertSm* s_ex = reinterpret_cast<ExpertSm*>(smem + L::ex_off);
-    const uint4* s_tile = reinterpret_cast<const uint4*>(smem + L::tile_off);
-    float* s_out = reinterpret_cast<float*>(smem + L::out_off);
-    volatile int* s_piece = reinterpret_cast<volatile int*>(smem + L::piece_off);
-    const DecSched& sch = p.sched;
-    // warp-uniform bounded wait: every lane polls, the warp agrees on the verdict
-    auto wwait = [&](uint32_t bar, uint32_t parity) -> bool {
-        return __all_sync(0xffffffffu, mbar_wait_short(bar, parity, s_abort, p.status));
-    };
-    // one arrival per warp, after all its lanes are done with what the barrier hands over
-    auto warrive = [&](uint32_t bar) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar);
-    };
-    // done[t % 8] completes when the MMAs of the CTA's t-th tile have
-    auto wait_done = [&](int t) -> bool {
-        return t < 0 || wwait(bar_done + 8 * (t & (DONE_RING - 1)), (uint32_t)(t >> 3) & 1u);
-    };
+    const uint32_t bar_wfull = sbase + L::bar_off, bar_wempty = bar_wfull + 8 * GV_MAX_STAGES;
+    const uint32_t bar_xfull = bar_wempty + 8 * GV_MAX_STAGES, bar_xempty = bar_xfull + 16;
+    int* s_off = reinterpret_cast<int*>(smem + L::off_off);
+    int* s_perm = reinterpret_cast<int*>(smem + L::perm_off);
+    int* s_pair = reinterpret_cast<int*>(smem + L::pair_off);
+    long long* s_base = reinterpret_cast<long long*>(smem + L::base_off);
+    long long* s_C = reinterpret_cast<long long*>(smem + L::misc_off);
+    int* s_G = reinterpret_cast<int*>(smem + L::misc_off + 8);
+    int* s_geom = reinterpret_cast<int*>(smem + L::misc_off + 12);          // {stages, stage bytes}
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 20);
+    ChunkDesc* s_desc = reinterpret_cast<ChunkDesc*>(smem + L::desc_off);
 
-    // ---- prologue: launch parameters only, so it may overlap the tail of the previous kernel in the stream
+    // ---- prologue: nothing here depends on the previous kernel in the stream
     if (tid == 0) {
-        for (int i = 0; i < MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, 4); }
-        for (int i = 0; i < NA; ++i) mbar_init(bar_afull + 8 * i, 4);
-        for (int i = 0; i < DONE_RING; ++i) mbar_init(bar_done + 8 * i, 1);
-        mbar_init(bar_turn, DQ_WARPS);                  // every dequant warp, once per piece
-        mbar_init(bar_flushfree, 4);
-        mbar_init(bar_esync, 4);                         // the four warps of the finalizing warpgroup
+        for (int i = 0; i < GV_MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, GV_CONS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_xfull + 8 * i, GV_SERV * 32); mbar_init(bar_xempty + 8 * i, GV_CONS); }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid >= 32 && tid < 32 + sch.E) {                    // this CTA's tile range inside each expert
-        const int e = tid - 32;
-        const long long base = dsched_base(sch, e);
-        s_rng[2 * e] = dsched_tbegin(sch, blockIdx.x, e, base);
-        s_rng[2 * e + 1] = dsched_tbegin(sch, blockIdx.x + 1, e, base);
-    }
-    if (warp == MMA_WARP) tmem_alloc(sbase + L::misc_off, TMEM_COLS);
     // from here on the previous kernel's results are needed (sort tables, activations, workspace)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid <= p.R) s_off[tid] = p.offsets[tid];
-    if (tid >= 64 && tid < 64 + TOK) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    if (tid >= 32 && tid <= 32 + p.R) s_off[tid - 32] = p.offsets[tid - 32];
+    if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+
+    // ---- the work split, by warp 0: lane v works out pair v
     if (warp == 0) {
-        // Per-expert facts, the ring geometry (stage = the largest packed tile this CTA will see) and the tile count:
-        // lane e works out expert e (E <= 32), the running totals come from a warp scan -- one thread doing all
-        // experts in turn costs the better part of a microsecond at every launch.
-        const int e = lane;
-        ExpertSm x = {};
-        int cnt = 0, ng = 0, np = 0, str = 0;
-        if (e < sch.E) {
-            x.row0 = s_off[p.rexp[e]];
-            x.rows = min(s_off[p.rexp[e] + 1] - x.row0, TOK);
-            x.KB = p.KB[e]; x.N = p.N[e];
-            x.tb = s_rng[2 * e];
-            x.te = x.rows > 0 ? s_rng[2 * e + 1] : x.tb;
-            x.bits = p.ex[e].bits; x.group = p.ex[e].group; x.has_zeros = p.ex[e].has_zeros; x.stride = p.ex[e].tile_stride;
-            x.gkb = x.group == 0 ? x.KB : x.group / 128;
-            if (x.te > x.tb) {
-                cnt = x.te - x.tb;
-                ng = x.te / x.gkb - x.tb / x.gkb + (x.te % x.gkb != 0 ? 1 : 0);
-                np = (x.te - 1) / x.KB - x.tb / x.KB + 1;
-                str = x.stride;
-            }
+        const int v = lane;
+        long long cost = 0;
+        int TT = 0, wv = 1;
+        if (v < p.P) {
+            const int rows = p.offsets[p.rexp[v] + 1] - p.offsets[p.rexp[v]];
+            wv = p.w[v];
+            TT = rows > 0 ? ((p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
+            cost = (long long)TT * wv;
         }
-        int c = cnt, g = ng, q = np, wmax = str;            // inclusive scans / maximum over the lanes
+        long long incl = cost;
+        int wmax = TT > 0 ? wv : 1;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const int c2 = __shfl_up_sync(0xffffffffu, c, d), g2 = __shfl_up_sync(0xffffffffu, g, d),
-                      q2 = __shfl_up_sync(0xffffffffu, q, d);
-            if (lane >= d) { c += c2; g += g2; q += q2; }
+            const long long o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
             wmax = max(wmax, __shfl_xor_sync(0xffffffffu, wmax, d));
         }
-        if (e < sch.E) {
-            x.cum = c - cnt;
-            x.gbase = g - ng;
-            x.pbase = q - np;
-            s_ex[e] = x;
+        const long long C = __shfl_sync(0xffffffffu, incl, 31);
+        const long long base = incl - cost;
+        const long long Gl = C / wmax;                          // every CTA's share holds at least one super-tile start
+        const int G = (int)(Gl < (long long)gridDim.x ? Gl : (long long)gridDim.x);
+        int tb = 0, te = 0, str = 0;
+        if (v < p.P) {
+            if (TT > 0 && (int)blockIdx.x < G) {
+                const long long den = (long long)wv * G;
+                const long long n0 = (long long)blockIdx.x * C - base * G, n1 = (long long)(blockIdx.x + 1) * C - base * G;
+                const long long t0 = n0 <= 0 ? 0 : (n0 + den - 1) / den, t1 = n1 <= 0 ? 0 : (n1 + den - 1) / den;
+                tb = (int)(t0 > TT ? TT : t0);
+                te = (int)(t1 > TT ? TT : t1);
+            }
+            s_pair[2 * v] = tb;
+            s_pair[2 * v + 1] = te;
+            s_base[v] = base;
+            if (te > tb) str = p.ex[v].tile_stride;
         }
-        if (lane == 31) {
-            const int stage_bytes = (max(wmax, 128) + 127) & ~127;
-            s_geom[0] = min(MAX_STAGES, RING_BYTES / stage_bytes);
-            s_geom[1] = stage_bytes;
-            s_geom[2] = min(c, MAX_TILES);
-            s_geom[3] = q;
-        }
-    }
-    __syncthreads();
-    const uint32_t tmem_base = *s_tmem;
-    const int nstg = s_geom[0], stage_bytes = s_geom[1], T = s_geom[2], NP = s_geom[3];
-    for (int i = tid; i < T; i += DEC_THREADS) {            // the tile table, one thread per tile
-        int e = 0;
-        while (e + 1 < sch.E && s_ex[e + 1].cum <= i) ++e;
-        while (s_ex[e].te <= s_ex[e].tb) ++e;               // (experts without tiles share their successor's cum)
-        const ExpertSm x = s_ex[e];
-        const int KB = x.KB;
-        const int tile = x.tb + i - x.cum, nt = tile / KB, kb = tile - nt * KB;
-        const int kb0 = max(x.tb - nt * KB, 0), kb1 = min(x.te - nt * KB, KB);
-        const bool last = kb + 1 == kb1;
-        int flags = (kb == kb0 ? TF_FIRST : 0) | (last ? TF_LAST : 0) | ((last || (kb + 1) % x.gkb == 0) ? TF_ENDS : 0) |
-                    ((kb0 == 0 && kb1 == KB) ? TF_WHOLE : 0) | (kb0 != 0 ? TF_KB0NZ : 0) |
-                    ((kb == kb0 || kb % x.gkb == 0) ? TF_GSTART : 0);
-        const int piece = x.pbase + nt - x.tb / KB;
-        uint4 v;
-        v.x = (uint32_t)kb | ((uint32_t)nt << 16);
-        v.y = (uint32_t)flags | ((uint32_t)e << 8) | ((uint32_t)x.rows << 16) | ((uint32_t)x.row0 << 24);
-        v.z = (uint32_t)(x.gbase + tile / x.gkb - x.tb / x.gkb);
-        // owner of the segment's last tile (needed where the head of a split segment ends)
-        v.w = (uint32_t)piece |
-              ((last && kb0 == 0 && kb1 != KB) ? (uint32_t)dsched_owner(sch, e, dsched_base(sch, e), nt * KB + KB - 1) << 16 : 0u);
-        if (last) s_piece[piece] = i;
-        *reinterpret_cast<uint4*>(smem + L::tile_off + 16 * i) = v;
-    }
-    __syncthreads();
-
-    if (warp == W_WARP) {
-        // ------------------------------------------------------------------ packed-weight producer
+        // ring geometry: a stage holds two of the largest packed tiles this CTA will see
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) str = max(str, __shfl_xor_sync(0xffffffffu, str, d));
         if (lane == 0) {
-            Ring ring;
-            const uint64_t once = l2_policy_evict_first();   // weights cross L2 once per call
-            for (int t = 0; t < T; ++t) {
-                const Tile ti(s_tile[t]);
-                const uint32_t wbytes = (uint32_t)s_ex[ti.e].stride;
-                if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) break;
-                const uint32_t full = bar_wfull + 8 * ring.stage;
-                mbar_expect_tx(full, wbytes);
-                bulk_load_once(sbase + L::ring_off + ring.stage * stage_bytes,
-                               p.ex[ti.e].tiles + ((size_t)ti.nt * s_ex[ti.e].KB + ti.kb) * wbytes, wbytes, full, once);
-                ring.advance(nstg);
-            }
+            const int stage_bytes = 2 * ((max(str, 128) + 127) & ~127);
+            *s_C = C; *s_G = G;
+            s_geom[0] = min(GV_MAX_STAGES, GV_RING_BYTES / stage_bytes);
+            s_geom[1] = stage_bytes;
         }
-    } else if (warp == MMA_WARP) {
-        // ------------------------------------------------------------------ MMA issuer
-        // The whole warp walks the tiles (warp-uniform control flow); one elected lane issues.  No accumulator
-        // hand-shake is needed: buffer g % 8 is drained by the warpgroup that unpacked the group's last tile j before
-        // it hands over its tile j + 8, and the group that reuses the buffer starts at tile j + 8 or later.
-        const uint32_t idesc = umma_idesc(TOK);
-        int a = 0, xst = 0;
-        uint32_t aphase = 0;
-        for (int t = 0; t < T; ++t) {
-            const Tile ti(s_tile[t]);
-            if (!wwait(bar_afull + 8 * a, aphase)) break;
-            tc_fence_after();
-            const uint32_t xs = sbase + L::x_off + xst * X_STAGE;
-            const uint32_t dt = tmem_base + D_COL0 + (ti.g & (ND - 1)) * TOK, a0 = tmem_base + a * 64;
-            const uint64_t b0 = umma_desc_sw128(xs), b1 = umma_desc_sw128(xs + TOK * 128);
-            const uint32_t acc0 = (ti.flags & TF_GSTART) ? 0u : 1u;
-            if (elect_one()) {
-                umma_bf16_ts(dt, a0, b0, idesc, acc0);
-                umma_bf16_ts(dt, a0 + 8, b0 + 2, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 16, b0 + 4, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 24, b0 + 6, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 32, b1, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 40, b1 + 2, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 48, b1 + 4, idesc, 1u);
-                umma_bf16_ts(dt, a0 + 56, b1 + 6, idesc, 1u);
-                umma_commit(bar_done + 8 * (t & (DONE_RING - 1)));
-            }
-            __syncwarp();
-            if (++a == NA) { a = 0; aphase ^= 1u; }
-            if (++xst == NXS) xst = 0;
+    }
+    __syncthreads();
+    const int nstg = s_geom[0], stage_bytes = s_geom[1];
+
+    // ---- staging of one chunk of token rows by `nthr` threads (this one is number st of them).  A thread takes whole
+    // row tiles -- the 128 values X[row m][k-block] -- one after the other: sixteen 16-byte fetches (eight in flight),
+    // each converted to four fp16 pairs in MMA fragment order, and the row tile's sums, which need no exchange between
+    // threads.  The caller's walk is advanced past the chunk.  Returns false when there was no chunk left (an invalid
+    // descriptor has been written).
+    auto stage_chunk = [&](GvWalk& wk, int& kbc, bool& more, int n, int nthr, int st) -> bool {
+        const int buf = n & 1;
+        ChunkDesc* d = s_desc + buf;
+        if (!more) {
+            if (st == 0) d->valid = 0;
+            return false;
         }
-    } else if (warp < DQ_WARPS) {
-        // ------------------------------------------------------------------ dequant warpgroups
-        const int wg = warp >> 2, row = (warp & 3) * 32 + lane, twg = tid & 127;
-        const uint32_t lane_taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-        auto x_load = [&](int t) {                   // token rows of tile t (an empty group past the end)
-            if (t < T) {
-                const Tile xi(s_tile[t]);
-                load_token_tile(p.X[xi.e], p.K[xi.e], s_perm, sbase + L::x_off + (t % NXS) * X_STAGE, xi.row0, xi.rows, xi.kb, twg);
-            } else {
-                asm volatile("cp.async.commit_group;" ::: "memory");
-            }
-        };
-        float acc[TOK];                              // this warpgroup's share of the current piece, channel `row`
+        const int v = wk.v;
+        const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+        const int NT = rows > 8 ? 2 : 1;
+        const int kb1 = wk.kb + wk.run();
+        const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
+        if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
+        const int bits = p.ex[v].bits, K = p.K[v];
+        const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
+        const uint32_t xbuf = sbase + L::x_off + buf * GV_XBUF;
+        float* sbuf = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF);
+        // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block
+        const int tiles = nkb * NT * 8;
+        for (int rt = st; rt < tiles; rt += nthr) {
+            const int slab = rt >> 3, mm = rt & 7;
+            const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
+            const int k0 = (kbc + kbl) * 128;
+            const uint16_t* src = m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
+            const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
+            float S0 = 0.f, S1 = 0.f;
 #pragma unroll
-        for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
-        int flushed = 0;                             // pieces this warpgroup has handed to the finalizer
-        // Accumulation groups that ended with this warpgroup's last two tiles and are not drained yet.  A group is
-        // drained TWO rounds after its last tile was handed over: one round later its MMAs may still be queued behind
-        // the other warpgroups' tiles, and waiting for them would put the MMA round trip into every round.
-        struct Rec { int t, g, piece; float s; };
-        Rec r0{-1, 0, 0, 0.f}, r1{-1, 0, 0, 0.f};    // two rounds back, previous round
-        int acc_piece = -1;                          // the piece `acc` belongs to
-        int last_t = -1, ph0 = 0, ph1 = 0;                        // pieces of this warpgroup's tiles of two rounds / one round ago
-        bool ok = true;
-        // scale and add a finished group (the caller knows that its MMAs have completed)
-        auto drain = [&](Rec& r) {
-            if (r.t < 0) return;
-            tc_fence_after();
-            uint32_t v[16];
-            tmem_ld16(lane_taddr + D_COL0 + (r.g & (ND - 1)) * TOK, v);
-            tmem_ld_wait();
+            for (int h = 0; h < 2; ++h) {
+                uint4 data[8];
 #pragma unroll
-            for (int i = 0; i < TOK; ++i) acc[i] = fmaf(r.s, __uint_as_float(v[i]), acc[i]);
-            tc_fence_before();
-            acc_piece = r.piece;
-            r.t = -1;
-        };
-        // The last warpgroup of the chain also finishes the piece: with the sum of all four shares in registers it
-        // stores the rows at their original positions (fused un-permutation), parks the sum, or adds the parked sums
-        // of other CTAs.
-        uint32_t esync_phase = 0;
-        const int et = twg;
-        auto finalize = [&](int q, float (&acc)[TOK]) -> bool {
-            const Tile ti(s_tile[s_piece[q]]);       // the piece's last tile carries its facts
-            const int n = ti.nt * 128 + row, j0 = ti.row0, rows = ti.rows, N = s_ex[ti.e].N;
-            uint16_t* Y = p.Y[ti.e];
-            if (ti.flags & TF_WHOLE) {
-                // the whole K of this segment was ours: round and store rows at their original positions
-                if (n < N) {
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m)
-                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
+                for (int i = 0; i < 8; ++i) {
+                    const int a = 8 * h + i;
+                    data[i] = make_uint4(0, 0, 0, 0);
+                    if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
                 }
-            } else if (ti.flags & TF_KB0NZ) {
-                // A piece that starts inside its segment -- always a CTA's FIRST piece: park the partial sum and raise
-                // this CTA's flag.  Nobody waits here: the barrier puts the 128 threads' stores before thread 0's
-                // release, which publishes them together with the flag.
-                float* dst = p.partials + (size_t)blockIdx.x * TOK * 128 + row;
 #pragma unroll
-                for (int m = 0; m < TOK; ++m)
-                    if (m < rows) dst[m * 128] = acc[m];
-                warrive(bar_esync);
-                if (!wwait(bar_esync, esync_phase)) return false;
-                esync_phase ^= 1u;
-                if (et == 0) st_release_gpu(p.flags + blockIdx.x, 1u);
-            } else {
-                // The head of a segment whose tail belongs to the following CTAs -- always a CTA's LAST piece, while
-                // the later pieces are parked by CTAs blockIdx.x + 1 .. c_last (each as its first piece).  Every thread
-                // waits for their flags itself (bounded; an acquire load, so its reads of the parked sums need no
-                // further fence), adds the sums in CTA order (deterministic) and stores.
-                const int n_others = ti.c_last - (int)blockIdx.x;
-                for (int c0 = 0; c0 < n_others; ++c0) {
-                    const unsigned* f = p.flags + blockIdx.x + 1 + c0;
-                    unsigned long long t_start = 0;
-                    for (unsigned it = 1; ld_acquire_gpu(f) == 0u; ++it) {
-                        if ((it & 63u) == 0) {
-                            if (*s_abort) break;
-                            const unsigned long long now = global_ns();
-                            if (t_start == 0) t_start = now;
-                            else if (now - t_start > WAIT_LIMIT_NS) { *s_abort = 1; latch_status(p.status, (int)MOQE_ERR_TIMEOUT); break; }
+                for (int i = 0; i < 8; ++i) {
+                    const int a = 8 * h + i, G = a >> 2, q = a & 3;       // chunk (G, q) of the k-block: k = 32G + 8q ..
+                    const uint32_t w[4] = {data[i].x, data[i].y, data[i].z, data[i].w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
+                        const int e = sigma_shift(bits, 4 * G + j);
+                        const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
+                        const float sum = lo + hi;
+                        S0 += sum;
+                        S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
+                        __half2 hh = __floats2half2_rn(lo, hi);
+                        const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
+                        hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
+                        o[j] = *reinterpret_cast<uint32_t*>(&hh);
+                    }
+                    // fragments at [slab][G][lane = 4 mm + q]
+                    sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
+                }
+            }
+            // sums at [slab][t = mm / 2][4]
+            float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
+            S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
+            S[2] = S0;
+        }
+        kbc += nkb;
+        if (kbc >= kb1) {
+            bool changed;
+            more = wk.next(s_pair, p, changed);
+            kbc = more ? wk.kb : 0;
+        }
+        return true;
+    };
+    // the first chunk is staged by the consumer and service warps together: one fetch latency instead of many
+    GvWalk swk;
+    swk.start();
+    bool s_changed, s_more = swk.next(s_pair, p, s_changed);
+    int s_kbc = s_more ? swk.kb : 0;
+    if (warp < GV_CONS + GV_SERV) {
+        stage_chunk(swk, s_kbc, s_more, 0, (GV_CONS + GV_SERV) * 32, tid);
+        asm volatile("bar.sync 1, %0;" ::"n"((GV_CONS + GV_SERV) * 32) : "memory");   // (the producer is already streaming)
+    }
+
+    if (warp == GV_CONS + GV_SERV) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint64_t once = l2_policy_evict_first();
+            GvWalk wk;
+            wk.start();
+            Ring ring;
+            bool changed, ok = true;
+            int issued = 0;
+            while (ok && wk.next(s_pair, p, changed)) {
+                const int v = wk.v, n = wk.run();
+                const uint32_t stride = (uint32_t)p.ex[v].tile_stride;
+                const int nt = 2 * wk.nt2;
+                const bool two = nt + 1 < p.NT1[v];
+                const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * stride;
+                const uint8_t* b = a + (size_t)wk.KB * stride;
+                for (int i = 0; i < n; ++i) {
+                    // Ramp-up: when all CTAs ask for a full ring at once, a CTA's first tile queues behind everybody's
+                    // ninth; so the first two stages go out alone and the rest follows once the first has landed.
+                    if (issued == 2 && !mbar_wait(bar_wfull, 0u, s_abort, p.status)) { ok = false; break; }
+                    ++issued;
+                    if (!mbar_wait(bar_wempty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)) { ok = false; break; }
+                    const uint32_t full = bar_wfull + 8 * ring.stage;
+                    const uint32_t dst = sbase + L::ring_off + ring.stage * stage_bytes;
+                    mbar_expect_tx(full, two ? 2 * stride : stride);
+                    bulk_load_once(dst, a, stride, full, once);
+                    if (two) bulk_load_once(dst + (stage_bytes >> 1), b, stride, full, once);
+                    a += stride; b += stride;
+                    ring.advance(nstg);
+                }
+            }
+        }
+    } else if (warp >= GV_CONS) {
+        // ------------------------------------------------------------------ service warps: token rows, one chunk ahead
+        const int st = tid - GV_CONS * 32;
+        for (int n = 1;; ++n) {
+            const int buf = n & 1;
+            if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_xempty + 8 * buf, (uint32_t)((n >> 1) - 1) & 1u, s_abort, p.status))) break;
+            const bool staged = stage_chunk(swk, s_kbc, s_more, n, GV_SERV * 32, st);
+            mbar_arrive(bar_xfull + 8 * buf);
+            if (!staged) break;
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        const int g = lane >> 2, t = lane & 3;
+        const int half = warp >> 3, blob = warp & 7;
+        const int slot16 = (t * 8 + (g ^ (2 * t))) * 16;          // this lane's 16-byte slot inside a 512-byte half blob
+        const uint32_t tile_base = sbase + L::ring_off + half * (stage_bytes >> 1);
+        Ring ring;
+        GvConst kc;
+        kc.init();
+        float fin[8];                                     // the running sums of the current piece: [token block][4]
+#pragma unroll
+        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+        float sc_r = 0.f, sc_r8 = 0.f, z_r = 0.f, z_r8 = 0.f;     // per-channel experts: scale / zero-point of rows g, g + 8
+        bool ok = true;
+
+        // One chunk of k-blocks of one piece, for a format fixed at compile time.
+        auto run_chunk = [&](auto tag, int nkb, int buf, bool active) {
+            constexpr int BITS = decltype(tag)::bits, NT = decltype(tag)::nt;
+            constexpr bool GROUPED = decltype(tag)::grouped, ASYM = decltype(tag)::asym;
+            const uint32_t xb0 = sbase + L::x_off + buf * GV_XBUF + lane * 16;
+            const float4* sS = reinterpret_cast<const float4*>(smem + L::s_off + buf * GV_SBUF) + t;
+            const uint32_t blob_off = blob * (BITS * 256);
+            const uint32_t meta_off = moqe_tile_bytes(BITS) + (blob * 16 + g) * 2;
+#pragma unroll 1
+            for (int kbl = 0; kbl < nkb; ++kbl) {
+                if (!__all_sync(0xffffffffu, mbar_wait_short(bar_wfull + 8 * ring.stage, ring.phase, s_abort, p.status))) { ok = false; return; }
+                if (active) {
+                    const uint32_t tile = tile_base + ring.stage * stage_bytes;
+                    float acc[NT][4], S0[NT][2];
+#pragma unroll
+                    for (int tb = 0; tb < NT; ++tb) {
+                        const float4 sv = sS[(kbl * NT + tb) * 4];
+                        acc[tb][0] = acc[tb][2] = sv.x;
+                        acc[tb][1] = acc[tb][3] = sv.y;
+                        S0[tb][0] = sv.z;
+                        S0[tb][1] = sv.w;
+                    }
+                    float s0 = sc_r, s8 = sc_r8, z0 = z_r, z8 = z_r8;
+                    if constexpr (GROUPED) {
+                        const uint32_t meta = tile + meta_off;
+                        s0 = __half2float(__ushort_as_half((unsigned short)lds16(meta)));
+                        s8 = __half2float(__ushort_as_half((unsigned short)lds16(meta + 16)));
+                        if constexpr (ASYM) {
+                            z0 = __uint_as_float(lds16(meta + 256) << 16);
+                            z8 = __uint_as_float(lds16(meta + 256 + 16) << 16);
                         }
                     }
-                    const float* src = p.partials + (size_t)(blockIdx.x + 1 + c0) * TOK * 128 + row;
-                    float part[TOK];
+                    tile_mma<BITS, NT>(kc, tile + blob_off, slot16, xb0 + ((kbl * NT * 4) << 9), acc);
+                    // the k-block is complete: scale and add
 #pragma unroll
-                    for (int m = 0; m < TOK; ++m) part[m] = m < rows ? __ldcg(src + m * 128) : 0.f;
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m) acc[m] += part[m];
-                }
-                // all 128 threads have seen the flags before any of them is cleared for the next call
-                warrive(bar_esync);
-                if (!wwait(bar_esync, esync_phase)) return false;
-                esync_phase ^= 1u;
-                if (*s_abort) return false;
-                for (int i = et; i < n_others; i += 128) p.flags[blockIdx.x + 1 + i] = 0u;
-                if (n < N) {
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m)
-                        if (m < rows) Y[(size_t)s_perm[j0 + m] * N + n] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[m]));
-                }
-            }
-            return true;
-        };
-        // Pieces before `upto` are complete as far as this warpgroup goes: hand its share over.
-        auto flush_to = [&](int upto) -> bool {
-            for (; flushed < upto; ++flushed) {
-                const uint32_t par = (uint32_t)flushed & 1u;
-                // every warpgroup has a slot of its own for its share, so none waits for another here -- only for the
-                // last warpgroup to have read the previous piece's slots
-                if (!wwait(bar_flushfree, par ^ 1u)) return false;
-                const bool mine = acc_piece == flushed;
-                float* slot = s_out + wg * (TOK * 128);
-                if (wg != NWG - 1) {
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m) slot[m * 128 + row] = mine ? acc[m] : 0.f;
-                }
-                warrive(bar_turn);
-                if (wg == NWG - 1) {
-                    // the last warpgroup adds the shares in warpgroup order (deterministic) once all have arrived
-                    if (!wwait(bar_turn, par)) return false;
-                    float total[TOK];
-#pragma unroll
-                    for (int m = 0; m < TOK; ++m) {
-                        float v = s_out[m * 128 + row];
-#pragma unroll
-                        for (int u = 1; u < NWG - 1; ++u) v += s_out[u * (TOK * 128) + m * 128 + row];
-                        total[m] = v + (mine ? acc[m] : 0.f);
+                    for (int tb = 0; tb < NT; ++tb) {
+                        if constexpr (ASYM) {
+                            fin[4 * tb + 0] = fmaf(s0, fmaf(-z0, S0[tb][0], acc[tb][0]), fin[4 * tb + 0]);
+                            fin[4 * tb + 1] = fmaf(s0, fmaf(-z0, S0[tb][1], acc[tb][1]), fin[4 * tb + 1]);
+                            fin[4 * tb + 2] = fmaf(s8, fmaf(-z8, S0[tb][0], acc[tb][2]), fin[4 * tb + 2]);
+                            fin[4 * tb + 3] = fmaf(s8, fmaf(-z8, S0[tb][1], acc[tb][3]), fin[4 * tb + 3]);
+                        } else {
+                            fin[4 * tb + 0] = fmaf(s0, acc[tb][0], fin[4 * tb + 0]);
+                            fin[4 * tb + 1] = fmaf(s0, acc[tb][1], fin[4 * tb + 1]);
+                            fin[4 * tb + 2] = fmaf(s8, acc[tb][2], fin[4 * tb + 2]);
+                            fin[4 * tb + 3] = fmaf(s8, acc[tb][3], fin[4 * tb + 3]);
+                        }
                     }
-                    warrive(bar_flushfree);
-                    if (!finalize(flushed, total)) return false;
                 }
-                if (mine) {
-#pragma unroll
-                    for (int i = 0; i < TOK; ++i) acc[i] = 0.f;
-                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_wempty + 8 * ring.stage);
+                ring.advance(nstg);
             }
-            return true;
         };
-        x_load(wg);
-        int stg = wg % nstg, a = wg % NA;            // ring stage and A buffer of tile t, kept incrementally
-        uint32_t wphase = (uint32_t)(wg / nstg) & 1u;
-        for (int t = wg; ok && t < T; t += NWG) {
-            const Tile ti(s_tile[t]);
-            const ExpertSm& ex = s_ex[ti.e];
-            // tile t - 6 is done, and so are all before it (MMAs are issued in tile order and a commit covers every
-            // earlier one): A buffer t % 6 and token-tile stage (t + 4) % 10 are free, and the group that ended two
-            // rounds ago (tile t - 8) can be drained without a wait of its own
-            // First of all the warpgroup takes its turn for the pieces before the one its tile of two rounds ago
-            // belongs to: all four warpgroups do this at the same distance behind their tiles and before they wait
-            // for anything else, so none of them can be waiting for a tile that another holds back while it waits
-            // for its turn.
-            if (!(ok = flush_to(ph0))) break;
-            if (!(ok = wait_done(t - NA))) break;
-            x_load(t + NWG);
-            drain(r0);
-            r0 = r1;
-            r1.t = -1;
-            if (!(ok = wwait(bar_wfull + 8 * stg, wphase))) break;
-            tc_fence_after();
-            const unsigned char* stage = smem + L::ring_off + stg * stage_bytes;
-            const int bits = ex.bits, group = ex.group, has_zeros = ex.has_zeros;
-            // zero-point of this row for the tile: the tile's own meta, the per-channel array, or 2^(bits-1)
-            float z = (float)(1 << (bits - 1));
-            if (has_zeros)
-                z = group == 0 ? __bfloat162float(p.ex[ti.e].zeros_pc[ti.nt * 128 + row])
-                               : __bfloat162float(moqe_tile_zeros(stage, bits, 0)[row]);
-            if (bits == 4) dequant_tile<4>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
-            else if (bits == 8) dequant_tile<8>(stage, row, pack_bf16x2(-z * 0.0001220703125f, -z * 0.0001220703125f), lane_taddr + a * 64);
-            else dequant_tile<3>(stage, row, pack_bf16x2(128.f + z, 128.f + z), lane_taddr + a * 64);
-            if (ti.ends()) {
-                // the scale of the group that ends with this tile; its accumulator is drained two rounds later
-                r1.t = t;
-                r1.g = ti.g;
-                r1.piece = ti.piece;
-                r1.s = (group == 0 ? __half2float(p.ex[ti.e].scales_pc[ti.nt * 128 + row])
-                                     : __half2float(moqe_tile_scales(stage, bits, has_zeros, 0)[row])) *
-                         (bits == 8 ? W8_PRESCALE : 1.f);
+
+        for (int n = 0; ok; ++n) {
+            const int buf = n & 1;
+            if (n > 0 && !__all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * buf, (uint32_t)((n - 1) >> 1) & 1u, s_abort, p.status))) break;
+            const ChunkDesc* d = s_desc + buf;
+            if (!d->valid) break;
+            const int v = d->v, nt2 = d->nt2, kbc = d->kbc, nkb = d->nkb, kb0 = d->kb0, kb1 = d->kb1;
+            const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+            const int bits = p.ex[v].bits, group = p.ex[v].group, has_zeros = p.ex[v].has_zeros;
+            const int nt = 2 * nt2 + half;
+            const bool active = nt < p.NT1[v];
+            const int n_r = nt * 128 + blob * 16 + g;
+            if (kbc == kb0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+                if (group == 0 && active) {
+                    sc_r = __half2float(p.ex[v].scales_pc[n_r]);
+                    sc_r8 = __half2float(p.ex[v].scales_pc[n_r + 8]);
+                    if (has_zeros) {
+                        z_r = __bfloat162float(p.ex[v].zeros_pc[n_r]);
+                        z_r8 = __bfloat162float(p.ex[v].zeros_pc[n_r + 8]);
+                    }
+                }
             }
-            warrive(bar_wempty + 8 * stg);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");      // this tile's token rows have landed
-            fence_proxy_async();
-            tmem_st_wait();
-            tc_fence_before();
-            warrive(bar_afull + 8 * a);
-            ph0 = ph1;
-            ph1 = ti.piece;
-            last_t = t;
-            stg += NWG;
-            while (stg >= nstg) { stg -= nstg; wphase ^= 1u; }
-            a += NWG;
-            while (a >= NA) a -= NA;
+            // dispatch on the format (uniform over the CTA)
+            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : 2)) * 8 + (rows > 8 ? 4 : 0) + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
+            switch (fmt) {
+#define GV_CASE(B, BI, NTV, GR, AS) \
+                case BI * 8 + (NTV - 1) * 4 + GR * 2 + AS: run_chunk(GvTag<B, NTV, GR != 0, AS != 0>{}, nkb, buf, active); break;
+#define GV_CASES(B, BI) GV_CASE(B, BI, 1, 0, 0) GV_CASE(B, BI, 1, 0, 1) GV_CASE(B, BI, 1, 1, 0) GV_CASE(B, BI, 1, 1, 1) \
+                        GV_CASE(B, BI, 2, 0, 0) GV_CASE(B, BI, 2, 0, 1) GV_CASE(B, BI, 2, 1, 0) GV_CASE(B, BI, 2, 1, 1)
+                GV_CASES(4, 0)
+                GV_CASES(8, 1)
+                GV_CASES(3, 2)
+#undef GV_CASES
+#undef GV_CASE
+                default: break;
+            }
+            if (!ok) break;
+
+            if (kbc + nkb == kb1 && active) {
+                // ---- the piece is complete
+                const int NT = rows > 8 ? 2 : 1;
+                const int KB = p.KB[v], N = p.N[v];
+                uint16_t* Y = p.Y[v];
+                auto store_rows = [&]() {
+#pragma unroll
+                    for (int tb = 0; tb < 2; ++tb) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int m = 8 * tb + 2 * t + (j & 1), nn = n_r + (j >> 1) * 8;
+                            if (tb < NT && m < rows && nn < N)
+                                Y[(size_t)s_perm[row0 + m] * N + nn] = __bfloat16_as_ushort(__float2bfloat16_rn(fin[4 * tb + j]));
+                        }
+                    }
+                };
+                if (kb0 == 0 && kb1 == KB) {
+                    store_rows();
+                } else {
+                    // part of a segment: park this warp's sums, announce, and add everything up if this was the last arrival
+                    const long long C = *s_C, base = s_base[v];
+                    const int G = *s_G, wv = p.w[v];
+                    const int c_a = (int)(((base + (long long)(nt2 * KB) * wv) * G) / C);
+                    const int c_b = (int)(((base + (long long)(nt2 * KB + KB - 1) * wv) * G) / C);
+                    float* slot = p.partials + (size_t)(2 * blockIdx.x + (kb0 == 0 ? 1 : 0)) * GV_SLOT_FLOATS;
+#pragma unroll
+                    for (int tb = 0; tb < 2; ++tb)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (tb < NT) __stcg(slot + ((warp * 2 + tb) * 4 + j) * 32 + lane, fin[4 * tb + j]);
+                    __syncwarp();
+                    unsigned arrived = 0;
+                    if (lane == 0) {
+                        __threadfence();
+                        arrived = atomicAdd(p.counters + c_a * GV_CONS + warp, 1u);
+                    }
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    if (arrived == (unsigned)(c_b - c_a)) {
+                        __threadfence();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+                        for (int c = c_a; c <= c_b; ++c) {
+                            const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
+#pragma unroll
+                            for (int tb = 0; tb < 2; ++tb)
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    if (tb < NT) fin[4 * tb + j] += __ldcg(src + ((warp * 2 + tb) * 4 + j) * 32 + lane);
+                        }
+                        store_rows();
+                        if (lane == 0) p.counters[c_a * GV_CONS + warp] = 0u;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_xempty + 8 * buf);
         }
-        if (ok) ok = flush_to(ph0);
-        // the MMAs of this warpgroup's last tile (hence of all earlier ones) -- not of an older tile: a barrier of the
-        // ring tells apart only tiles that are less than 8 apart
-        if (ok && last_t >= 0) ok = wait_done(last_t);
-        if (ok) {
-            drain(r0);
-            ok = flush_to(ph1);
-        }
-        if (ok) {
-            drain(r1);
-            flush_to(NP);
-        }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------------------------- teardown
-    tc_fence_before();
     __syncthreads();
     if (*s_abort) {
         // let bulk copies that may still be in flight land before the shared memory is released
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
-        __syncthreads();
-    }
-    if (warp == MMA_WARP) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
-int g_dec_sm_count = 0;
 int dec_sm_count() {
-    if (!g_dec_sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_dec_sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (g_dec_sm_count <= 0) g_dec_sm_count = 148;
-    }
-    return g_dec_sm_count;
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
 }
 
-constexpr int DEC_MAX_GRID = 256;             // bound on CTAs the partial slots are sized for
+// relative cost of one super-tile in the work split, by code width
+int g_dec_cost[9] = {0, 0, 0, 10, 10, 0, 0, 0, 10};
 
-// Relative cost of one packed tile in the work split (0 = its bytes).  Measured: an 8-bit tile is paced by its
-// 16 KiB of HBM traffic, the narrower ones by the unpacking arithmetic, which is dearer per tile.
-int g_dec_tile_cost[9] = {0, 0, 0, 11, 10, 0, 0, 0, 8};
-
-}  // namespace
-
-void decode_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost >= 0) g_dec_tile_cost[bits] = cost; }
-
-namespace {
-// the work split of one call over `nl` layers of E experts each (pair index = layer * E + expert): costs, grid, and
-// whether every CTA's tiles fit its tile table
-bool decode_plan(const moqe_expert* const* ex, int nl, int E, DecSched& s, int& grid) {
-    if (nl * E > MOQE_MAX_EXPERTS) return false;
-    s.E = nl * E;
-    s.C = 0;
-    int wmax = 1, wmin = 1 << 30;
-    for (int v = 0; v < nl * E; ++v) {
-        const int cost = g_dec_tile_cost[ex[v]->bits];
-        s.TT[v] = (ex[v]->Np / 128) * (ex[v]->Kp / 128);
-        s.w[v] = cost > 0 ? cost : ex[v]->dev().tile_stride / 256;
-        s.C += (long long)s.TT[v] * s.w[v];
-        wmax = s.w[v] > wmax ? s.w[v] : wmax;
-        wmin = s.w[v] < wmin ? s.w[v] : wmin;
-    }
-    // every CTA's cost share must be at least one tile of the dearest kind, so that every CTA between the owners of
-    // a segment's first and last tile really owns a tile of it (the reduction counts them)
-    grid = dec_sm_count();
-    if (grid > DEC_MAX_GRID) grid = DEC_MAX_GRID;
-    const long long work_items = s.C / wmax;
-    if (work_items < grid) grid = work_items < 1 ? 1 : (int)work_items;
-    s.G = grid;
-    return s.C / grid / wmin + nl * E + 2 <= MAX_TILES;
-}
-bool formats_ok(const moqe_expert* const* ex, int n) {
-    for (int v = 0; v < n; ++v)
+bool dec_formats_ok(const moqe_expert* const* ex, int n) {
+    for (int v = 0; v < n; ++v) {
+        if (ex[v]->bits != 3 && ex[v]->bits != 4 && ex[v]->bits != 8) return false;
         if (ex[v]->group != 0 && (ex[v]->group < 128 || ex[v]->group % 128 != 0)) return false;
+    }
     return true;
 }
+
 }  // namespace
 
-bool decode_supported(int M, const moqe_expert* const* ex, int E) { return decode_supported_multi(M, ex, 1, E); }
+void decode_set_tile_cost(int bits, int cost) { if (bits >= 0 && bits <= 8 && cost > 0) g_dec_cost[bits] = cost; }
 
 bool decode_supported_multi(int M, const moqe_expert* const* ex, int nl, int E) {
-    if (M > DECODE_MAX_ROWS || nl < 1 || nl * E > MOQE_MAX_EXPERTS || !formats_ok(ex, nl * E)) return false;
-    DecSched s;
-    int grid;
-    return decode_plan(ex, nl, E, s, grid);
+    return M <= DECODE_MAX_ROWS && nl >= 1 && nl * E <= MOQE_MAX_EXPERTS && dec_formats_ok(ex, nl * E);
 }
 
-size_t decode_zero_bytes(int M, int Np) {
+size_t decode_zero_bytes(int M) { return M > DECODE_MAX_ROWS ? 0 : (size_t)GV_MAX_GRID * GV_CONS * sizeof(uint32_t); }
+
+size_t decode_workspace_bytes(int M) {
     if (M > DECODE_MAX_ROWS) return 0;
-    (void)Np;
-    return (size_t)DEC_MAX_GRID * sizeof(uint32_t);
-}
-
-size_t decode_workspace_bytes(int M, int Np, int E) {
-    (void)E;
-    if (M > DECODE_MAX_ROWS) return 0;
-    const size_t counters = (decode_zero_bytes(M, Np) + 255) / 256 * 256;
-    const size_t partials = (size_t)DEC_MAX_GRID * TOK * 128 * sizeof(float);
-    return counters + partials;
-}
-
-moqe_status launch_qgemm_decode(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
-                                const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
-    (void)N; (void)K;
-    return launch_qgemm_decode_multi(&X, M, 1, ex, E, &Y, perm, offsets, ws, ws_bytes, st);
+    return (decode_zero_bytes(M) + 255) / 256 * 256 + (size_t)GV_MAX_GRID * 2 * GV_SLOT_FLOATS * sizeof(float);
 }
 
 // nl layers that share the routing; ex[l * E + e] = expert e of layer l; X[l] / Y[l] the layer's input / output
 moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
-                                      void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
-                                      size_t ws_bytes, cudaStream_t st) {
+                                    void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
+                                    size_t ws_bytes, cudaStream_t st) {
     if (M == 0) return MOQE_OK;
     if (!decode_supported_multi(M, ex, nl, E)) return MOQE_ERR_UNSUPPORTED;
-    DecParams p;
-    int grid = 1;
-    if (!decode_plan(ex, nl, E, p.sched, grid)) return MOQE_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < decode_workspace_bytes(M)) return MOQE_ERR_WORKSPACE;
+    GvParams p;
     for (int l = 0; l < nl; ++l)
         for (int e = 0; e < E; ++e) {
             const int v = l * E + e;
@@ -735,25 +704,24 @@ moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const
             p.N[v] = ex[v]->N;
             p.K[v] = ex[v]->K;
             p.KB[v] = ex[v]->Kp / 128;
+            p.NT1[v] = ex[v]->Np / 128;
             p.rexp[v] = e;
+            p.w[v] = g_dec_cost[ex[v]->bits];
         }
-    if (!ws || ws_bytes < decode_workspace_bytes(M, ex[0]->Np, E)) return MOQE_ERR_WORKSPACE;
-    p.flags = (uint32_t*)ws;
-    p.partials = (float*)((char*)ws + (decode_zero_bytes(M, ex[0]->Np) + 255) / 256 * 256);
+    p.counters = (uint32_t*)ws;
+    p.partials = (float*)((char*)ws + (decode_zero_bytes(M) + 255) / 256 * 256);
     p.perm = perm;
     p.offsets = offsets;
     p.M = M;
     p.R = E;
+    p.P = nl * E;
     p.status = device_status_word();
-    static bool attr_set = false;
-    cudaError_t err = cudaSuccess;
-    if (!attr_set) {
-        err = cudaFuncSetAttribute(qgemm_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DecSmem::dyn_bytes);
-        attr_set = (err == cudaSuccess);
-    }
+    int grid = dec_sm_count();
+    if (grid > GV_MAX_GRID) grid = GV_MAX_GRID;
+    cudaError_t err = cudaFuncSetAttribute(qgemm_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GvSmem::dyn_bytes);
     if (err == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(DEC_THREADS); cfg.dynamicSmemBytes = DecSmem::dyn_bytes; cfg.stream = st;
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GV_THREADS); cfg.dynamicSmemBytes = GvSmem::dyn_bytes; cfg.stream = st;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         at[0].val.programmaticStreamSerializationAllowed = 1;

@@ -77,3 +77,101 @@ def test_workload_at_full_size(name):
         assert_close(got, ref, f"{name}/{layer.name}")
         del experts, What, Xd, Y, ws
         torch.cuda.empty_cache()
+
+
+def test_decode_block_in_the_launches_the_bench_times():
+    """llama7b_decode exactly as bench.py sends it down: one sort, then q/k/v in ONE launch and gate/up in ONE launch
+    (moqe_routed_qgemm_sorted_multi) at M = 16 and full layer sizes; every element of every layer against the oracle,
+    twice on the same workspace (the arrival counters must come back to zero by themselves), same bits both times."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import dev, bf16_to_torch, torch_to_bits, assert_close
+    w = wl.get("llama7b_decode")
+    E = w.n_experts
+    logits = _logits(w)
+    ids = moqe.moqe_route(torch.from_numpy(logits).to(dev()))
+    ids_ref = oracle.route(logits)
+    byname = {l.name: l for l in w.layers}
+    for group in (("q_proj", "k_proj", "v_proj"), ("gate_proj", "up_proj")):
+        layers = [byname[n] for n in group]
+        off = w.row_offsets(layers[0])
+        M = int(off[-1])
+        row_ids = moqe.moqe_expand_ids(ids, torch.from_numpy(off).to(dev()), M)
+        row_ids_ref = oracle.expand_ids(ids_ref, off)
+        _, perm, offsets = moqe.moqe_permute(None, row_ids, E)
+        Xs, Ys, gpus, refs = [], [], [], []
+        for layer in layers:
+            W, X = wl.layer_inputs(w, layer)
+            Wd = torch.from_numpy(W).to(dev())
+            experts, What = [], []
+            for sp in w.experts:
+                experts.append(moqe.moqe_quantize_rtn(Wd, sp.bits, sp.group, sp.sym))
+                c, s, z = oracle.quantize_rtn(W, sp.bits, sp.group, sp.sym)
+                What.append(oracle.dequantize(c, s, z, sp.group))
+            del Wd
+            refs.append(oracle.routed_gemm(X, row_ids_ref, What))
+            del What
+            Xs.append(bf16_to_torch(X))
+            Ys.append(torch.full((M, layer.N), float("nan"), dtype=torch.bfloat16, device=dev()))
+            gpus.append(experts)
+        ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, layers[0].N, layers[0].K, E))
+        moqe.moqe_routed_qgemm_workspace_clear(ws, M, layers[0].N, layers[0].K, E)
+        bits = None
+        for rep in range(2):
+            for Y in Ys:
+                Y.fill_(float("nan"))
+            moqe.moqe_routed_qgemm_sorted_multi(Xs, perm, offsets, gpus, Ys, ws)
+            assert moqe.moqe_async_status() == moqe.OK
+            got = [torch_to_bits(Y) for Y in Ys]
+            for name, g, r in zip(group, got, refs):
+                assert_close(g, r, f"{name} in the {'+'.join(group)} launch")
+            if bits is not None:
+                assert all(np.array_equal(a, b) for a, b in zip(bits, got))
+            bits = got
+        del Xs, Ys, gpus, refs, ws
+        torch.cuda.empty_cache()
+
+
+def test_prefill_every_expert_gets_rows():
+    """llama7b_prefill at full size with a routing draw that gives every expert at least one sequence (the bench seed's
+    draw leaves the 4-bit expert idle): q_proj and down_proj, 64 sampled rows per expert plus every segment's first and
+    last row, all N columns, full K."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import dev, bf16_to_torch, torch_to_bits, assert_close, sample_rows
+    w = wl.get("llama7b_prefill")
+    E = w.n_experts
+    seed = wl.BASE_SEED + 1000
+    logits = wl.router_logits(w, seed=seed)
+    ids_ref = oracle.route(logits)
+    assert len(set(ids_ref.tolist())) == E, ids_ref
+    ids = moqe.moqe_route(torch.from_numpy(logits).to(dev()))
+    assert np.array_equal(ids.cpu().numpy(), ids_ref)
+    byname = {l.name: l for l in w.layers}
+    for lname in ("q_proj", "down_proj"):
+        layer = byname[lname]
+        W, X = wl.layer_inputs(w, layer)
+        M = X.shape[0]
+        off = w.row_offsets(layer)
+        row_ids = moqe.moqe_expand_ids(ids, torch.from_numpy(off).to(dev()), M)
+        row_ids_ref = oracle.expand_ids(ids_ref, off)
+        _, perm, offsets = moqe.moqe_permute(None, row_ids, E)
+        _, off_ref, perm_ref, _ = oracle.permutation(row_ids_ref, E)
+        assert np.array_equal(perm.cpu().numpy(), perm_ref)
+        Wd = torch.from_numpy(W).to(dev())
+        experts, What = [], []
+        for sp in w.experts:
+            experts.append(moqe.moqe_quantize_rtn(Wd, sp.bits, sp.group, sp.sym))
+            c, s, z = oracle.quantize_rtn(W, sp.bits, sp.group, sp.sym)
+            What.append(oracle.dequantize(c, s, z, sp.group))
+        del Wd
+        Xd = bf16_to_torch(X)
+        Y = torch.empty((M, layer.N), dtype=torch.bfloat16, device=dev())
+        ws = moqe.alloc_workspace(moqe.moqe_routed_qgemm_workspace(M, layer.N, layer.K, E))
+        moqe.moqe_routed_qgemm_workspace_clear(ws, M, layer.N, layer.K, E)
+        moqe.moqe_routed_qgemm_sorted(Xd, perm, offsets, experts, Y, ws)
+        assert moqe.moqe_async_status() == moqe.OK
+        rows = sample_rows(off_ref, 64, 11, perm_ref)
+        ref = oracle.routed_gemm(X, row_ids_ref, What, rows=rows)
+        got = torch_to_bits(Y[torch.from_numpy(rows.astype(np.int64)).to(dev())])
+        assert_close(got, ref, f"llama7b_prefill/{lname}, every expert with rows")
+        del experts, What, Xd, Y, ws
+        torch.cuda.empty_cache()

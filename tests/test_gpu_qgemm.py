@@ -77,7 +77,7 @@ DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True)
 @pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (13, 136, 2304), (16, 1000, 640),
                                    (7, 4096, 1024), (16, 512, 11008), (9, 128, 32768)])
 def test_decode_kernel_all_formats(M, N, K):
-    """The tcgen05 decode kernel (path 5: at most 16 rows, per-channel experts or groups of >= 128 k): every such
+    """The decode kernel (path 5: at most 16 rows, per-channel experts or groups of >= 128 k): every such
     format as its own expert, ragged N, K not a multiple of 128, split K with several contributors per segment
     (dozens in the last, one-tile-wide case, where most CTAs hold nothing but the middle of a segment), an expert
     that gets no rows."""
@@ -154,13 +154,13 @@ def test_decode_kernel_refuses_what_it_cannot_take():
         moqe.moqe_routed_qgemm(bf16_to_torch(X), torch.zeros(4, dtype=torch.int32, device=dev()), gpu, path=moqe.PATH_DECODE)
 
 
-@pytest.mark.parametrize("path", [1, 3, 4])
+@pytest.mark.parametrize("path", [1, 3, 4, 5])
 def test_exact_integer_case_on_gpu(path):
     """On-grid W8 weights with power-of-two scale and small-integer activations: the exact int64 product."""
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts
     rs = np.random.default_rng(55)
-    M, N, K = 24, 256, 512
+    M, N, K = (16 if path == 5 else 24), 256, 512
     q = rs.integers(-127, 128, size=(N, K))
     q[:, 0], q[:, 1] = 127, -127
     s0 = 2.0 ** -9
@@ -173,20 +173,23 @@ def test_exact_integer_case_on_gpu(path):
     assert np.array_equal(Y, wl.f32_to_bf16_bits(exact.astype(np.float32)))
 
 
-@pytest.mark.parametrize("path", [1, 3, 4])
+@pytest.mark.parametrize("path", [1, 3, 4, 5])
 def test_degenerate_batches(path):
+    """All rows to one expert, a shuffled batch, M = 0, ids outside [0, E) -- on every kernel; the decode kernel
+    (path 5) takes batches of at most 16 rows."""
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, assert_close, dev, bf16_to_torch
     N, K = 256, 512
+    Mb = 16 if path == 5 else 40
     W = wl.weights_f32("deg", N, K)
     specs = [(8, 0, True), (4, 128, False), (3, 128, False)]
     gpu, What, _ = build_experts(W, specs)
     # all rows to one expert == that expert alone (one expert per sample)
-    X = wl.activations_bf16("deg/X", 40, K)
+    X = wl.activations_bf16("deg/X", Mb, K)
     for e in range(3):
-        ids = np.full(40, e, np.int32)
+        ids = np.full(Mb, e, np.int32)
         Y, st = _run(X, ids, gpu, path)
-        Y1, _ = _run(X, np.zeros(40, np.int32), [gpu[e]], path)
+        Y1, _ = _run(X, np.zeros(Mb, np.int32), [gpu[e]], path)
         assert st == moqe.OK
         if path == 1:
             # the streaming kernel splits K at points that depend on the set of experts in the call, so the
@@ -197,9 +200,9 @@ def test_degenerate_batches(path):
         assert_close(Y, oracle.routed_gemm(X, ids, What), f"single expert {e}")
     # batch shuffle: rows move with their inputs, bit for bit
     rs = np.random.default_rng(3)
-    ids = rs.integers(0, 3, size=40).astype(np.int32)
+    ids = rs.integers(0, 3, size=Mb).astype(np.int32)
     Y, _ = _run(X, ids, gpu, path)
-    p = rs.permutation(40)
+    p = rs.permutation(Mb)
     Yp, _ = _run(X[p], ids[p], gpu, path)
     assert np.array_equal(Yp, Y[p])
     # M = 0
@@ -208,12 +211,41 @@ def test_degenerate_batches(path):
     assert Y0.shape == (0, N)
     # invalid ids: zero rows + latched status, other rows unaffected
     bad = ids.copy()
-    bad[[3, 17]] = [7, -2]
+    bad[[3, Mb - 3]] = [7, -2]
     Yb, st = _run(X, bad, gpu, path)
     assert st == moqe.ERR_EXPERT_ID
-    assert np.all(Yb[[3, 17]] == 0)
-    keep = np.setdiff1d(np.arange(40), [3, 17])
-    assert np.array_equal(Yb[keep], Y[keep])
+    assert np.all(Yb[[3, Mb - 3]] == 0)
+    keep = np.setdiff1d(np.arange(Mb), [3, Mb - 3])
+    if path in (1, 5):
+        # the split-K kernels place their split points by the rows each expert received, so taking two rows
+        # out may change the fp32 summation order (not the value within tolerance) of the others
+        assert_close(Yb[keep], Y[keep], "rows beside the invalid ones")
+    else:
+        assert np.array_equal(Yb[keep], Y[keep])
+    # a single row, and a whole batch, on one expert of several: the untouched experts must cost nothing and
+    # the result must be that expert's
+    for Ms in (1, Mb):
+        ids1 = np.full(Ms, 2, np.int32)
+        Ys, st = _run(X[:Ms], ids1, gpu, path)
+        assert st == moqe.OK
+        assert_close(Ys, oracle.routed_gemm(X[:Ms], ids1, What), f"{Ms} rows on expert 2")
+
+
+def test_tcgen05_kernel_full_token_tiles_every_element():
+    """The tcgen05 kernel with 256-token tiles (path 4): 1536 rows over three experts -- several full token tiles and a
+    ragged one per expert, three channel tiles, eight k-blocks -- every element against the oracle."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close
+    M, N, K = 1536, 384, 1024
+    W = wl.weights_f32("tc/full", N, K)
+    X = wl.activations_bf16("tc/full/X", M, K)
+    gpu, What, _ = build_experts(W, [(8, 0, True), (4, 128, False), (3, 128, False)])
+    ids = np.repeat(np.array([0, 1, 2, 1, 0, 2], np.int32), [600, 300, 200, 212, 24, 200])
+    assert ids.size == M
+    for path in (3, 4):
+        Y, st = _run(X, ids, gpu, path)
+        assert st == moqe.OK
+        assert_close(Y, oracle.routed_gemm(X, ids, What), f"path {path}, M{M} N{N} K{K}")
 
 
 def test_argument_errors():
