@@ -184,8 +184,11 @@ MOQE_API moqe_status moqe_permute_static(const void* X_bf16, const int32_t* row_
  * moqe_routed_qgemm_workspace(M, N, K, E) bytes, contents irrelevant on entry;
  * calls that share a workspace must not overlap on the device.
  * Decode batches (at most 16 rows, experts per-channel or with groups of 128 k or more) stream each touched
- * expert's packed weights once through the tcgen05 decode kernel (TMEM-operand MMAs, stream-K split); other
- * small batches take the split-K mma.sync streaming kernel; large batches run the persistent tcgen05 grouped GEMM.
+ * expert's packed weights once through the decode kernel (bulk-copy ring, warp-level MMAs on fp16 operands,
+ * stream-K split that follows the routing: experts without rows cost nothing).  That kernel converts the bf16
+ * activations to fp16: values with |x| > 65504 are outside its domain (they become infinities); every other
+ * kernel takes the whole bf16 range.  Other small batches take the split-K mma.sync streaming kernel; large
+ * batches run the persistent tcgen05 grouped GEMM.
  * ------------------------------------------------------------------------- */
 MOQE_API size_t moqe_routed_qgemm_workspace(int M, int N, int K, int E);
 MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_ids, int M,
@@ -194,7 +197,7 @@ MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_id
 
 /* Same, with the kernel chosen by the caller (testing / measurement):
  * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM (automatic
- * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles, 5 = tcgen05 decode kernel
+ * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles, 5 = decode kernel
  * (MOQE_ERR_UNSUPPORTED if the batch has more than 16 rows or an expert has groups narrower than 128 k). */
 MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
                                    const moqe_expert* const* h_experts, int E, void* Y_bf16,
@@ -237,11 +240,17 @@ MOQE_API const char* moqe_status_str(moqe_status s);
  *   "stream_tile_cost_w8" / "_w4" / "_w3" : relative cost of one packed 128x128 tile of
  *                            that bit-width in the streaming kernel's work split
  *                            (defaults 8 / 8 / 8).
- *   "decode_tile_cost_w8" / "_w4" / "_w3" : the same for the tcgen05 decode kernel
- *                            (defaults 8 / 10 / 11; 0 = the tile's bytes).
+ *   "decode_tile_cost_w8" / "_w4" / "_w3" : the same for the decode kernel (defaults 10 / 10 / 10).
  *   "auto_decode"          : whether path 0 takes the decode kernel where it applies (default 1).
  * Unknown key: MOQE_ERR_UNSUPPORTED. */
 MOQE_API moqe_status moqe_tune(const char* key, int value);
+
+/* Self-test of the bounded waits every kernel of this library uses (no counterpart in the paper): launches one
+ * small kernel whose only thread waits, with a limit of `limit_us` microseconds (1 .. 1 000 000), on an mbarrier
+ * nobody ever arrives on.  The wait must give up by itself: the kernel then writes 2 to *d_returned (device int;
+ * 1 would mean the barrier completed), latches MOQE_ERR_TIMEOUT in the device status word -- read and cleared by
+ * the next moqe_async_status -- and returns; the context stays usable and later calls work as usual. */
+MOQE_API moqe_status moqe_selftest_timeout(unsigned limit_us, int* d_returned, void* stream);
 
 /* Number of kernels this library has launched so far in this process. */
 MOQE_API unsigned long long moqe_launch_count(void);

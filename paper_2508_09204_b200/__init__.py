@@ -27,7 +27,7 @@ EXPORTED = (
     "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
     "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
-    "moqe_status_str", "moqe_launch_count", "moqe_tune",
+    "moqe_status_str", "moqe_launch_count", "moqe_tune", "moqe_selftest_timeout",
 )
 
 
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
         L.moqe_status_str.argtypes = [i32]
         L.moqe_status_str.restype = C.c_char_p
         L.moqe_tune.argtypes = [C.c_char_p, i32]
+        L.moqe_selftest_timeout.argtypes = [C.c_uint, vp, vp]
         L.moqe_launch_count.argtypes = []
         L.moqe_launch_count.restype = C.c_ulonglong
         _lib = L
@@ -304,6 +305,13 @@ def moqe_async_status() -> int:
 
 def moqe_tune(key: str, value: int) -> None:
     _check(lib().moqe_tune(key.encode(), int(value)), "moqe_tune")
+
+
+def moqe_selftest_timeout(limit_us: int = 1000) -> int:
+    """Runs the bounded-wait self-test; returns what the kernel wrote (2 = the wait gave up by itself)."""
+    out = torch.zeros(1, dtype=torch.int32, device=torch.device("cuda", torch.cuda.current_device()))
+    _check(lib().moqe_selftest_timeout(int(limit_us), out.data_ptr(), _stream()), "moqe_selftest_timeout")
+    return out
 
 
 def moqe_launch_count() -> int:

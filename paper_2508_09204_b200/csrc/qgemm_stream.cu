@@ -611,15 +611,11 @@ int pick_ntmax(int M) { return M <= 8 ? 1 : (M <= 16 ? 2 : 4); }
 
 constexpr int MAX_GRID = 512;                 // bound on resident CTAs the partial slots are sized for
 
-int g_sm_count = 0;
-int sm_count() {
-    if (!g_sm_count) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (g_sm_count <= 0) g_sm_count = 148;
-    }
-    return g_sm_count;
+int sm_count() {                              // of the current device (asked every time: a process may drive several)
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
 }
 
 // relative cost of one packed tile in the work split.  Measured: a tile costs about the same time whatever its
@@ -694,12 +690,8 @@ moqe_status launch_qgemm_stream(const void* X, int M, int N, int K, const moqe_e
     cudaError_t err = cudaSuccess;
 #define MOQE_LAUNCH(NT)                                                                                           \
     do {                                                                                                          \
-        static bool attr_set = false;                                                                             \
         const int smem = StreamSmem<NT>::dyn_bytes;                                                               \
-        if (!attr_set) {                                                                                          \
-            err = cudaFuncSetAttribute(qgemm_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); \
-            attr_set = (err == cudaSuccess);                                                                      \
-        }                                                                                                         \
+        err = cudaFuncSetAttribute(qgemm_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);   \
         if (err == cudaSuccess) {                                                                                 \
             cudaLaunchConfig_t cfg = {};                                                                          \
             cfg.gridDim = dim3(grid); cfg.blockDim = dim3(STREAM_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st; \

@@ -482,20 +482,13 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
     int grid = (int)(max_tiles < sms ? max_tiles : sms);
     cudaError_t err;
     if (tn == 256) {
-        static bool attr = false;
-        if (!attr) {
-            if (cudaFuncSetAttribute(qgemm_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<256>::dyn_bytes) != cudaSuccess)
-                return MOQE_ERR_CUDA;
-            attr = true;
-        }
+        // (set at every launch: the attribute belongs to the current device, and the call is cheap)
+        if (cudaFuncSetAttribute(qgemm_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<256>::dyn_bytes) != cudaSuccess)
+            return MOQE_ERR_CUDA;
         qgemm_tc_kernel<256, true><<<grid, TC_THREADS, Smem<256>::dyn_bytes, st>>>(p, tmap, tmap_x);
     } else {
-        static bool attr = false;
-        if (!attr) {
-            if (cudaFuncSetAttribute(qgemm_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::dyn_bytes) != cudaSuccess)
-                return MOQE_ERR_CUDA;
-            attr = true;
-        }
+        if (cudaFuncSetAttribute(qgemm_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::dyn_bytes) != cudaSuccess)
+            return MOQE_ERR_CUDA;
         qgemm_tc_kernel<128, false><<<grid, TC_THREADS, Smem<128>::dyn_bytes, st>>>(p, tmap, tmap_x);
     }
     err = cudaGetLastError();

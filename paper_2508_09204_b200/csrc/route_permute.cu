@@ -123,15 +123,29 @@ __global__ void __launch_bounds__(SORT_THREADS) sort_hist_kernel(const int32_t* 
     if (threadIdx.x <= E) block_tot[(size_t)blockIdx.x * MAXB + threadIdx.x] = s_tot[threadIdx.x];
 }
 
-// (2) exclusive scan in (bucket-major, block-minor) order; block_tot becomes the base slot of (block, bucket)
-__global__ void sort_scan_kernel(int32_t* __restrict__ block_tot, int nblk, int E, int32_t* __restrict__ offsets) {
+// (2) exclusive scan in (bucket-major, block-minor) order; block_tot becomes the base slot of (block, bucket).
+// One warp per bucket: the lanes read 32 consecutive blocks' totals, scan them with shuffles and carry the running
+// sum to the next 32 (a serial walk over all blocks costs two dependent global round trips per block).
+__global__ void __launch_bounds__(1024) sort_scan_kernel(int32_t* __restrict__ block_tot, int nblk, int E,
+                                                              int32_t* __restrict__ offsets) {
     __shared__ int s_sum[MAXB];
     __shared__ int s_off[MAXB + 1];
-    int b = threadIdx.x;
-    if (b <= E) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int b = warp; b <= E; b += 32) {
         int run = 0;
-        for (int i = 0; i < nblk; ++i) { int c = block_tot[(size_t)i * MAXB + b]; block_tot[(size_t)i * MAXB + b] = run; run += c; }
-        s_sum[b] = run;
+        for (int i0 = 0; i0 < nblk; i0 += 32) {
+            const int i = i0 + lane;
+            const int c = i < nblk ? block_tot[(size_t)i * MAXB + b] : 0;
+            int incl = c;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += o;
+            }
+            if (i < nblk) block_tot[(size_t)i * MAXB + b] = run + incl - c;
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) s_sum[b] = run;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -139,9 +153,10 @@ __global__ void sort_scan_kernel(int32_t* __restrict__ block_tot, int nblk, int 
         for (int i = 0; i <= E; ++i) { s_off[i] = run; run += s_sum[i]; }
     }
     __syncthreads();
-    if (b <= E) {
-        offsets[b] = s_off[b];
-        for (int i = 0; i < nblk; ++i) block_tot[(size_t)i * MAXB + b] += s_off[b];
+    for (int b = warp; b <= E; b += 32) {
+        const int off = s_off[b];
+        if (lane == 0) offsets[b] = off;
+        for (int i = lane; i < nblk; i += 32) block_tot[(size_t)i * MAXB + b] += off;
     }
 }
 
@@ -236,7 +251,7 @@ moqe_status launch_sort(const int32_t* row_ids, int M, int E, int32_t* perm, int
     int nblk = (M + SORT_THREADS - 1) / SORT_THREADS;
     int32_t* block_tot = (int32_t*)ws;
     sort_hist_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, block_tot, status);
-    sort_scan_kernel<<<1, 64, 0, st>>>(block_tot, nblk, E, offsets);
+    sort_scan_kernel<<<1, 1024, 0, st>>>(block_tot, nblk, E, offsets);
     sort_scatter_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, block_tot, perm, Y_zero_invalid, N);
     count_launch(3);
     return cuda_ok(cudaGetLastError());
@@ -382,7 +397,7 @@ extern "C" moqe_status moqe_permute_static(const void* X_bf16, const int32_t* ro
     } else {
         int nblk = (M + SORT_THREADS - 1) / SORT_THREADS;
         sort_hist_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, scratch, nullptr);
-        sort_scan_kernel<<<1, 64, 0, st>>>(scratch, nblk, E, offsets);
+        sort_scan_kernel<<<1, 1024, 0, st>>>(scratch, nblk, E, offsets);
         sort_scatter_kernel<<<nblk, SORT_THREADS, 0, st>>>(row_ids, M, E, scratch, perm, nullptr, 0);
         count_launch(3);
     }

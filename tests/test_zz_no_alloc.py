@@ -28,7 +28,8 @@ def test_static_permute_matches_permute_twice_in_a_row():
     g = np.random.default_rng(2024)
     # two different batches back to back: a large one that fills the scratch, then a smaller one with
     # another expert count that must not be disturbed by what the first call left behind
-    for M, Cc, E in [(70001, 64, 5), (5000, 16, 3), (600, 8, 2)]:
+    first = True
+    for M, Cc, E in [(70001, 64, 5), (5000, 16, 3), (600, 8, 2), (moqe.PERMUTE_STATIC_MAX_ROWS, 8, 4)]:
         ids_h = g.integers(0, E, size=M).astype(np.int32)
         if E >= 3:
             ids_h[ids_h == 1] = 0
@@ -39,14 +40,36 @@ def test_static_permute_matches_permute_twice_in_a_row():
         Xp = torch.empty_like(X)
         perm = torch.full((M,), -7, dtype=torch.int32, device=dev)
         offsets = torch.full((E + 1,), -7, dtype=torch.int32, device=dev)
+        if first:
+            # the first call on a device looks up the address of the built-in scratch array (no allocation, but
+            # it may load the module's data); the measurement below starts after it
+            assert _call_static(moqe, X, ids, E, Xp, perm, offsets) == moqe.OK
+            first = False
         torch.cuda.synchronize()
-        before = torch.cuda.memory_allocated(dev)
+        before, before_free = torch.cuda.memory_allocated(dev), torch.cuda.mem_get_info(dev)[0]
         assert _call_static(moqe, X, ids, E, Xp, perm, offsets) == moqe.OK
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated(dev) == before
+        assert torch.cuda.memory_allocated(dev) == before          # nothing from torch's allocator
+        assert torch.cuda.mem_get_info(dev)[0] == before_free      # and nothing from the driver either
         assert torch.equal(perm, perm_ref)
         assert torch.equal(offsets, off_ref)
         assert torch.equal(Xp.view(torch.int16), Xp_ref.view(torch.int16))
+    # ids outside [0, E): sorted behind the valid rows exactly as moqe_permute does, but no status is latched
+    M, Cc, E = 3000, 8, 3
+    ids_h = g.integers(0, E, size=M).astype(np.int32)
+    ids_h[[5, 77, 2999]] = [E, -1, 1000]
+    ids = torch.from_numpy(ids_h).to(dev)
+    X = torch.from_numpy(g.integers(0, 65536, size=(M, Cc)).astype(np.uint16).view(np.int16)).to(dev).view(torch.bfloat16)
+    Xp_ref, perm_ref, off_ref = moqe.moqe_permute(X, ids, E)
+    assert moqe.moqe_async_status() == moqe.ERR_EXPERT_ID           # (the allocating entry point latches it; now cleared)
+    Xp = torch.empty_like(X)
+    perm = torch.full((M,), -7, dtype=torch.int32, device=dev)
+    offsets = torch.full((E + 1,), -7, dtype=torch.int32, device=dev)
+    assert _call_static(moqe, X, ids, E, Xp, perm, offsets) == moqe.OK
+    assert moqe.moqe_async_status() == moqe.OK
+    assert int(offsets[E]) == M - 3
+    assert torch.equal(perm, perm_ref) and torch.equal(offsets, off_ref)
+    assert torch.equal(Xp.view(torch.int16), Xp_ref.view(torch.int16))
     # indices only, and the size limit
     ids = torch.zeros(2000, dtype=torch.int32, device=dev)
     perm = torch.empty(2000, dtype=torch.int32, device=dev)
