@@ -184,6 +184,59 @@ def routed_gemm_f64(X: np.ndarray, row_ids: np.ndarray, What: Sequence[np.ndarra
     return Y
 
 
+def router_mlp(X: np.ndarray, row_offsets: np.ndarray, W1: np.ndarray, W2: np.ndarray):
+    """Router front end -> (logits fp64 [S][E], pooled fp64 [S][H]): mean-pooled rows, two-layer ReLU MLP, fp64."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    off = np.ascontiguousarray(row_offsets, dtype=np.int32)
+    W1 = np.ascontiguousarray(W1, dtype=np.float32)
+    W2 = np.ascontiguousarray(W2, dtype=np.float32)
+    S, H, D, E = len(off) - 1, X.shape[1], W1.shape[0], W2.shape[0]
+    if W1.shape[1] != H or W2.shape[1] != D or (S and off[-1] > X.shape[0]):
+        raise ValueError("router_mlp: shapes disagree")
+    pooled = np.empty((S, H), dtype=np.float64)
+    logits = np.empty((S, E), dtype=np.float64)
+    _chk(lib().oracle_router_mlp(_p(X), _p(off), S, H, _p(W1), D, _p(W2), E, _p(pooled), _p(logits)), "router_mlp")
+    return logits, pooled
+
+
+def load_report(logits: np.ndarray, ids: np.ndarray):
+    """-> (P fp64 [E], F fp64 [E], L_bal): mean routing probability, dispatched fraction, balance term."""
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    S, E = logits.shape
+    P = np.empty(E, dtype=np.float64)
+    F = np.empty(E, dtype=np.float64)
+    lb = C.c_double(0.0)
+    _chk(lib().oracle_load_report(_p(logits), _p(ids), S, E, _p(P), _p(F), C.byref(lb)), "load_report")
+    return P, F, float(lb.value)
+
+
+def routed_gated_pair(X: np.ndarray, row_ids: np.ndarray, Wgate: Sequence[np.ndarray], Wup: Sequence[np.ndarray]) -> np.ndarray:
+    """bf16 bits of silu(X.Wgate_e^T) * (X.Wup_e^T), fp32 throughout, rounded once."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    row_ids = np.ascontiguousarray(row_ids, dtype=np.int32)
+    M, K = X.shape
+    N = Wgate[0].shape[0]
+    gk, ga = _what_array(Wgate)
+    uk, ua = _what_array(Wup)
+    Y = np.empty((M, N), dtype=np.uint16)
+    _chk(lib().oracle_routed_gated_pair(_p(X), _p(row_ids), M, K, N, len(Wgate), ga, ua, _p(Y)), "routed_gated_pair")
+    return Y
+
+
+def routed_gemm_residual(X: np.ndarray, row_ids: np.ndarray, What: Sequence[np.ndarray], R: np.ndarray) -> np.ndarray:
+    """bf16 bits of X.W_e^T + R (R bf16 bits), fp32, rounded once."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    row_ids = np.ascontiguousarray(row_ids, dtype=np.int32)
+    R = np.ascontiguousarray(R, dtype=np.uint16)
+    M, K = X.shape
+    N = What[0].shape[0]
+    wk, wa = _what_array(What)
+    Y = np.empty((M, N), dtype=np.uint16)
+    _chk(lib().oracle_routed_gemm_residual(_p(X), _p(row_ids), M, K, N, len(What), wa, _p(R), _p(Y)), "routed_gemm_residual")
+    return Y
+
+
 def f16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     L = lib()
     flat = np.ascontiguousarray(h, dtype=np.uint16).ravel()

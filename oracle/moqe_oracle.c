@@ -29,7 +29,11 @@
  * code ranges, closed-form grids that must be recovered exactly, brute-force
  * nearest-code search on small tiles, std::max_element / numpy.argsort(stable)
  * equivalences, exact-integer GEMM cases, single-expert equivalence, batch
- * shuffle invariance, X = I.  The end-to-end numbers of the routed layer have
+ * shuffle invariance, X = I; for the router front end and the load report:
+ * brute force in Python, hand-worked examples, sum P = sum F = 1, L_bal = 1 at
+ * perfect balance and E at collapse; for the gated pair and the residual add:
+ * X = I closed forms, silu(0) = 0, silu(a) - silu(-a) = a, R = 0 and X = 0
+ * reductions to the plain product.  The end-to-end numbers of the routed layer have
  * no value printed in the paper: "parity unpinned by the paper" for those;
  * they are pinned by the mathematical properties above instead.
  *
@@ -333,6 +337,125 @@ int oracle_routed_gemm_f64(const uint16_t *X, const int32_t *row_ids, int M, int
         double acc = 0.0;
         for (int k = 0; k < K; ++k) acc += (double)oracle_bf16_to_f32(x[k]) * (double)w[k];
         Y_f64[t] = acc;
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * Router front end.  Section 3.2 ("Router Model"): the router ends in an MLP that maps
+ * the sample's feature vector to one score per expert, and one expert index leaves it.
+ * The stand-in here (the paper's trained routers are not available): the feature
+ * vector of a sample is the mean of its rows; the MLP is two layers with a ReLU
+ * between them and no biases.  Everything in fp64:
+ *   pooled[s][h] = (1 / n_s) * sum_{rows r of sample s} X[r][h]
+ *   hidden[s][d] = max(0, sum_h pooled[s][h] * W1[d][h])
+ *   logits[s][e] = sum_d hidden[s][d] * W2[e][d]
+ * A sample without rows has pooled = 0.
+ * ------------------------------------------------------------------------- */
+int oracle_router_mlp(const uint16_t *X, const int32_t *row_offsets, int S, int H, const float *W1, int D,
+                      const float *W2, int E, double *pooled, double *logits)
+{
+    if (!X || !row_offsets || !W1 || !W2 || !logits || S < 0 || H <= 0 || D <= 0 || E <= 0) return -1;
+    double *pool = (double *)malloc(sizeof(double) * (size_t)H);
+    double *hid = (double *)malloc(sizeof(double) * (size_t)D);
+    if (!pool || !hid) { free(pool); free(hid); return -1; }
+    for (int s = 0; s < S; ++s) {
+        int r0 = row_offsets[s], r1 = row_offsets[s + 1];
+        if (r1 < r0) { free(pool); free(hid); return -1; }
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int r = r0; r < r1; ++r) acc += (double)oracle_bf16_to_f32(X[(size_t)r * H + h]);
+            pool[h] = r1 > r0 ? acc / (double)(r1 - r0) : 0.0;
+            if (pooled) pooled[(size_t)s * H + h] = pool[h];
+        }
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int h = 0; h < H; ++h) acc += pool[h] * (double)W1[(size_t)d * H + h];
+            hid[d] = acc > 0.0 ? acc : 0.0;
+        }
+        for (int e = 0; e < E; ++e) {
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += hid[d] * (double)W2[(size_t)e * D + d];
+            logits[(size_t)s * E + e] = acc;
+        }
+    }
+    free(pool);
+    free(hid);
+    return 0;
+}
+
+/* Load report of a routed batch.  Section 3.3 ("Router Fine-Tuning"), the balance term of the
+ * objective, evaluated at inference time on the batch's S samples (the paper's B) and E experts (its N):
+ *   p_i(x) = softmax(logits(x))_i,  P_i = (1/S) sum_x p_i(x),  F_i = n_i / S,  L_bal = E * sum_i P_i * F_i
+ * with n_i the number of samples dispatched to expert i (ids).  fp64. */
+int oracle_load_report(const double *logits, const int32_t *ids, int S, int E, double *P, double *F, double *Lbal)
+{
+    if (!logits || !ids || !P || !F || !Lbal || S <= 0 || E <= 0) return -1;
+    for (int e = 0; e < E; ++e) { P[e] = 0.0; F[e] = 0.0; }
+    for (int s = 0; s < S; ++s) {
+        if (ids[s] < 0 || ids[s] >= E) return -2;
+        const double *l = logits + (size_t)s * E;
+        double mx = l[0];
+        for (int e = 1; e < E; ++e) if (l[e] > mx) mx = l[e];
+        double den = 0.0;
+        for (int e = 0; e < E; ++e) den += exp(l[e] - mx);
+        for (int e = 0; e < E; ++e) P[e] += exp(l[e] - mx) / den;
+        F[ids[s]] += 1.0;
+    }
+    double lb = 0.0;
+    for (int e = 0; e < E; ++e) { P[e] /= (double)S; F[e] /= (double)S; lb += P[e] * F[e]; }
+    *Lbal = (double)E * lb;
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * Steps either side of the routed product inside an expert's forward pass (Section 4.4 times whole expert
+ * forwards, so what sits between two linear layers counts).  Both use the routed product above -- fp32,
+ * k increasing, product rounded then added -- and round to bf16 ONCE at the end:
+ *   gated pair   : Y[m][n] = bf16( silu(a) * b ),  a = (X . Wgate_e^T)[m][n],  b = (X . Wup_e^T)[m][n],
+ *                  silu(a) = a / (1 + exp(-a)) in fp32
+ *   residual add : Y[m][n] = bf16( a + float(R[m][n]) ),  R bf16
+ * ------------------------------------------------------------------------- */
+int oracle_routed_gated_pair(const uint16_t *X, const int32_t *row_ids, int M, int K, int N, int E,
+                             const float *const *Wgate, const float *const *Wup, uint16_t *Y_bf16)
+{
+    if (!X || !row_ids || !Wgate || !Wup || !Y_bf16 || M < 0 || K <= 0 || N <= 0 || E <= 0) return -1;
+    for (int m = 0; m < M; ++m)
+        if (row_ids[m] < 0 || row_ids[m] >= E) return -2;
+    long total = (long)M * N;
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < total; ++t) {
+        int m = (int)(t / N), n = (int)(t % N);
+        const float *wg = Wgate[row_ids[m]] + (size_t)n * K;
+        const float *wu = Wup[row_ids[m]] + (size_t)n * K;
+        const uint16_t *x = X + (size_t)m * K;
+        float a = 0.0f, b = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            float xf = oracle_bf16_to_f32(x[k]);
+            a += xf * wg[k];
+            b += xf * wu[k];
+        }
+        float silu = a / (1.0f + expf(-a));
+        Y_bf16[t] = oracle_f32_to_bf16(silu * b);
+    }
+    return 0;
+}
+
+int oracle_routed_gemm_residual(const uint16_t *X, const int32_t *row_ids, int M, int K, int N, int E,
+                                const float *const *What, const uint16_t *R, uint16_t *Y_bf16)
+{
+    if (!X || !row_ids || !What || !R || !Y_bf16 || M < 0 || K <= 0 || N <= 0 || E <= 0) return -1;
+    for (int m = 0; m < M; ++m)
+        if (row_ids[m] < 0 || row_ids[m] >= E) return -2;
+    long total = (long)M * N;
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < total; ++t) {
+        int m = (int)(t / N), n = (int)(t % N);
+        const float *w = What[row_ids[m]] + (size_t)n * K;
+        const uint16_t *x = X + (size_t)m * K;
+        float acc = 0.0f;
+        for (int k = 0; k < K; ++k) acc += oracle_bf16_to_f32(x[k]) * w[k];
+        Y_bf16[t] = oracle_f32_to_bf16(acc + oracle_bf16_to_f32(R[t]));
     }
     return 0;
 }
