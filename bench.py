@@ -391,11 +391,19 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
             layers[g[0]]["multi"] = ((C.c_void_p * len(g))(*[L["X"].data_ptr() for L in Ls]),
                                      (C.c_void_p * len(g))(*[L["Y"].data_ptr() for L in Ls]),
                                      (C.c_void_p * (len(g) * E))(*[e.handle for L in Ls for e in L["experts"]]))
-    lg = workload_logits(w, seed)
-    if force_expert is not None:                            # every sample to one expert
-        lg = np.full_like(lg, -1.0)
-        lg[:, force_expert] = 1.0
-    logits_h = torch.from_numpy(lg).pin_memory()
+    on_device_router = w.routing == "router_mlp" and force_expert is None
+    if on_device_router:
+        # the router front end runs on the device inside the step: mean-pool of the first layer's input -> MLP -> ids
+        W1h, W2h = wl.router_weights(w, seed)
+        rW1, rW2 = torch.from_numpy(W1h).to(dev), torch.from_numpy(W2h).to(dev)
+        r_ws = moqe.alloc_workspace(moqe.lib().moqe_router_mlp_workspace(w.n_samples, w.layers[0].K, 256), dev)
+        logits_h = torch.zeros((w.n_samples, E), dtype=torch.float32).pin_memory()
+    else:
+        lg = workload_logits(w, seed)
+        if force_expert is not None:                        # every sample to one expert
+            lg = np.full_like(lg, -1.0)
+            lg[:, force_expert] = 1.0
+        logits_h = torch.from_numpy(lg).pin_memory()
     logits = logits_h.to(dev)
     torch.cuda.synchronize()
 
@@ -411,9 +419,14 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
     # groups of layers that share one row structure share one sort
     def hot_path(from_host: bool):
         lgd = logits
-        if from_host:
-            lgd.copy_(logits_h, non_blocking=True)
-        ids = moqe.moqe_route(lgd)
+        if on_device_router:
+            if from_host:
+                layers[0]["X"].copy_(layers[0]["Xh"], non_blocking=True)
+            _, ids = moqe.moqe_router_mlp(layers[0]["X"], layers[0]["row_off"], rW1, rW2, workspace=r_ws)
+        else:
+            if from_host:
+                lgd.copy_(logits_h, non_blocking=True)
+            ids = moqe.moqe_route(lgd)
         sorted_for = {}
         for g in groups:
             Ls = [layers[j] for j in g]
@@ -547,7 +560,8 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
         "config": {"workload": w.name, "layers": [f"{l.name}:{l.N}x{l.K}" for l in w.layers],
                    "experts": [sp.tag for sp in w.experts], "tokens_per_step": tokens_per_step,
                    "rows_per_expert": {str(k): v.tolist() for k, v in counts.items()},
-                   "routing": "every sample to expert %d" % force_expert if force_expert is not None else w.routing,
+                   "routing": "every sample to expert %d" % force_expert if force_expert is not None else
+                              (w.routing + (" (computed on the device inside the step)" if on_device_router else "")),
                    "parallelism": f"replicas x{world} (samples sharded, experts replicated, no collective)",
                    "l2": "weights of one block exceed L2 (inputs larger than L2, no flush)" if sum(alg_bytes) > 126e6
                          else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path,

@@ -174,6 +174,29 @@ MOQE_API moqe_status moqe_permute_static(const void* X_bf16, const int32_t* row_
                                          void* Xp_bf16, int32_t* perm, int32_t* offsets, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Router front end on the device (Section 3.2 "Router Model": the router ends in an MLP that maps the sample's
+ * feature vector to one score per expert, and one expert index leaves it).  The paper's trained encoders are not
+ * part of this library; the feature vector is the mean of the sample's rows:
+ *   pooled[s][h] = mean over rows r in [row_offsets[s], row_offsets[s+1]) of X[r][h]   (0 for a sample without rows)
+ *   hidden[s][d] = max(0, sum_h pooled[s][h] * W1[d][h]),   logits[s][e] = sum_d hidden[s][d] * W2[e][d]
+ *   ids[s]       = first maximum of logits[s] (as moqe_route)
+ * X bf16 [rows][H] (H a multiple of 8, 16-byte aligned), row_offsets int32 [S+1], W1 fp32 [D][H] (16-byte aligned),
+ * W2 fp32 [E][D], logits fp32 [S][E] and ids int32 [S] are written.  All device pointers; fp32 arithmetic in a fixed
+ * summation order (the same call gives the same bits).  workspace: moqe_router_mlp_workspace(S, H, D) bytes,
+ * 256-byte aligned, contents irrelevant.  E <= MOQE_MAX_EXPERTS.
+ *
+ * moqe_router_load_report (Section 3.3 "Router Fine-Tuning", the balance term, evaluated on a routed batch):
+ *   report[i] = P_i = mean over the S samples of softmax(logits[s])_i,   report[E + i] = F_i = n_i / S,
+ *   report[2E] = L_bal = E * sum_i P_i * F_i,   counts[i] = n_i = samples with ids[s] == i   (counts may be NULL).
+ * ------------------------------------------------------------------------- */
+MOQE_API size_t moqe_router_mlp_workspace(int S, int H, int D);
+MOQE_API moqe_status moqe_router_mlp(const void* X_bf16, const int32_t* row_offsets, int S, int H, const float* W1, int D,
+                                     const float* W2, int E, float* logits, int32_t* ids, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+MOQE_API moqe_status moqe_router_load_report(const float* logits, const int32_t* ids, int S, int E, float* report,
+                                             int32_t* counts, void* stream);
+
+/* ---------------------------------------------------------------------------
  * The routed dequant-GEMM (Section 3.1: "the activated quantization expert
  * performs the inference on this sample" -- here for a whole mixed batch):
  *   Y[m][n] = bf16( sum_k X[m][k] * s_e[n][k/g] * (c_e[n][k] - z_e[n][k/g]) ),

@@ -220,6 +220,14 @@ def router_logits(w: Workload, seed: int = BASE_SEED, pooled: Optional[np.ndarra
     raise ValueError(w.routing)
 
 
+def router_weights(w: Workload, seed: int = BASE_SEED):
+    """The random fp32 weights ``(W1 [256][hidden], W2 [E][256])`` of the ``router_mlp`` workloads' stand-in router."""
+    H, E = w.layers[0].K, w.n_experts
+    w1 = normal_f32(f"{w.name}/router/w1", (256, H), 1.0 / np.sqrt(H), seed)
+    w2 = normal_f32(f"{w.name}/router/w2", (E, 256), 1.0 / np.sqrt(256.0), seed)
+    return w1, w2
+
+
 def mean_pool(x_bf16: np.ndarray, row_offsets: np.ndarray) -> np.ndarray:
     """fp32 mean of each sample's rows (input preparation for ``router_mlp``)."""
     x = bf16_bits_to_f32(x_bf16)

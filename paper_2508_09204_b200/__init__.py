@@ -28,6 +28,7 @@ EXPORTED = (
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
     "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count", "moqe_tune", "moqe_selftest_timeout",
+    "moqe_router_mlp_workspace", "moqe_router_mlp", "moqe_router_load_report",
 )
 
 
@@ -74,6 +75,10 @@ def lib() -> C.CDLL:
         L.moqe_status_str.restype = C.c_char_p
         L.moqe_tune.argtypes = [C.c_char_p, i32]
         L.moqe_selftest_timeout.argtypes = [C.c_uint, vp, vp]
+        L.moqe_router_mlp_workspace.argtypes = [i32, i32, i32]
+        L.moqe_router_mlp_workspace.restype = sz
+        L.moqe_router_mlp.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, sz, vp]
+        L.moqe_router_load_report.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.moqe_launch_count.argtypes = []
         L.moqe_launch_count.restype = C.c_ulonglong
         _lib = L
@@ -305,6 +310,29 @@ def moqe_async_status() -> int:
 
 def moqe_tune(key: str, value: int) -> None:
     _check(lib().moqe_tune(key.encode(), int(value)), "moqe_tune")
+
+
+def moqe_router_mlp(X: torch.Tensor, row_offsets: torch.Tensor, W1: torch.Tensor, W2: torch.Tensor,
+                    workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """-> (logits fp32 [S][E], ids int32 [S]) of the router front end, all on the device."""
+    S, H, D, E = row_offsets.numel() - 1, X.shape[1], W1.shape[0], W2.shape[0]
+    logits = torch.empty((S, E), dtype=torch.float32, device=X.device)
+    ids = torch.empty((S,), dtype=torch.int32, device=X.device)
+    need = int(lib().moqe_router_mlp_workspace(S, H, D))
+    ws = workspace if workspace is not None else alloc_workspace(need, X.device)
+    _check(lib().moqe_router_mlp(X.data_ptr(), row_offsets.data_ptr(), S, H, W1.data_ptr(), D, W2.data_ptr(), E,
+                                 logits.data_ptr(), ids.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "moqe_router_mlp")
+    return logits, ids
+
+
+def moqe_router_load_report(logits: torch.Tensor, ids: torch.Tensor):
+    """-> (P fp32 [E], F fp32 [E], L_bal fp32 scalar tensor, counts int32 [E])."""
+    S, E = logits.shape
+    report = torch.empty((2 * E + 1,), dtype=torch.float32, device=logits.device)
+    counts = torch.empty((E,), dtype=torch.int32, device=logits.device)
+    _check(lib().moqe_router_load_report(logits.data_ptr(), ids.data_ptr(), S, E, report.data_ptr(), counts.data_ptr(),
+                                         _stream()), "moqe_router_load_report")
+    return report[:E], report[E:2 * E], report[2 * E], counts
 
 
 def moqe_selftest_timeout(limit_us: int = 1000) -> int:
