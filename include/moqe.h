@@ -57,7 +57,8 @@ typedef enum {
     MOQE_ERR_MISMATCH = 6,     /* experts of one call disagree on N or K */
     MOQE_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
     MOQE_ERR_EXPERT_ID = 8,    /* asynchronous: an id outside [0,E) was seen by a kernel */
-    MOQE_ERR_TIMEOUT = 9       /* asynchronous: a bounded in-kernel wait ran out */
+    MOQE_ERR_TIMEOUT = 9,      /* asynchronous: a bounded in-kernel wait ran out */
+    MOQE_ERR_IO = 10           /* a file could not be opened, read or written, or is not a whole expert image */
 } moqe_status;
 
 #define MOQE_MAX_EXPERTS 32
@@ -108,6 +109,32 @@ MOQE_API moqe_status moqe_expert_info(const moqe_expert* e, int* N, int* K, int*
 
 /* Frees the expert's device buffers (cudaFree: synchronises the device). */
 MOQE_API moqe_status moqe_expert_destroy(moqe_expert* e);
+
+/* ---------------------------------------------------------------------------
+ * Expert residency (Section 4.4 and the appendix table "Router model and expert loading overhead": one expert
+ * stays on the GPU, the others wait in CPU RAM and are loaded when the routing changes).  A packed expert is a
+ * plain byte image, so parking and reloading it is copy-engine work only:
+ *   moqe_expert_offload   : device expert -> a copy in PINNED host memory (synchronises `stream`; the device expert
+ *                           is left as it is and may be destroyed afterwards).
+ *   moqe_expert_prefetch  : pinned host copy -> a NEW device expert; allocates (synchronously), then enqueues the
+ *                           host-to-device copies on `stream` and returns at once.  Give it a side stream to
+ *                           overlap the copy with the layer that is running; the expert may be used by work
+ *                           ordered after those copies (same stream, or an event recorded on it).  The host copy
+ *                           must stay alive until the copies have completed.
+ *   moqe_expert_host_save / _load : the host copy to / from a file.  The file holds a header (magic, packed-layout
+ *                           version, N, K, bits, group, sym, byte counts) and the packed image; it is tied to
+ *                           the packed layout of the library that wrote it.  A file that is not exactly one
+ *                           image of a supported format is refused (MOQE_ERR_IO / _UNSUPPORTED / _SHAPE).
+ * The library owns what *out points at; destroy with moqe_expert_host_destroy / moqe_expert_destroy.
+ * ------------------------------------------------------------------------- */
+typedef struct moqe_expert_host moqe_expert_host;
+MOQE_API moqe_status moqe_expert_offload(const moqe_expert* e, void* stream, moqe_expert_host** out);
+MOQE_API moqe_status moqe_expert_prefetch(const moqe_expert_host* h, void* stream, moqe_expert** out);
+MOQE_API moqe_status moqe_expert_host_info(const moqe_expert_host* h, int* N, int* K, int* bits, int* group, int* sym,
+                                           size_t* image_bytes);
+MOQE_API moqe_status moqe_expert_host_save(const moqe_expert_host* h, const char* path);
+MOQE_API moqe_status moqe_expert_host_load(const char* path, moqe_expert_host** out);
+MOQE_API moqe_status moqe_expert_host_destroy(moqe_expert_host* h);
 
 /* ---------------------------------------------------------------------------
  * Hard routing (Section 3.2; Appendix: the router's decision r(x) is one expert

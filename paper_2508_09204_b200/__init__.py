@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmoqe.so")
 
 OK = 0
-ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_WORKSPACE, ERR_MISMATCH, ERR_CUDA, ERR_EXPERT_ID, ERR_TIMEOUT = range(1, 10)
+ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_WORKSPACE, ERR_MISMATCH, ERR_CUDA, ERR_EXPERT_ID, ERR_TIMEOUT, ERR_IO = range(1, 11)
 MAX_EXPERTS = 32
 PATH_AUTO, PATH_STREAM, PATH_TCGEN05, PATH_DECODE = 0, 1, 2, 5
 
@@ -29,6 +29,8 @@ EXPORTED = (
     "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count", "moqe_tune", "moqe_selftest_timeout",
     "moqe_router_mlp_workspace", "moqe_router_mlp", "moqe_router_load_report",
+    "moqe_expert_offload", "moqe_expert_prefetch", "moqe_expert_host_info", "moqe_expert_host_save", "moqe_expert_host_load",
+    "moqe_expert_host_destroy",
 )
 
 
@@ -75,6 +77,12 @@ def lib() -> C.CDLL:
         L.moqe_status_str.restype = C.c_char_p
         L.moqe_tune.argtypes = [C.c_char_p, i32]
         L.moqe_selftest_timeout.argtypes = [C.c_uint, vp, vp]
+        L.moqe_expert_offload.argtypes = [vp, vp, C.POINTER(vp)]
+        L.moqe_expert_prefetch.argtypes = [vp, vp, C.POINTER(vp)]
+        L.moqe_expert_host_info.argtypes = [vp] + [C.POINTER(i32)] * 5 + [C.POINTER(sz)]
+        L.moqe_expert_host_save.argtypes = [vp, C.c_char_p]
+        L.moqe_expert_host_load.argtypes = [C.c_char_p, C.POINTER(vp)]
+        L.moqe_expert_host_destroy.argtypes = [vp]
         L.moqe_router_mlp_workspace.argtypes = [i32, i32, i32]
         L.moqe_router_mlp_workspace.restype = sz
         L.moqe_router_mlp.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, vp, vp, vp, sz, vp]
@@ -135,6 +143,53 @@ class Expert:
             self.close()
         except Exception:
             pass
+
+
+class HostExpert:
+    """Owner of one ``moqe_expert_host*``: a packed expert parked in pinned host memory."""
+
+    def __init__(self, handle: int):
+        self.handle = C.c_void_p(handle)
+        N, K, bits, group, sym = (C.c_int() for _ in range(5))
+        nb = C.c_size_t()
+        _check(lib().moqe_expert_host_info(self.handle, N, K, bits, group, sym, nb), "moqe_expert_host_info")
+        self.N, self.K, self.bits, self.group, self.sym = N.value, K.value, bits.value, group.value, bool(sym.value)
+        self.image_bytes = nb.value
+
+    def close(self):
+        if self.handle is not None and self.handle.value:
+            lib().moqe_expert_host_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def moqe_expert_offload(e: Expert) -> HostExpert:
+    out = C.c_void_p()
+    _check(lib().moqe_expert_offload(e.handle, _stream(), C.byref(out)), "moqe_expert_offload")
+    return HostExpert(out.value)
+
+
+def moqe_expert_prefetch(h: HostExpert, stream: Optional[torch.cuda.Stream] = None) -> Expert:
+    """Enqueues the host-to-device copies on ``stream`` (default: the current one) and returns the new expert."""
+    out = C.c_void_p()
+    st = C.c_void_p(stream.cuda_stream) if stream is not None else _stream()
+    _check(lib().moqe_expert_prefetch(h.handle, st, C.byref(out)), "moqe_expert_prefetch")
+    return Expert(out.value)
+
+
+def moqe_expert_host_save(h: HostExpert, path: str) -> None:
+    _check(lib().moqe_expert_host_save(h.handle, os.fsencode(path)), "moqe_expert_host_save")
+
+
+def moqe_expert_host_load(path: str) -> HostExpert:
+    out = C.c_void_p()
+    _check(lib().moqe_expert_host_load(os.fsencode(path), C.byref(out)), "moqe_expert_host_load")
+    return HostExpert(out.value)
 
 
 def moqe_quantize_rtn(W: torch.Tensor, bits: int, group: int, sym: bool) -> Expert:

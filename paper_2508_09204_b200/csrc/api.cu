@@ -254,6 +254,7 @@ extern "C" const char* moqe_status_str(moqe_status s) {
         case MOQE_ERR_CUDA: return "a CUDA call failed";
         case MOQE_ERR_EXPERT_ID: return "an expert id outside [0,E) was seen on the device";
         case MOQE_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
+        case MOQE_ERR_IO: return "file missing, unreadable, unwritable or not a whole expert image";
     }
     return "unknown status";
 }

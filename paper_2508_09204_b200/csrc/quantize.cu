@@ -6,6 +6,8 @@
 // for the exact arithmetic.  Every fp32 operation below is a single IEEE
 // operation (explicit __f*_rn intrinsics, no fused multiply-add, no fast
 // math), so codes, scales and zero-points are reproducible bit for bit.
+#include <cstdio>
+#include <cstring>
 #include <new>
 
 #include "dequant.cuh"
@@ -450,4 +452,134 @@ extern "C" moqe_status moqe_expert_destroy(moqe_expert* e) {
     cudaError_t a = cudaFree(e->tiles), b = cudaFree(e->scales_pc), c = cudaFree(e->zeros_pc);
     delete e;
     return (a == cudaSuccess && b == cudaSuccess && c == cudaSuccess) ? MOQE_OK : MOQE_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------- expert residency
+// Section 4.4 of the paper and its appendix table "Router model and expert loading overhead": one expert is kept on
+// the GPU, the others wait in CPU RAM (or on disk) and are loaded when the routing changes.  A packed expert is a
+// plain byte image (its tiles, and for per-channel experts the scale / zero-point arrays), so moving it is pure
+// copy-engine work: to a file, to pinned host memory, and back on a side stream while the current layer runs.
+namespace moqe {
+namespace {
+
+struct ImageHeader {
+    char magic[8];                 // "MOQEXP1\0"
+    int32_t layout;                // version of the packed layout this library writes
+    int32_t N, K, bits, group, sym;
+    uint64_t tiles_bytes, pc_bytes;
+};
+constexpr int32_t PACKED_LAYOUT_VERSION = 1;
+
+ImageHeader header_of(const moqe_expert* e) {
+    ImageHeader h = {};
+    memcpy(h.magic, "MOQEXP1", 8);
+    h.layout = PACKED_LAYOUT_VERSION;
+    h.N = e->N; h.K = e->K; h.bits = e->bits; h.group = e->group; h.sym = e->sym;
+    h.tiles_bytes = e->tiles_alloc; h.pc_bytes = e->pc_alloc;
+    return h;
+}
+// does the header describe an expert this library would lay out in exactly these sizes?
+moqe_status header_ok(const ImageHeader& h) {
+    if (memcmp(h.magic, "MOQEXP1", 8) != 0 || h.layout != PACKED_LAYOUT_VERSION) return MOQE_ERR_UNSUPPORTED;
+    moqe_status s = check_format(h.N, h.K, h.bits, h.group);
+    if (s != MOQE_OK) return s;
+    const size_t Np = (size_t)(h.N + 127) / 128 * 128, Kp = (size_t)(h.K + 127) / 128 * 128;
+    const size_t tiles = (Np / 128) * (Kp / 128) * moqe_tile_stride(h.bits, h.group, !h.sym);
+    const size_t pc = h.group == 0 ? Np * 2 : 0;
+    return (h.tiles_bytes == tiles && h.pc_bytes == pc && (h.sym == 0 || h.sym == 1)) ? MOQE_OK : MOQE_ERR_SHAPE;
+}
+size_t image_bytes(const ImageHeader& h) { return (size_t)h.tiles_bytes + (size_t)h.pc_bytes * (h.sym ? 1 : 2); }
+
+}  // namespace
+}  // namespace moqe
+
+// A packed expert parked in pinned host memory: header + byte image.
+struct moqe_expert_host {
+    moqe::ImageHeader h;
+    uint8_t* image;                // pinned: tiles, then scales_pc, then zeros_pc
+};
+
+extern "C" moqe_status moqe_expert_offload(const moqe_expert* e, void* stream, moqe_expert_host** out) {
+    if (!e || !out) return MOQE_ERR_NULL;
+    moqe_expert_host* hx = new (std::nothrow) moqe_expert_host();
+    if (!hx) return MOQE_ERR_ALLOC;
+    hx->h = header_of(e);
+    hx->image = nullptr;
+    if (cudaMallocHost(&hx->image, image_bytes(hx->h)) != cudaSuccess) { cudaGetLastError(); delete hx; return MOQE_ERR_ALLOC; }
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t err = cudaMemcpyAsync(hx->image, e->tiles, e->tiles_alloc, cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess && e->scales_pc) err = cudaMemcpyAsync(hx->image + e->tiles_alloc, e->scales_pc, e->pc_alloc, cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess && e->zeros_pc) err = cudaMemcpyAsync(hx->image + e->tiles_alloc + e->pc_alloc, e->zeros_pc, e->pc_alloc, cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(st);       // the image is complete when the call returns
+    if (err != cudaSuccess) { cudaFreeHost(hx->image); delete hx; return MOQE_ERR_CUDA; }
+    *out = hx;
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_prefetch(const moqe_expert_host* hx, void* stream, moqe_expert** out) {
+    if (!hx || !out) return MOQE_ERR_NULL;
+    moqe_status s = header_ok(hx->h);
+    if (s != MOQE_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    moqe_expert* e = nullptr;
+    s = alloc_expert(hx->h.N, hx->h.K, hx->h.bits, hx->h.group, hx->h.sym, st, &e);
+    if (s != MOQE_OK) return s;
+    cudaError_t err = cudaMemcpyAsync(e->tiles, hx->image, e->tiles_alloc, cudaMemcpyHostToDevice, st);
+    if (err == cudaSuccess && e->scales_pc) err = cudaMemcpyAsync(e->scales_pc, hx->image + e->tiles_alloc, e->pc_alloc, cudaMemcpyHostToDevice, st);
+    if (err == cudaSuccess && e->zeros_pc) err = cudaMemcpyAsync(e->zeros_pc, hx->image + e->tiles_alloc + e->pc_alloc, e->pc_alloc, cudaMemcpyHostToDevice, st);
+    if (err != cudaSuccess) { moqe_expert_destroy(e); return MOQE_ERR_CUDA; }
+    *out = e;
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_host_info(const moqe_expert_host* hx, int* N, int* K, int* bits, int* group, int* sym,
+                                             size_t* image_bytes_out) {
+    if (!hx) return MOQE_ERR_NULL;
+    if (N) *N = hx->h.N;
+    if (K) *K = hx->h.K;
+    if (bits) *bits = hx->h.bits;
+    if (group) *group = hx->h.group;
+    if (sym) *sym = hx->h.sym;
+    if (image_bytes_out) *image_bytes_out = image_bytes(hx->h);
+    return MOQE_OK;
+}
+
+extern "C" moqe_status moqe_expert_host_destroy(moqe_expert_host* hx) {
+    if (!hx) return MOQE_ERR_NULL;
+    cudaError_t a = cudaFreeHost(hx->image);
+    delete hx;
+    return a == cudaSuccess ? MOQE_OK : MOQE_ERR_CUDA;
+}
+
+extern "C" moqe_status moqe_expert_host_save(const moqe_expert_host* hx, const char* path) {
+    if (!hx || !path) return MOQE_ERR_NULL;
+    FILE* f = fopen(path, "wb");
+    if (!f) return MOQE_ERR_IO;
+    const size_t n = image_bytes(hx->h);
+    const bool ok = fwrite(&hx->h, sizeof(hx->h), 1, f) == 1 && (n == 0 || fwrite(hx->image, 1, n, f) == n);
+    const bool closed = fclose(f) == 0;
+    return ok && closed ? MOQE_OK : MOQE_ERR_IO;
+}
+
+extern "C" moqe_status moqe_expert_host_load(const char* path, moqe_expert_host** out) {
+    if (!path || !out) return MOQE_ERR_NULL;
+    FILE* f = fopen(path, "rb");
+    if (!f) return MOQE_ERR_IO;
+    ImageHeader h;
+    if (fread(&h, sizeof(h), 1, f) != 1) { fclose(f); return MOQE_ERR_IO; }
+    moqe_status s = header_ok(h);
+    if (s != MOQE_OK) { fclose(f); return s; }
+    // the file must hold exactly the image the header promises
+    const size_t n = image_bytes(h);
+    if (fseek(f, 0, SEEK_END) != 0 || (size_t)ftell(f) != sizeof(h) + n || fseek(f, (long)sizeof(h), SEEK_SET) != 0) { fclose(f); return MOQE_ERR_IO; }
+    moqe_expert_host* hx = new (std::nothrow) moqe_expert_host();
+    if (!hx) { fclose(f); return MOQE_ERR_ALLOC; }
+    hx->h = h;
+    hx->image = nullptr;
+    if (cudaMallocHost(&hx->image, n ? n : 1) != cudaSuccess) { cudaGetLastError(); delete hx; fclose(f); return MOQE_ERR_ALLOC; }
+    const bool ok = fread(hx->image, 1, n, f) == n;
+    fclose(f);
+    if (!ok) { cudaFreeHost(hx->image); delete hx; return MOQE_ERR_IO; }
+    *out = hx;
+    return MOQE_OK;
 }

@@ -93,3 +93,15 @@ def test_missing_library_fails_loudly(moqe, monkeypatch):
     monkeypatch.setattr(m, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libmoqe.so"))
     with pytest.raises(ImportError):
         m.lib()
+
+
+def test_expert_image_file_errors_without_a_gpu(moqe, tmp_path):
+    """A missing file and a file that is not an expert image are refused on the host, before any device call."""
+    L = moqe.lib()
+    out = C.c_void_p()
+    assert L.moqe_expert_host_load(str(tmp_path / "nothing.moqe").encode(), C.byref(out)) == moqe.ERR_IO
+    p = tmp_path / "junk.moqe"
+    p.write_bytes(b"not an expert image, just forty-eight bytes....!!")
+    assert L.moqe_expert_host_load(str(p).encode(), C.byref(out)) == moqe.ERR_UNSUPPORTED
+    assert L.moqe_expert_host_load(None, C.byref(out)) == moqe.ERR_NULL
+    assert moqe.status_str(moqe.ERR_IO).startswith("file")

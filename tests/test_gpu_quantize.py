@@ -71,6 +71,18 @@ def test_storage_ratios_match_the_papers_table():
     for name, fp16, int8, int4, unit in rows:
         assert abs(float(int8) / float(fp16) - e8.code_bytes / fp16_bytes) < 0.02
         assert abs(float(int4) / float(fp16) - e4.code_bytes / fp16_bytes) < 0.02
+    # what is really allocated (and what a parked expert's image holds): codes + scales / zero-points, nothing else when
+    # N and K are multiples of 128 -- for every format, true 3.0 bits per weight included
+    for bits, group, sym in [(8, 0, True), (4, 0, True), (4, 128, False), (3, 128, False), (3, 0, False), (4, 32, False), (8, 128, True)]:
+        e = moqe.moqe_quantize_rtn(W, bits, group, sym)
+        assert e.code_bytes == 256 * 512 * bits // 8
+        assert e.meta_bytes == 256 * (1 if group == 0 else 512 // group) * 2 * (1 if sym else 2)
+        assert e.alloc_bytes == e.code_bytes + e.meta_bytes, (bits, group, sym)
+        assert moqe.moqe_expert_offload(e).image_bytes == e.alloc_bytes
+    # ragged shapes are padded to whole 128 x 128 tiles: the padding is accounted for exactly
+    W2 = torch.from_numpy(wl.weights_f32("ratios2", 200, 320)).to(dev())
+    e = moqe.moqe_quantize_rtn(W2, 4, 64, False)
+    assert e.alloc_bytes == 256 * 384 * 4 // 8 + 256 * (384 // 64) * 2 * 2
 
 
 def test_argument_errors():
