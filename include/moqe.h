@@ -277,6 +277,21 @@ MOQE_API moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16,
                                                     int M, int n_layers, const moqe_expert* const* h_experts, int E,
                                                     void* const* h_Y_bf16, void* workspace, size_t workspace_bytes,
                                                     void* stream);
+/* Two steps of an expert's forward pass fused into the routed product of a DECODE batch (Section 4.4 times whole
+ * expert forwards, so what sits between two linear layers counts).  Same `perm` / `offsets` / workspace rules as
+ * moqe_routed_qgemm_sorted; only what the decode kernel takes (M <= 16, experts per-channel or with groups of
+ * 128 k or more), otherwise MOQE_ERR_UNSUPPORTED and nothing is launched.
+ *   _gated    : Y[m][n] = bf16( silu(a) * b ),  a = (X . Wgate_e^T)[m][n],  b = (X . Wup_e^T)[m][n],  e = the row's
+ *               expert, silu(a) = a / (1 + exp(-a)); a and b are the fp32 sums, rounded once at the end.  h_gate[e] and
+ *               h_up[e] must agree on N, K, bits, group and sym (MOQE_ERR_MISMATCH).  One launch streams both experts'
+ *               weights; the [M][N] intermediate of each projection is never written.
+ *   _residual : Y[m][n] = bf16( (X . W_e^T)[m][n] + R[m][n] ),  R bf16 [M][N] in original row order (may be Y itself). */
+MOQE_API moqe_status moqe_routed_qgemm_sorted_gated(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                                    const moqe_expert* const* h_gate, const moqe_expert* const* h_up, int E,
+                                                    void* Y_bf16, void* workspace, size_t workspace_bytes, void* stream);
+MOQE_API moqe_status moqe_routed_qgemm_sorted_residual(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                                       const moqe_expert* const* h_experts, int E, const void* R_bf16,
+                                                       void* Y_bf16, void* workspace, size_t workspace_bytes, void* stream);
 MOQE_API moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
                                                        int E, void* stream);
 

@@ -29,6 +29,7 @@ EXPORTED = (
     "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count", "moqe_tune", "moqe_selftest_timeout",
     "moqe_router_mlp_workspace", "moqe_router_mlp", "moqe_router_load_report",
+    "moqe_routed_qgemm_sorted_gated", "moqe_routed_qgemm_sorted_residual",
     "moqe_expert_offload", "moqe_expert_prefetch", "moqe_expert_host_info", "moqe_expert_host_save", "moqe_expert_host_load",
     "moqe_expert_host_destroy",
 )
@@ -71,6 +72,8 @@ def lib() -> C.CDLL:
         L.moqe_routed_qgemm_path.argtypes = [vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
         L.moqe_routed_qgemm_sorted.argtypes = [vp, vp, vp, i32, C.POINTER(vp), i32, vp, vp, sz, vp, i32]
         L.moqe_routed_qgemm_sorted_multi.argtypes = [C.POINTER(vp), vp, vp, i32, i32, C.POINTER(vp), i32, C.POINTER(vp), vp, sz, vp]
+        L.moqe_routed_qgemm_sorted_gated.argtypes = [vp, vp, vp, i32, C.POINTER(vp), C.POINTER(vp), i32, vp, vp, sz, vp]
+        L.moqe_routed_qgemm_sorted_residual.argtypes = [vp, vp, vp, i32, C.POINTER(vp), i32, vp, vp, vp, sz, vp]
         L.moqe_routed_qgemm_workspace_clear.argtypes = [vp, sz, i32, i32, i32, i32, vp]
         L.moqe_async_status.argtypes = [vp]
         L.moqe_status_str.argtypes = [i32]
@@ -335,6 +338,28 @@ def moqe_routed_qgemm_sorted(X: torch.Tensor, perm: torch.Tensor, offsets: torch
     arr = _arr if _arr is not None else (C.c_void_p * E)(*[e.handle for e in experts])
     _check(lib().moqe_routed_qgemm_sorted(_ptr(X), _ptr(perm), _ptr(offsets), M, arr, E, _ptr(Y), _ptr(workspace),
                                           workspace.numel(), _stream(), int(path)), "moqe_routed_qgemm_sorted")
+    return Y
+
+
+def moqe_routed_qgemm_sorted_gated(X: torch.Tensor, perm: torch.Tensor, offsets: torch.Tensor, gate: Sequence[Expert],
+                                   up: Sequence[Expert], Y: torch.Tensor, workspace: torch.Tensor, _arrs=None) -> torch.Tensor:
+    """``Y = silu(X . Wgate_e^T) * (X . Wup_e^T)`` for a sorted decode batch, one launch."""
+    M = X.shape[0]
+    E = len(gate)
+    ag, au = _arrs if _arrs is not None else ((C.c_void_p * E)(*[e.handle for e in gate]), (C.c_void_p * E)(*[e.handle for e in up]))
+    _check(lib().moqe_routed_qgemm_sorted_gated(_ptr(X), _ptr(perm), _ptr(offsets), M, ag, au, E, _ptr(Y), _ptr(workspace),
+                                                workspace.numel(), _stream()), "moqe_routed_qgemm_sorted_gated")
+    return Y
+
+
+def moqe_routed_qgemm_sorted_residual(X: torch.Tensor, perm: torch.Tensor, offsets: torch.Tensor, experts: Sequence[Expert],
+                                      R: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, _arr=None) -> torch.Tensor:
+    """``Y = X . W_e^T + R`` for a sorted decode batch (``R`` bf16 ``[M][N]``, may be ``Y``)."""
+    M = X.shape[0]
+    E = len(experts)
+    arr = _arr if _arr is not None else (C.c_void_p * E)(*[e.handle for e in experts])
+    _check(lib().moqe_routed_qgemm_sorted_residual(_ptr(X), _ptr(perm), _ptr(offsets), M, arr, E, _ptr(R), _ptr(Y),
+                                                   _ptr(workspace), workspace.numel(), _stream()), "moqe_routed_qgemm_sorted_residual")
     return Y
 
 

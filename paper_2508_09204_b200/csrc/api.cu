@@ -176,6 +176,54 @@ extern "C" moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf1
                              w.total - w.body, (cudaStream_t)stream);
 }
 
+namespace {
+// shared argument checks of the decode-only fused entry points
+moqe_status fused_args(const void* X, const int32_t* perm, const int32_t* offsets, int M, const moqe_expert* const* ex, int E,
+                       const void* Y, void* workspace, size_t workspace_bytes, size_t& body, size_t& total) {
+    if (!ex) return MOQE_ERR_NULL;
+    if (E <= 0 || M < 0) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
+    for (int e = 0; e < E; ++e)
+        if (!ex[e]) return MOQE_ERR_NULL;
+    const int N = ex[0]->N, K = ex[0]->K;
+    for (int e = 1; e < E; ++e)
+        if (ex[e]->N != N || ex[e]->K != K) return MOQE_ERR_MISMATCH;
+    if (M == 0) return MOQE_OK;
+    if (!X || !perm || !offsets || !Y) return MOQE_ERR_NULL;
+    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X % 16 || (uintptr_t)Y % 16) return MOQE_ERR_UNSUPPORTED;
+    if (!decode_supported_multi(M, ex, 1, E)) return MOQE_ERR_UNSUPPORTED;
+    WsLayout w = ws_layout(M, ex[0]->Np, K, E);
+    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    body = w.body;
+    total = w.total;
+    return MOQE_OK;
+}
+}  // namespace
+
+extern "C" moqe_status moqe_routed_qgemm_sorted_gated(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                                      const moqe_expert* const* h_gate, const moqe_expert* const* h_up, int E,
+                                                      void* Y_bf16, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h_up) return MOQE_ERR_NULL;
+    size_t body = 0, total = 0;
+    moqe_status s = fused_args(X_bf16, perm, offsets, M, h_gate, E, Y_bf16, workspace, workspace_bytes, body, total);
+    if (s != MOQE_OK || M == 0) return s;
+    for (int e = 0; e < E; ++e)
+        if (!h_up[e]) return MOQE_ERR_NULL;
+    return launch_qgemm_decode_ext(&X_bf16, M, 1, h_gate, h_up, E, &Y_bf16, nullptr, perm, offsets, (char*)workspace + body,
+                                   total - body, (cudaStream_t)stream);
+}
+
+extern "C" moqe_status moqe_routed_qgemm_sorted_residual(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
+                                                         const moqe_expert* const* h_experts, int E, const void* R_bf16,
+                                                         void* Y_bf16, void* workspace, size_t workspace_bytes, void* stream) {
+    size_t body = 0, total = 0;
+    moqe_status s = fused_args(X_bf16, perm, offsets, M, h_experts, E, Y_bf16, workspace, workspace_bytes, body, total);
+    if (s != MOQE_OK || M == 0) return s;
+    if (!R_bf16) return MOQE_ERR_NULL;
+    return launch_qgemm_decode_ext(&X_bf16, M, 1, h_experts, nullptr, E, &Y_bf16, &R_bf16, perm, offsets,
+                                   (char*)workspace + body, total - body, (cudaStream_t)stream);
+}
+
 extern "C" moqe_status moqe_routed_qgemm_workspace_clear(void* workspace, size_t workspace_bytes, int M, int N, int K,
                                                          int E, void* stream) {
     if (M < 0 || N <= 0 || K <= 0 || E <= 0) return MOQE_ERR_SHAPE;

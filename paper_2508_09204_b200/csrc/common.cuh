@@ -124,6 +124,9 @@ size_t decode_zero_bytes(int M);
 moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
                                       void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
                                       size_t ws_bytes, cudaStream_t st);
+moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const moqe_expert* const* ex,
+                                    const moqe_expert* const* ex2, int E, void* const* Y, const void* const* R,
+                                    const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st);
 void decode_set_tile_cost(int bits, int cost);   // relative cost of one super-tile in the work split, by code width
 
 // qgemm_tcgen05.cu

@@ -51,18 +51,22 @@ constexpr int GV_CONS = 16;                                    // consumer warps
 constexpr int GV_SERV = 2;                                     // service warps
 constexpr int GV_THREADS = (GV_CONS + GV_SERV + 1) * 32;       // + the producer's warp
 constexpr int GV_MAX_STAGES = 12;
-constexpr int GV_RING_BYTES = 158 * 1024;
+constexpr int GV_XCHG_BYTES = 8 * 8 * 32 * 4;                  // gated pairs: [8 blobs][8 values][32 lanes] floats
 constexpr int GV_XBUF = 32 * 1024;                             // one chunk of staged token rows
 constexpr int GV_CHUNK_KB = 16;                                // k-blocks per chunk for one token block (8 for two)
 constexpr int GV_SBUF = GV_CHUNK_KB * 8 * 2 * 4;               // the chunk's sums: [k-block][token block][t][4] floats
 constexpr int GV_SLOT_FLOATS = GV_CONS * 2 * 4 * 32;           // a parked partial sum: 256 channels x 16 tokens
 constexpr int GV_MAX_GRID = 256;
 
+// FUSED: the variant with gated pairs and residual adds (it gives 8 KB of the ring to the exchange buffer)
+template <bool FUSED>
 struct GvSmem {
+    static constexpr int ring_bytes = (FUSED ? 150 : 158) * 1024;
     static constexpr int ring_off = 0;
-    static constexpr int x_off = GV_RING_BYTES;
+    static constexpr int x_off = ring_bytes;
     static constexpr int s_off = x_off + 2 * GV_XBUF;
-    static constexpr int desc_off = s_off + 2 * GV_SBUF;                  // 2 chunk descriptors of 32 bytes
+    static constexpr int xchg_off = s_off + 2 * GV_SBUF;
+    static constexpr int desc_off = xchg_off + (FUSED ? GV_XCHG_BYTES : 0);   // 2 chunk descriptors of 32 bytes
     static constexpr int bar_off = desc_off + 2 * 32;                     // wfull[12] wempty[12] xfull[2] xempty[2]
     static constexpr int off_off = bar_off + (2 * GV_MAX_STAGES + 4) * 8;
     static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;
@@ -72,7 +76,7 @@ struct GvSmem {
     static constexpr int total = misc_off + 32;
     static constexpr int dyn_bytes = total;
 };
-static_assert(GvSmem::dyn_bytes <= 227 * 1024, "shared memory budget");
+static_assert(GvSmem<false>::dyn_bytes <= 227 * 1024 && GvSmem<true>::dyn_bytes <= 227 * 1024, "shared memory budget");
 
 struct GvParams {
     ExpertDev ex[MOQE_MAX_EXPERTS];         // per (layer, expert) pair
@@ -82,6 +86,12 @@ struct GvParams {
     int NT1[MOQE_MAX_EXPERTS];              // 128-channel tiles of the layer
     int rexp[MOQE_MAX_EXPERTS];             // the routing expert whose rows the pair takes
     int w[MOQE_MAX_EXPERTS];                // cost of one super-tile
+    // A gated pair (tiles2 != nullptr): the pair's second expert (same format and shape), whose product multiplies
+    // silu of the first one's; the super-tile is then {tile nt of the first, tile nt of the second}.
+    const uint8_t* tiles2[MOQE_MAX_EXPERTS];
+    const __half* scales_pc2[MOQE_MAX_EXPERTS];
+    const __nv_bfloat16* zeros_pc2[MOQE_MAX_EXPERTS];
+    const uint16_t* Res[MOQE_MAX_EXPERTS];  // residual added to the product before the rounding, or nullptr
     const int32_t* perm;
     const int32_t* offsets;
     float* partials;                        // [CTA][2][GV_SLOT_FLOATS]
@@ -270,8 +280,9 @@ __device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int s
 }
 
 // ---------------------------------------------------------------------------- the kernel
+template <bool FUSED>
 __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __grid_constant__ GvParams p) {
-    using L = GvSmem;
+    using L = GvSmem<FUSED>;
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
@@ -308,7 +319,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         if (v < p.P) {
             const int rows = p.offsets[p.rexp[v] + 1] - p.offsets[p.rexp[v]];
             wv = p.w[v];
-            TT = rows > 0 ? ((p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
+            TT = rows > 0 ? ((FUSED && p.tiles2[v]) ? p.NT1[v] : (p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
             cost = (long long)TT * wv;
         }
         long long incl = cost;
@@ -343,7 +354,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         if (lane == 0) {
             const int stage_bytes = 2 * ((max(str, 128) + 127) & ~127);
             *s_C = C; *s_G = G;
-            s_geom[0] = min(GV_MAX_STAGES, GV_RING_BYTES / stage_bytes);
+            s_geom[0] = min(GV_MAX_STAGES, L::ring_bytes / stage_bytes);
             s_geom[1] = stage_bytes;
         }
     }
@@ -447,10 +458,11 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             while (ok && wk.next(s_pair, p, changed)) {
                 const int v = wk.v, n = wk.run();
                 const uint32_t stride = (uint32_t)p.ex[v].tile_stride;
-                const int nt = 2 * wk.nt2;
-                const bool two = nt + 1 < p.NT1[v];
+                const bool gated = FUSED && p.tiles2[v] != nullptr;
+                const int nt = gated ? wk.nt2 : 2 * wk.nt2;
+                const bool two = gated || nt + 1 < p.NT1[v];
                 const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * stride;
-                const uint8_t* b = a + (size_t)wk.KB * stride;
+                const uint8_t* b = gated ? p.tiles2[v] + ((size_t)nt * wk.KB + wk.kb) * stride : a + (size_t)wk.KB * stride;
                 for (int i = 0; i < n; ++i) {
                     // Ramp-up: when all CTAs ask for a full ring at once, a CTA's first tile queues behind everybody's
                     // ninth; so the first two stages go out alone and the rest follows once the first has landed.
@@ -555,18 +567,21 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             const int v = d->v, nt2 = d->nt2, kbc = d->kbc, nkb = d->nkb, kb0 = d->kb0, kb1 = d->kb1;
             const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
             const int bits = p.ex[v].bits, group = p.ex[v].group, has_zeros = p.ex[v].has_zeros;
-            const int nt = 2 * nt2 + half;
+            const bool gated = FUSED && p.tiles2[v] != nullptr;
+            const int nt = gated ? nt2 : 2 * nt2 + half;
             const bool active = nt < p.NT1[v];
             const int n_r = nt * 128 + blob * 16 + g;
             if (kbc == kb0) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) fin[i] = 0.f;
                 if (group == 0 && active) {
-                    sc_r = __half2float(p.ex[v].scales_pc[n_r]);
-                    sc_r8 = __half2float(p.ex[v].scales_pc[n_r + 8]);
+                    const __half* sp = gated && half ? p.scales_pc2[v] : p.ex[v].scales_pc;
+                    sc_r = __half2float(sp[n_r]);
+                    sc_r8 = __half2float(sp[n_r + 8]);
                     if (has_zeros) {
-                        z_r = __bfloat162float(p.ex[v].zeros_pc[n_r]);
-                        z_r8 = __bfloat162float(p.ex[v].zeros_pc[n_r + 8]);
+                        const __nv_bfloat16* zp = gated && half ? p.zeros_pc2[v] : p.ex[v].zeros_pc;
+                        z_r = __bfloat162float(zp[n_r]);
+                        z_r8 = __bfloat162float(zp[n_r + 8]);
                     }
                 }
             }
@@ -591,21 +606,50 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                 const int NT = rows > 8 ? 2 : 1;
                 const int KB = p.KB[v], N = p.N[v];
                 uint16_t* Y = p.Y[v];
+                const uint16_t* R = FUSED ? p.Res[v] : nullptr;
                 auto store_rows = [&]() {
 #pragma unroll
                     for (int tb = 0; tb < 2; ++tb) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const int m = 8 * tb + 2 * t + (j & 1), nn = n_r + (j >> 1) * 8;
-                            if (tb < NT && m < rows && nn < N)
-                                Y[(size_t)s_perm[row0 + m] * N + nn] = __bfloat16_as_ushort(__float2bfloat16_rn(fin[4 * tb + j]));
+                            if (tb < NT && m < rows && nn < N) {
+                                const size_t at = (size_t)s_perm[row0 + m] * N + nn;
+                                float y = fin[4 * tb + j];
+                                if (R) y += __uint_as_float((uint32_t)R[at] << 16);
+                                Y[at] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+                            }
                         }
                     }
                 };
+                // gated pair: fin <- silu(fin) * other, the second expert's product of the same channels and rows
+                auto gate_with = [&](const float (&other)[8]) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) fin[i] = fin[i] / (1.f + expf(-fin[i])) * other[i];
+                };
+                float* xchg = reinterpret_cast<float*>(smem + L::xchg_off) + blob * 256 + lane;
                 if (kb0 == 0 && kb1 == KB) {
-                    store_rows();
+                    if (FUSED && gated) {
+                        // warps w and w + 8 hold the two products of the same channels: hand the second to the first
+                        if (half == 1) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) xchg[i * 32] = fin[i];
+                        }
+                        asm volatile("bar.sync %0, 64;" ::"r"(2 + blob) : "memory");
+                        if (half == 0) {
+                            float other[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) other[i] = xchg[i * 32];
+                            gate_with(other);
+                            store_rows();
+                        }
+                        asm volatile("bar.sync %0, 64;" ::"r"(2 + blob) : "memory");     // the buffer may be written again
+                    } else {
+                        store_rows();
+                    }
                 } else {
                     // part of a segment: park this warp's sums, announce, and add everything up if this was the last arrival
+                    // (for a gated pair the two warps of a blob share one counter and whoever is last finishes both products)
                     const long long C = *s_C, base = s_base[v];
                     const int G = *s_G, wv = p.w[v];
                     const int c_a = (int)(((base + (long long)(nt2 * KB) * wv) * G) / C);
@@ -617,26 +661,38 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                         for (int j = 0; j < 4; ++j)
                             if (tb < NT) __stcg(slot + ((warp * 2 + tb) * 4 + j) * 32 + lane, fin[4 * tb + j]);
                     __syncwarp();
+                    unsigned* counter = p.counters + c_a * GV_CONS + (gated ? blob : warp);
+                    const unsigned last = (unsigned)(gated ? 2 * (c_b - c_a) + 1 : c_b - c_a);
                     unsigned arrived = 0;
                     if (lane == 0) {
                         __threadfence();
-                        arrived = atomicAdd(p.counters + c_a * GV_CONS + warp, 1u);
+                        arrived = atomicAdd(counter, 1u);
                     }
                     arrived = __shfl_sync(0xffffffffu, arrived, 0);
-                    if (arrived == (unsigned)(c_b - c_a)) {
+                    if (arrived == last) {
                         __threadfence();
+                        auto gather = [&](int wsrc, float (&dst)[8]) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
-                        for (int c = c_a; c <= c_b; ++c) {
-                            const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
+                            for (int i = 0; i < 8; ++i) dst[i] = 0.f;
+                            for (int c = c_a; c <= c_b; ++c) {
+                                const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
 #pragma unroll
-                            for (int tb = 0; tb < 2; ++tb)
+                                for (int tb = 0; tb < 2; ++tb)
 #pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    if (tb < NT) fin[4 * tb + j] += __ldcg(src + ((warp * 2 + tb) * 4 + j) * 32 + lane);
+                                    for (int j = 0; j < 4; ++j)
+                                        if (tb < NT) dst[4 * tb + j] += __ldcg(src + ((wsrc * 2 + tb) * 4 + j) * 32 + lane);
+                            }
+                        };
+                        if (FUSED && gated) {
+                            float other[8];
+                            gather(blob, fin);
+                            gather(blob + 8, other);
+                            gate_with(other);
+                        } else {
+                            gather(warp, fin);
                         }
                         store_rows();
-                        if (lane == 0) p.counters[c_a * GV_CONS + warp] = 0u;
+                        if (lane == 0) *counter = 0u;
                     }
                 }
             }
@@ -691,8 +747,21 @@ size_t decode_workspace_bytes(int M) {
 moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const moqe_expert* const* ex, int E,
                                     void* const* Y, const int32_t* perm, const int32_t* offsets, void* ws,
                                     size_t ws_bytes, cudaStream_t st) {
+    return launch_qgemm_decode_ext(X, M, nl, ex, nullptr, E, Y, nullptr, perm, offsets, ws, ws_bytes, st);
+}
+
+// ex2 (or nullptr): per (layer, expert) the second expert of a gated pair, Y = silu(X.W1^T) * (X.W2^T), or nullptr for a
+// plain layer; R (or nullptr): per layer a residual [M][N] added before the rounding, or nullptr
+moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const moqe_expert* const* ex,
+                                  const moqe_expert* const* ex2, int E, void* const* Y, const void* const* R,
+                                  const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st) {
     if (M == 0) return MOQE_OK;
     if (!decode_supported_multi(M, ex, nl, E)) return MOQE_ERR_UNSUPPORTED;
+    if (ex2)
+        for (int v = 0; v < nl * E; ++v)
+            if (ex2[v] && (ex2[v]->N != ex[v]->N || ex2[v]->K != ex[v]->K || ex2[v]->bits != ex[v]->bits ||
+                           ex2[v]->group != ex[v]->group || ex2[v]->sym != ex[v]->sym))
+                return MOQE_ERR_MISMATCH;
     if (!ws || ws_bytes < decode_workspace_bytes(M)) return MOQE_ERR_WORKSPACE;
     GvParams p;
     for (int l = 0; l < nl; ++l)
@@ -707,6 +776,11 @@ moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const
             p.NT1[v] = ex[v]->Np / 128;
             p.rexp[v] = e;
             p.w[v] = g_dec_cost[ex[v]->bits];
+            const moqe_expert* second = ex2 ? ex2[v] : nullptr;
+            p.tiles2[v] = second ? second->tiles : nullptr;
+            p.scales_pc2[v] = second ? second->scales_pc : nullptr;
+            p.zeros_pc2[v] = second ? second->zeros_pc : nullptr;
+            p.Res[v] = R ? (const uint16_t*)R[l] : nullptr;
         }
     p.counters = (uint32_t*)ws;
     p.partials = (float*)((char*)ws + (decode_zero_bytes(M) + 255) / 256 * 256);
@@ -718,15 +792,18 @@ moqe_status launch_qgemm_decode_multi(const void* const* X, int M, int nl, const
     p.status = device_status_word();
     int grid = dec_sm_count();
     if (grid > GV_MAX_GRID) grid = GV_MAX_GRID;
-    cudaError_t err = cudaFuncSetAttribute(qgemm_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GvSmem::dyn_bytes);
+    const bool fused = ex2 != nullptr || R != nullptr;
+    const int smem = fused ? GvSmem<true>::dyn_bytes : GvSmem<false>::dyn_bytes;
+    auto kernel = fused ? qgemm_decode_kernel<true> : qgemm_decode_kernel<false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GV_THREADS); cfg.dynamicSmemBytes = GvSmem::dyn_bytes; cfg.stream = st;
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GV_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         at[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        err = cudaLaunchKernelEx(&cfg, qgemm_decode_kernel, p);
+        err = cudaLaunchKernelEx(&cfg, kernel, p);
     }
     if (err != cudaSuccess) return MOQE_ERR_CUDA;
     count_launch();
