@@ -254,6 +254,8 @@ def main():
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to moqe_tune (measurement knob)")
     ap.add_argument("--repeats", type=int, default=5, help="timings of --steps steps each; the median is reported")
     ap.add_argument("--no-workloads", action="store_true", help="skip the sub-records of the other workloads")
+    ap.add_argument("--fused-block", action="store_true",
+                    help="decode workloads: gate/up as ONE gated launch (silu(gate) * up), residual add in the o / down stores")
     args = ap.parse_args()
     w = wl.get(args.workload)
     heavy = w.kind in ("prefill", "mixed", "conv")
@@ -385,9 +387,15 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
         for j in g:
             used.add(j)
         groups.append(g)
+    fused_block = bool(args.fused_block) and max(L["M"] for L in layers) <= 16
     for g in groups:
+        Ls = [layers[j] for j in g]
+        names = tuple(L["spec"].name for L in Ls)
+        if fused_block and names == ("gate_proj", "up_proj"):
+            Ls[0]["gated"] = ((C.c_void_p * E)(*[e.handle for e in Ls[0]["experts"]]), (C.c_void_p * E)(*[e.handle for e in Ls[1]["experts"]]))
+        elif fused_block and names in (("o_proj",), ("down_proj",)):
+            Ls[0]["resid"] = torch.randn((Ls[0]["M"], Ls[0]["spec"].N), device=dev).to(torch.bfloat16)
         if len(g) > 1:
-            Ls = [layers[j] for j in g]
             layers[g[0]]["multi"] = ((C.c_void_p * len(g))(*[L["X"].data_ptr() for L in Ls]),
                                      (C.c_void_p * len(g))(*[L["Y"].data_ptr() for L in Ls]),
                                      (C.c_void_p * (len(g) * E))(*[e.handle for L in Ls for e in L["experts"]]))
@@ -409,7 +417,13 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
 
     def run_group(g, perm, offsets):
         Ls = [layers[j] for j in g]
-        if len(g) > 1:
+        if "gated" in Ls[0]:
+            moqe.moqe_routed_qgemm_sorted_gated(Ls[0]["X"], perm, offsets, Ls[0]["experts"], Ls[1]["experts"], Ls[0]["Y"],
+                                                Ls[0]["ws"], _arrs=Ls[0]["gated"])
+        elif "resid" in Ls[0]:
+            L = Ls[0]
+            moqe.moqe_routed_qgemm_sorted_residual(L["X"], perm, offsets, L["experts"], L["resid"], L["Y"], L["ws"], _arr=L["arr"])
+        elif len(g) > 1:
             moqe.moqe_routed_qgemm_sorted_multi([L["X"] for L in Ls], perm, offsets, [L["experts"] for L in Ls],
                                                 [L["Y"] for L in Ls], Ls[0]["ws"], _arrs=Ls[0]["multi"])
         else:
@@ -519,6 +533,10 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
             if cnt[e] > 0:
                 b += ex.code_bytes + ex.meta_bytes
         a = L["M"] * L["spec"].K * 2 + L["M"] * L["spec"].N * 2
+        if fused_block and L["spec"].name == "up_proj":
+            a -= L["M"] * L["spec"].N * 2                    # the gated launch writes one output for the pair
+        if "resid" in L:
+            a += L["M"] * L["spec"].N * 2                    # the residual is read
         alg_bytes.append(b + a)
         act_bytes.append(a)
         flops.append(2.0 * L["M"] * L["spec"].N * L["spec"].K)
@@ -566,6 +584,10 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
                    "l2": "weights of one block exceed L2 (inputs larger than L2, no flush)" if sum(alg_bytes) > 126e6
                          else "working set fits L2", "cuda_graph": bool(graph_launches), "path": args.path,
                    "timing": f"median of {max(1, repeats)} repeats of {steps} steps",
+                   "fused_block": ({"gate_up": "one gated launch, silu(gate) * up", "o_down": "residual added in the store",
+                                    "bytes_not_moved_per_step": int(sum(3 * L["M"] * L["spec"].N * 2 for L in layers if L["spec"].name == "up_proj")),
+                                    "note": "the [M][N] bf16 outputs of gate and up are never written nor re-read by a separate "
+                                            "silu-mul kernel, which would also write its own output"} if fused_block else False),
                    "launch_groups": ["+".join(layers[j]["spec"].name for j in g) for g in groups]},
         "roofline": roofline, "gpu_launches": int(launches), "device_status": moqe.status_str(status),
     }
