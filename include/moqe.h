@@ -248,7 +248,10 @@ MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_id
 /* Same, with the kernel chosen by the caller (testing / measurement):
  * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM (automatic
  * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles, 5 = decode kernel
- * (MOQE_ERR_UNSUPPORTED if the batch has more than 16 rows or an expert has groups narrower than 128 k). */
+ * (MOQE_ERR_UNSUPPORTED if the batch has more than 16 rows or an expert has groups narrower than 128 k),
+ * 6 = dense-weights tcgen05 GEMM for large batches on small layers (more than 128 rows, K <= 1024, at most 1024
+ * output channels; the automatic choice there: the layer is bound by its activations, so each expert's weights
+ * are expanded to bf16 once per call and X / Y are streamed; MOQE_ERR_UNSUPPORTED otherwise). */
 MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
                                    const moqe_expert* const* h_experts, int E, void* Y_bf16,
                                    void* workspace, size_t workspace_bytes, void* stream, int path);
@@ -307,6 +310,7 @@ MOQE_API const char* moqe_status_str(moqe_status s);
  *                            (defaults 8 / 8 / 8).
  *   "decode_tile_cost_w8" / "_w4" / "_w3" : the same for the decode kernel (defaults 10 / 10 / 10).
  *   "auto_decode"          : whether path 0 takes the decode kernel where it applies (default 1).
+ *   "auto_dense"           : whether path 0 takes the dense-weights GEMM where it applies (default 1).
  * Unknown key: MOQE_ERR_UNSUPPORTED. */
 MOQE_API moqe_status moqe_tune(const char* key, int value);
 

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libmoqe.so")
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_WORKSPACE, ERR_MISMATCH, ERR_CUDA, ERR_EXPERT_ID, ERR_TIMEOUT, ERR_IO = range(1, 11)
 MAX_EXPERTS = 32
-PATH_AUTO, PATH_STREAM, PATH_TCGEN05, PATH_DECODE = 0, 1, 2, 5
+PATH_AUTO, PATH_STREAM, PATH_TCGEN05, PATH_DECODE, PATH_DENSE = 0, 1, 2, 5, 6
 
 EXPORTED = (
     "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",

@@ -46,22 +46,30 @@ WsLayout ws_layout(int M, int Np, int K, int E) {
     w.sort = off;    off += align256(sort_workspace_bytes(M, E));
     w.body = off;
     size_t a = stream_workspace_bytes(M, Np, E), b = tc_workspace_bytes(M, K, E, Np), c = decode_workspace_bytes(M);
+    const size_t d = dense_workspace_bytes(M, K, E, Np, (K + 127) / 128 * 128);
     a = a > b ? a : b;
+    a = a > d ? a : d;
     off += align256(a > c ? a : c);
     w.total = off;
     return w;
 }
 
 constexpr int AUTO_STREAM_MAX_ROWS = 128;
-constexpr int LAST_PATH = 5;
+constexpr int LAST_PATH = 6;
 
 bool g_auto_decode = true;   // whether the automatic choice takes a decode kernel where it applies
+bool g_auto_dense = true;    // ... and the dense-weights GEMM for large batches on small layers
 
-// 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = decode kernel
+// 0 = tcgen05 grouped GEMM, 1 = mma.sync streaming kernel, 2 = decode kernel, 3 = dense-weights GEMM (small layers)
 int pick_kernel(int path, int M, const moqe_expert* const* ex, int E) {
     if (path == 5) return 2;
+    if (path == 6) return 3;
     if (path == 1) return 1;
-    if (path == 0) return (g_auto_decode && decode_supported_multi(M, ex, 1, E)) ? 2 : (M <= AUTO_STREAM_MAX_ROWS ? 1 : 0);
+    if (path == 0) {
+        if (g_auto_decode && decode_supported_multi(M, ex, 1, E)) return 2;
+        if (M <= AUTO_STREAM_MAX_ROWS) return 1;
+        return (g_auto_dense && dense_supported(M, ex[0]->N, ex[0]->K, ex, E)) ? 3 : 0;
+    }
     return 0;
 }
 
@@ -115,6 +123,8 @@ extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t*
     if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
+    if (kernel == 3)
+        return launch_qgemm_dense(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
     tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
     return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
@@ -146,6 +156,8 @@ extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_
     if (kernel == 1)
         return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
                                    w.total - w.body, st);
+    if (kernel == 3)
+        return launch_qgemm_dense(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
     tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
     return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
@@ -247,6 +259,7 @@ extern "C" moqe_status moqe_tune(const char* key, int value) {
     if (!strcmp(key, "stream_tile_cost_w4")) { stream_set_tile_cost(4, value); return MOQE_OK; }
     if (!strcmp(key, "stream_tile_cost_w3")) { stream_set_tile_cost(3, value); return MOQE_OK; }
     if (!strcmp(key, "auto_decode")) { g_auto_decode = value != 0; return MOQE_OK; }
+    if (!strcmp(key, "auto_dense")) { g_auto_dense = value != 0; return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w8")) { decode_set_tile_cost(8, value); return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w4")) { decode_set_tile_cost(4, value); return MOQE_OK; }
     if (!strcmp(key, "decode_tile_cost_w3")) { decode_set_tile_cost(3, value); return MOQE_OK; }

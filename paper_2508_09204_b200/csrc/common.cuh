@@ -129,6 +129,15 @@ moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const m
                                     const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st);
 void decode_set_tile_cost(int bits, int cost);   // relative cost of one super-tile in the work split, by code width
 
+// quantize.cu: a plain bf16 copy Wd[Np][2 Kp] (hi | lo halves) of a (small) expert and its per-channel output scale, for qgemm_dense.cu
+moqe_status launch_dense_unpack(const moqe_expert* const* ex, int E, uint16_t* Wd, float* col_scale, cudaStream_t st);   // experts that agree on N and K, one launch: Wd[E][Np][2 Kp], col_scale[E][Np]
+
+// qgemm_dense.cu: large batches on layers whose weights are small (activation-bound, e.g. 1x1 convolutions)
+bool dense_supported(int M, int N, int K, const moqe_expert* const* ex, int E);
+size_t dense_workspace_bytes(int M, int K, int E, int Np, int Kp);
+moqe_status launch_qgemm_dense(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
+                               const int32_t* perm, const int32_t* offsets, void* ws, size_t ws_bytes, cudaStream_t st);
+
 // qgemm_tcgen05.cu
 void tc_set_tile_tokens(int tn);   // 0 = automatic, else 128 or 256 (testing / measurement)
 size_t tc_workspace_bytes(int M, int K, int E, int Np);

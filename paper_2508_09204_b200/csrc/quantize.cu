@@ -454,6 +454,92 @@ extern "C" moqe_status moqe_expert_destroy(moqe_expert* e) {
     return (a == cudaSuccess && b == cudaSuccess && c == cudaSuccess) ? MOQE_OK : MOQE_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------- dense copy of a small expert
+// For layers whose weights are a few hundred kilobytes (1x1 convolutions) the routed product is bound by the
+// activations, and the weights are best handed to the tensor cores as a plain bf16 matrix Wd[Np][Kp] (row = output
+// channel, K contiguous).  Per-channel experts: Wd = c - z, an exact small integer, and col_scale[n] = the channel's
+// scale, applied to the fp32 sums.  Grouped experts: s * (c - z) (exact in fp32) is split into two bf16 numbers,
+// hi = bf16(w) in columns [0, Kp) and lo = bf16(w - hi) in columns [Kp, 2 Kp), and col_scale[n] = 1: the caller
+// multiplies the activations by both halves, which leaves a relative error of 2^-17 per weight.  Rows are 2 Kp wide.
+namespace moqe {
+namespace {
+struct DenseSrc {
+    const uint8_t* tiles[MOQE_MAX_EXPERTS];
+    const __half* scales_pc[MOQE_MAX_EXPERTS];
+    const __nv_bfloat16* zeros_pc[MOQE_MAX_EXPERTS];
+    int bits[MOQE_MAX_EXPERTS], group[MOQE_MAX_EXPERTS], sym[MOQE_MAX_EXPERTS];
+};
+
+template <int BITS>
+__device__ __forceinline__ void dense_unpack_piece(const uint8_t* __restrict__ tiles, const __half* __restrict__ scales_pc,
+                                                   const __nv_bfloat16* __restrict__ zeros_pc, int N, int K, int Kp, int KB, int group,
+                                                   int sym, uint16_t* __restrict__ Wd, float* __restrict__ col_scale, long long pid) {
+    PieceCoord pc = piece_coord(pid, KB);
+    const int stride = moqe_tile_stride(BITS, group, !sym);
+    uint32_t w[PieceWords<BITS>::n];
+    load_piece<BITS>(tiles + pc.tile_index * (size_t)stride + pc.nb * moqe_blob_bytes(BITS), pc.half, pc.slot, w);
+    uint32_t c[32];
+    decode_piece<BITS>(w, c);
+    const bool live = pc.n < N;
+    if (pc.kb == 0 && pc.q == 0) col_scale[pc.n] = !live ? 0.f : (group == 0 ? __half2float(scales_pc[pc.n]) : 1.f);
+#pragma unroll
+    for (int G = 0; G < 4; ++G) {
+        const int k0 = pc.kb * 128 + 32 * G + 8 * pc.q;
+        uint32_t o[4] = {0u, 0u, 0u, 0u}, o2[4] = {0u, 0u, 0u, 0u};
+        if (live && k0 < K) {
+            float s = 1.f, z = (float)(1 << (BITS - 1));
+            if (group == 0) {
+                if (!sym) z = __bfloat162float(zeros_pc[pc.n]);
+            } else {
+                MetaSlot m = meta_slot(const_cast<uint8_t*>(tiles), nullptr, nullptr, BITS, group, !sym, KB, pc.n, k0 / group, 0);
+                s = __half2float(*m.s);
+                if (!sym) z = __bfloat162float(*m.z);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float w0 = s * ((float)c[8 * G + 2 * i] - z), w1 = s * ((float)c[8 * G + 2 * i + 1] - z);
+                __nv_bfloat162 v = __floats2bfloat162_rn(w0, w1);
+                o[i] = *reinterpret_cast<uint32_t*>(&v);
+                if (group != 0) {
+                    __nv_bfloat162 r = __floats2bfloat162_rn(w0 - __low2float(v), w1 - __high2float(v));
+                    o2[i] = *reinterpret_cast<uint32_t*>(&r);
+                }
+            }
+        }
+        *reinterpret_cast<uint4*>(Wd + (size_t)pc.n * 2 * Kp + k0) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(Wd + (size_t)pc.n * 2 * Kp + Kp + k0) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
+    }
+}
+
+// blockIdx.y = expert
+__global__ void dense_unpack_kernel(const __grid_constant__ DenseSrc src, int N, int K, int Np, int Kp, int KB,
+                                    uint16_t* __restrict__ Wd, float* __restrict__ col_scale, long long npieces) {
+    const long long pid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pid >= npieces) return;
+    const int e = blockIdx.y;
+    uint16_t* wd = Wd + (size_t)e * Np * 2 * Kp;
+    float* cs = col_scale + (size_t)e * Np;
+    if (src.bits[e] == 4) dense_unpack_piece<4>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
+    else if (src.bits[e] == 8) dense_unpack_piece<8>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
+    else dense_unpack_piece<3>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
+}
+}  // namespace
+
+moqe_status launch_dense_unpack(const moqe_expert* const* ex, int E, uint16_t* Wd, float* col_scale, cudaStream_t st) {
+    DenseSrc src;
+    for (int e = 0; e < E; ++e) {
+        src.tiles[e] = ex[e]->tiles; src.scales_pc[e] = ex[e]->scales_pc; src.zeros_pc[e] = ex[e]->zeros_pc;
+        src.bits[e] = ex[e]->bits; src.group[e] = ex[e]->group; src.sym[e] = ex[e]->sym;
+    }
+    const int KB = ex[0]->Kp / 128;
+    const long long npieces = (long long)(ex[0]->Np / 128) * KB * 512;
+    dense_unpack_kernel<<<dim3((unsigned)((npieces + 127) / 128), E), 128, 0, st>>>(src, ex[0]->N, ex[0]->K, ex[0]->Np, ex[0]->Kp, KB, Wd,
+                                                                                  col_scale, npieces);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+}  // namespace moqe
+
 // ---------------------------------------------------------------------------- expert residency
 // Section 4.4 of the paper and its appendix table "Router model and expert loading overhead": one expert is kept on
 // the GPU, the others wait in CPU RAM (or on disk) and are loaded when the routing changes.  A packed expert is a

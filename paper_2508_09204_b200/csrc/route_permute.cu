@@ -200,9 +200,10 @@ __global__ void move_rows_kernel(const uint4* __restrict__ src, const int32_t* _
 // consecutive rows of X anyway (the usual case: a sample's rows are contiguous and share an expert) is NOT
 // copied: box_src[id] = its first source row, and the GEMM's TMA reads X directly; otherwise the rows are
 // copied to Xp[offsets[e] + 64*box ..] and box_src[id] = -1.
-__global__ void __launch_bounds__(256) gather_boxes_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ perm,
-                                                           const int32_t* __restrict__ offsets, int E, int vec_per_row,
-                                                           uint4* __restrict__ Xp, int32_t* __restrict__ box_src) {
+// (wide rows: one block per box, so that a box that has to be copied has 256 threads and the grid many blocks)
+__global__ void __launch_bounds__(256) gather_boxes_wide_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ perm,
+                                                                const int32_t* __restrict__ offsets, int E, int vec_per_row,
+                                                                uint4* __restrict__ Xp, int32_t* __restrict__ box_src) {
     int b = blockIdx.x, e = 0, rows_e = 0;
     for (; e < E; ++e) {
         rows_e = offsets[e + 1] - offsets[e];
@@ -220,6 +221,45 @@ __global__ void __launch_bounds__(256) gather_boxes_kernel(const uint4* __restri
     for (int i = threadIdx.x; i < cnt * vec_per_row; i += blockDim.x) {
         const int r = i / vec_per_row, v = i - r * vec_per_row;
         Xp[(size_t)(j0 + r) * vec_per_row + v] = X[(size_t)perm[j0 + r] * vec_per_row + v];
+    }
+}
+
+// (narrow rows, many boxes: eight boxes per block)
+__global__ void __launch_bounds__(256) gather_boxes_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ perm,
+                                                           const int32_t* __restrict__ offsets, int E, int vec_per_row,
+                                                           uint4* __restrict__ Xp, int32_t* __restrict__ box_src, int nboxes) {
+    // one warp per box looks at its 64 rows (lanes: rows l and l + 32); the boxes of the block that have to be
+    // copied are then copied by the whole block
+    __shared__ int s_j0[8], s_cnt[8];
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int box = blockIdx.x * 8 + wib;
+    int j0 = 0, cnt = 0;
+    if (box < nboxes) {
+        int b = box, e = 0, rows_e = 0;
+        for (; e < E; ++e) {
+            rows_e = offsets[e + 1] - offsets[e];
+            const int nb = (rows_e + 63) >> 6;
+            if (b < nb) break;
+            b -= nb;
+        }
+        if (e < E) {
+            j0 = offsets[e] + b * 64;
+            cnt = min(64, rows_e - b * 64);
+            const int first = perm[j0];
+            const bool ok = (lane >= cnt || perm[j0 + lane] == first + lane) && (lane + 32 >= cnt || perm[j0 + lane + 32] == first + lane + 32);
+            const bool all_ok = __all_sync(0xffffffffu, ok);
+            if (lane == 0) box_src[box] = all_ok ? first : -1;
+            if (all_ok) cnt = 0;
+        }
+    }
+    if (lane == 0) { s_j0[wib] = j0; s_cnt[wib] = cnt; }
+    __syncthreads();
+    for (int w = 0; w < 8; ++w) {
+        const int c = s_cnt[w], base = s_j0[w];
+        for (int i = threadIdx.x; i < c * vec_per_row; i += blockDim.x) {
+            const int r = i / vec_per_row, v = i - r * vec_per_row;
+            Xp[(size_t)(base + r) * vec_per_row + v] = X[(size_t)perm[base + r] * vec_per_row + v];
+        }
     }
 }
 
@@ -273,7 +313,11 @@ size_t gather_boxes_bytes(int M, int E) { return ((size_t)(M / 64 + E + 1) * siz
 moqe_status launch_gather_boxes(const void* X, const int32_t* perm, const int32_t* offsets, int M, int C, int E, void* Xp,
                                 int32_t* box_src, cudaStream_t st) {
     if (M == 0) return MOQE_OK;
-    gather_boxes_kernel<<<M / 64 + E, 256, 0, st>>>((const uint4*)X, perm, offsets, E, C / 8, (uint4*)Xp, box_src);
+    const int nboxes = M / 64 + E;
+    if (C >= 512 || nboxes < 2048)
+        gather_boxes_wide_kernel<<<nboxes, 256, 0, st>>>((const uint4*)X, perm, offsets, E, C / 8, (uint4*)Xp, box_src);
+    else
+        gather_boxes_kernel<<<(nboxes + 7) / 8, 256, 0, st>>>((const uint4*)X, perm, offsets, E, C / 8, (uint4*)Xp, box_src, nboxes);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }

@@ -248,6 +248,29 @@ def test_tcgen05_kernel_full_token_tiles_every_element():
         assert_close(Y, oracle.routed_gemm(X, ids, What), f"path {path}, M{M} N{N} K{K}")
 
 
+@pytest.mark.parametrize("M,N,K", [(200, 64, 256), (777, 256, 64), (1500, 1000, 1024), (392, 264, 200)])
+def test_dense_weights_kernel(M, N, K):
+    """The dense-weights GEMM (path 6: large batches on small layers): per-channel, grouped and 32-k-group experts,
+    per-image-like runs of rows and scattered rows, ragged tiles, ragged N and K, an idle expert; every element."""
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import build_experts, assert_close
+    specs = [f for f in [(8, 0, True), (4, 0, False), (4, 32, False), (3, 64, False), (8, 128, False)] if f[1] == 0 or K % f[1] == 0]
+    W = wl.weights_f32(f"dn/{N}/{K}", N, K)
+    X = wl.activations_bf16(f"dn/{M}/{K}", M, K, relu=True)
+    gpu, What, _ = build_experts(W, specs)
+    E = len(specs)
+    rs = np.random.default_rng(M + N)
+    for routing in ("runs", "scattered"):
+        if routing == "runs":                                    # whole runs of 64 rows share an expert (read in place)
+            ids = np.repeat(rs.integers(0, E, size=(M + 63) // 64), 64)[:M].astype(np.int32)
+        else:
+            ids = rs.integers(0, E, size=M).astype(np.int32)
+        ids[ids == 1] = 0                                        # expert 1 idle
+        Y, st = _run(X, ids, gpu, moqe.PATH_DENSE)
+        assert st == moqe.OK
+        assert_close(Y, oracle.routed_gemm(X, ids, What), f"dense {routing} M{M} N{N} K{K}")
+
+
 def test_argument_errors():
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, dev
