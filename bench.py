@@ -561,7 +561,9 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
         roofline = {"bound": "hbm", **hbm, "traffic": traffic,
                     "frac_whole_step": sum(alg_bytes) / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     max_m = max(L["M"] for L in layers)
-    kernel = "qgemm_tc_kernel" if max_m > 128 else ("qgemm_decode_kernel" if max_m <= 16 else "qgemm_stream_kernel")
+    small = all(L["spec"].N <= 1024 and L["spec"].K <= 1024 for L in layers)     # the library's dense-weights rule
+    kernel = (("qgemm_dense_kernel" if small and args.path == 0 else "qgemm_tc_kernel") if max_m > 128
+              else ("qgemm_decode_kernel" if max_m <= 16 else "qgemm_stream_kernel"))
     roofline.update({"peak_source": peaks["source"],
                      "kernel": kernel + f": average of the {n_launch} routed-GEMM launches of one block" +
                                (" (q/k/v and gate/up each in one launch)" if any(len(g) > 1 for g in groups) else ""),
