@@ -10,7 +10,7 @@
 //                           128-bit shared loads, unpacks them in registers and issues warp-level tensor-core MMAs
 //                           (fp16 operands, fp32 accumulation) against the token fragments; it applies the group's
 //                           scale in fp32 once per k-block and keeps the running sums of its piece in registers.
-//   4 service warps       : stage the token rows one chunk of k-blocks ahead, double buffered: gathered through
+//   2 service warps       : stage the token rows one chunk of k-blocks ahead, double buffered: gathered through
 //                           `perm` (the fused permutation), converted from bf16 to scaled fp16 in MMA fragment order,
 //                           with their sums.  Chunk descriptors travel with the buffers, so the consumers follow the
 //                           work split without walking it themselves.
@@ -361,12 +361,14 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
     __syncthreads();
     const int nstg = s_geom[0], stage_bytes = s_geom[1];
 
-    // ---- staging of one chunk of token rows by `nthr` threads (this one is number st of them).  A thread takes whole
-    // row tiles -- the 128 values X[row m][k-block] -- one after the other: sixteen 16-byte fetches (eight in flight),
-    // each converted to four fp16 pairs in MMA fragment order, and the row tile's sums, which need no exchange between
-    // threads.  The caller's walk is advanced past the chunk.  Returns false when there was no chunk left (an invalid
-    // descriptor has been written).
-    auto stage_chunk = [&](GvWalk& wk, int& kbc, bool& more, int n, int nthr, int st) -> bool {
+    // ---- staging of one chunk of token rows by `nthr` threads (a multiple of 32; this one is number st of them, st % 32 its
+    // lane).  A row tile -- the 128 values X[row m][k-block] -- is sixteen 16-byte fetches, each converted to four fp16
+    // pairs in MMA fragment order, plus the row tile's sums.  The service warps give a thread whole row tiles (eight
+    // fetches in flight, no exchange between threads); the first chunk, staged by all warps together, gives it one
+    // 32-value group of a row tile (one fetch latency; the sums are added up over four lanes).  The caller's walk is
+    // advanced past the chunk.  Returns false when there was no chunk left (an invalid descriptor has been written).
+    auto stage_chunk = [&](auto parts_tag, GvWalk& wk, int& kbc, bool& more, int n, int nthr, int st) -> bool {
+        constexpr int PARTS = decltype(parts_tag)::value;       // threads per row tile: 1, or 4 (one 32-value group each)
         const int buf = n & 1;
         ChunkDesc* d = s_desc + buf;
         if (!more) {
@@ -383,50 +385,82 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
         const uint32_t xbuf = sbase + L::x_off + buf * GV_XBUF;
         float* sbuf = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF);
-        // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block
-        const int tiles = nkb * NT * 8;
-        for (int rt = st; rt < tiles; rt += nthr) {
+        // one 16-byte fetch (chunk a = 4G + q of the k-block: k = 32G + 8q ..) -> four fp16 pairs in MMA fragment order at
+        // [slab][G][lane = 4 mm + q]; the pair sums go into the group's partial sums
+        auto convert = [&](const uint4& dat, int a, uint32_t xdst, float& S0, float& S1) {
+            const int G = a >> 2, q = a & 3;
+            const uint32_t w[4] = {dat.x, dat.y, dat.z, dat.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
+                const int e = sigma_shift(bits, 4 * G + j);
+                const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
+                const float sum = lo + hi;
+                S0 += sum;
+                S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
+                __half2 hh = __floats2half2_rn(lo, hi);
+                const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
+                hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
+                o[j] = *reinterpret_cast<uint32_t*>(&hh);
+            }
+            sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
+        };
+        // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block.  The sums of a row tile are
+        // (g0 + g1) + (g2 + g3) over its four 32-value groups, whoever stages it.
+        const int units = nkb * NT * 8 * PARTS;
+        for (int u0 = st & ~31; u0 < units; u0 += nthr) {
+            const int unit = u0 + (st & 31);
+            const bool live = unit < units;
+            const int rt = unit / PARTS, part = unit % PARTS;
             const int slab = rt >> 3, mm = rt & 7;
             const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
             const int k0 = (kbc + kbl) * 128;
-            const uint16_t* src = m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
+            const uint16_t* src = live && m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
             const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
-            float S0 = 0.f, S1 = 0.f;
+            float S0, S1;
+            if constexpr (PARTS == 4) {
+                uint4 data[4];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint4 data[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int a = 8 * h + i;
+                for (int i = 0; i < 4; ++i) {
+                    const int a = 4 * part + i;
                     data[i] = make_uint4(0, 0, 0, 0);
                     if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
                 }
+                S0 = 0.f; S1 = 0.f;
+                if (live) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int a = 8 * h + i, G = a >> 2, q = a & 3;       // chunk (G, q) of the k-block: k = 32G + 8q ..
-                    const uint32_t w[4] = {data[i].x, data[i].y, data[i].z, data[i].w};
-                    uint32_t o[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
-                        const int e = sigma_shift(bits, 4 * G + j);
-                        const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
-                        const float sum = lo + hi;
-                        S0 += sum;
-                        S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
-                        __half2 hh = __floats2half2_rn(lo, hi);
-                        const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
-                        hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
-                        o[j] = *reinterpret_cast<uint32_t*>(&hh);
-                    }
-                    // fragments at [slab][G][lane = 4 mm + q]
-                    sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
+                    for (int i = 0; i < 4; ++i) convert(data[i], 4 * part + i, xdst, S0, S1);
                 }
+                S0 += __shfl_xor_sync(0xffffffffu, S0, 1);
+                S1 += __shfl_xor_sync(0xffffffffu, S1, 1);
+                S0 += __shfl_xor_sync(0xffffffffu, S0, 2);
+                S1 += __shfl_xor_sync(0xffffffffu, S1, 2);
+            } else {
+                float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint4 data[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int a = 8 * h + i;
+                        data[i] = make_uint4(0, 0, 0, 0);
+                        if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
+                    }
+                    if (live) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) convert(data[i], 8 * h + i, xdst, g0[2 * h + (i >> 2)], g1[2 * h + (i >> 2)]);
+                    }
+                }
+                S0 = (g0[0] + g0[1]) + (g0[2] + g0[3]);
+                S1 = (g1[0] + g1[1]) + (g1[2] + g1[3]);
             }
             // sums at [slab][t = mm / 2][4]
-            float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
-            S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
-            S[2] = S0;
+            if (live && part == 0) {
+                float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
+                S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
+                S[2] = S0;
+            }
         }
         kbc += nkb;
         if (kbc >= kb1) {
@@ -442,7 +476,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
     bool s_changed, s_more = swk.next(s_pair, p, s_changed);
     int s_kbc = s_more ? swk.kb : 0;
     if (warp < GV_CONS + GV_SERV) {
-        stage_chunk(swk, s_kbc, s_more, 0, (GV_CONS + GV_SERV) * 32, tid);
+        stage_chunk(std::integral_constant<int, 4>{}, swk, s_kbc, s_more, 0, (GV_CONS + GV_SERV) * 32, tid);
         asm volatile("bar.sync 1, %0;" ::"n"((GV_CONS + GV_SERV) * 32) : "memory");   // (the producer is already streaming)
     }
 
@@ -485,7 +519,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         for (int n = 1;; ++n) {
             const int buf = n & 1;
             if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_xempty + 8 * buf, (uint32_t)((n >> 1) - 1) & 1u, s_abort, p.status))) break;
-            const bool staged = stage_chunk(swk, s_kbc, s_more, n, GV_SERV * 32, st);
+            const bool staged = stage_chunk(std::integral_constant<int, 1>{}, swk, s_kbc, s_more, n, GV_SERV * 32, st);
             mbar_arrive(bar_xfull + 8 * buf);
             if (!staged) break;
         }
