@@ -73,19 +73,28 @@ struct GvSmem {
     static constexpr int pair_off = perm_off + 16 * 4;                    // {tb, te} per pair
     static constexpr int base_off = pair_off + MOQE_MAX_EXPERTS * 8;     // cost before each pair (long long)
     static constexpr int misc_off = base_off + MOQE_MAX_EXPERTS * 8;     // C (long long), G, stages, stage bytes, abort
-    static constexpr int total = misc_off + 32;
+    static constexpr int ps_off = misc_off + 32;                         // the pairs' scalars (a copy of GvParams::ps)
+    static constexpr int total = ps_off + MOQE_MAX_EXPERTS * 48;
     static constexpr int dyn_bytes = total;
 };
 static_assert(GvSmem<false>::dyn_bytes <= 227 * 1024 && GvSmem<true>::dyn_bytes <= 227 * 1024, "shared memory budget");
 
+// what the kernel needs to know about a (layer, expert) pair besides pointers; copied to shared memory on entry
+struct PairS {
+    int bits, group, has_zeros, stride;     // the expert's format; bytes of one packed tile
+    int N, K, KB, NT1;                      // the layer's shape; k-blocks; 128-channel tiles
+    int rexp;                               // the routing expert whose rows the pair takes
+    int w;                                  // cost of one super-tile
+    int gated;                              // a gated pair (see tiles2)
+    int pad;
+};
+static_assert(sizeof(PairS) == 48, "PairS is copied word by word");
+
 struct GvParams {
     ExpertDev ex[MOQE_MAX_EXPERTS];         // per (layer, expert) pair
+    PairS ps[MOQE_MAX_EXPERTS];
     const uint16_t* X[MOQE_MAX_EXPERTS];    // the layer's input and output
     uint16_t* Y[MOQE_MAX_EXPERTS];
-    int N[MOQE_MAX_EXPERTS], K[MOQE_MAX_EXPERTS], KB[MOQE_MAX_EXPERTS];
-    int NT1[MOQE_MAX_EXPERTS];              // 128-channel tiles of the layer
-    int rexp[MOQE_MAX_EXPERTS];             // the routing expert whose rows the pair takes
-    int w[MOQE_MAX_EXPERTS];                // cost of one super-tile
     // A gated pair (tiles2 != nullptr): the pair's second expert (same format and shape), whose product multiplies
     // silu of the first one's; the super-tile is then {tile nt of the first, tile nt of the second}.
     const uint8_t* tiles2[MOQE_MAX_EXPERTS];
@@ -98,6 +107,7 @@ struct GvParams {
     uint32_t* counters;                     // [CTA][warp]: arrivals for the segment whose head that CTA holds; zero on entry, left zero
     int* status;
     int M, R, P;                            // rows of the batch, routing experts, pairs
+    int small;                              // (total cost) x (grid) fits 31 bits: the work split runs in 32-bit arithmetic
 };
 
 // one chunk of work: k-blocks [kbc, kbc + nkb) of segment (pair v, channel-tile pair nt2), part of the piece [kb0, kb1)
@@ -109,13 +119,13 @@ struct GvWalk {
     int v, st, te, kb, KB, nt2;
     __device__ __forceinline__ void start() { v = -1; st = te = kb = nt2 = 0; KB = 1; }
     // opens the next run; returns false at the end.  `changed`: the run belongs to another pair than the last one
-    __device__ __forceinline__ bool next(const int* s_pair, const GvParams& p, bool& changed) {
+    __device__ __forceinline__ bool next(const int* s_pair, const PairS* ps, int P, bool& changed) {
         changed = false;
         if (v >= 0) st += run();
         if (v < 0 || st >= te) {
-            do { ++v; } while (v < p.P && s_pair[2 * v + 1] <= s_pair[2 * v]);
-            if (v >= p.P) return false;
-            st = s_pair[2 * v]; te = s_pair[2 * v + 1]; KB = p.KB[v];
+            do { ++v; } while (v < P && s_pair[2 * v + 1] <= s_pair[2 * v]);
+            if (v >= P) return false;
+            st = s_pair[2 * v]; te = s_pair[2 * v + 1]; KB = ps[v].KB;
             nt2 = st / KB; kb = st - nt2 * KB;
             changed = true;
         } else {
@@ -297,8 +307,10 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
     int* s_geom = reinterpret_cast<int*>(smem + L::misc_off + 12);          // {stages, stage bytes}
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::misc_off + 20);
     ChunkDesc* s_desc = reinterpret_cast<ChunkDesc*>(smem + L::desc_off);
+    const PairS* s_ps = reinterpret_cast<const PairS*>(smem + L::ps_off);
 
     // ---- prologue: nothing here depends on the previous kernel in the stream
+    if (tid < p.P * 12) reinterpret_cast<int*>(smem + L::ps_off)[tid] = reinterpret_cast<const int*>(p.ps)[tid];
     if (tid == 0) {
         for (int i = 0; i < GV_MAX_STAGES; ++i) { mbar_init(bar_wfull + 8 * i, 1); mbar_init(bar_wempty + 8 * i, GV_CONS); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_xfull + 8 * i, GV_SERV * 32); mbar_init(bar_xempty + 8 * i, GV_CONS); }
@@ -317,9 +329,10 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         long long cost = 0;
         int TT = 0, wv = 1;
         if (v < p.P) {
-            const int rows = p.offsets[p.rexp[v] + 1] - p.offsets[p.rexp[v]];
-            wv = p.w[v];
-            TT = rows > 0 ? ((FUSED && p.tiles2[v]) ? p.NT1[v] : (p.NT1[v] + 1) >> 1) * p.KB[v] : 0;
+            const PairS q = p.ps[v];
+            const int rows = p.offsets[q.rexp + 1] - p.offsets[q.rexp];
+            wv = q.w;
+            TT = rows > 0 ? ((FUSED && q.gated) ? q.NT1 : (q.NT1 + 1) >> 1) * q.KB : 0;
             cost = (long long)TT * wv;
         }
         long long incl = cost;
@@ -332,21 +345,30 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         }
         const long long C = __shfl_sync(0xffffffffu, incl, 31);
         const long long base = incl - cost;
-        const long long Gl = C / wmax;                          // every CTA's share holds at least one super-tile start
+        // every CTA's share holds at least one super-tile start
+        const long long Gl = p.small ? (long long)((unsigned)C / (unsigned)wmax) : C / wmax;
         const int G = (int)(Gl < (long long)gridDim.x ? Gl : (long long)gridDim.x);
         int tb = 0, te = 0, str = 0;
         if (v < p.P) {
             if (TT > 0 && (int)blockIdx.x < G) {
                 const long long den = (long long)wv * G;
                 const long long n0 = (long long)blockIdx.x * C - base * G, n1 = (long long)(blockIdx.x + 1) * C - base * G;
-                const long long t0 = n0 <= 0 ? 0 : (n0 + den - 1) / den, t1 = n1 <= 0 ? 0 : (n1 + den - 1) / den;
+                long long t0, t1;
+                if (p.small) {                                  // the same quotients from 32-bit divisions
+                    const unsigned d32 = (unsigned)den;
+                    t0 = n0 <= 0 ? 0 : (long long)(((unsigned)n0 + d32 - 1) / d32);
+                    t1 = n1 <= 0 ? 0 : (long long)(((unsigned)n1 + d32 - 1) / d32);
+                } else {
+                    t0 = n0 <= 0 ? 0 : (n0 + den - 1) / den;
+                    t1 = n1 <= 0 ? 0 : (n1 + den - 1) / den;
+                }
                 tb = (int)(t0 > TT ? TT : t0);
                 te = (int)(t1 > TT ? TT : t1);
             }
             s_pair[2 * v] = tb;
             s_pair[2 * v + 1] = te;
             s_base[v] = base;
-            if (te > tb) str = p.ex[v].tile_stride;
+            if (te > tb) str = p.ps[v].stride;
         }
         // ring geometry: a stage holds two of the largest packed tiles this CTA will see
 #pragma unroll
@@ -376,13 +398,13 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             return false;
         }
         const int v = wk.v;
-        const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
+        const int row0 = s_off[s_ps[v].rexp], rows = s_off[s_ps[v].rexp + 1] - row0;
         const int NT = rows > 8 ? 2 : 1;
         const int kb1 = wk.kb + wk.run();
         const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
         if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
-        const int bits = p.ex[v].bits, K = p.K[v];
-        const float fold = p.ex[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
+        const int bits = s_ps[v].bits, K = s_ps[v].K;
+        const float fold = s_ps[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
         const uint32_t xbuf = sbase + L::x_off + buf * GV_XBUF;
         float* sbuf = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF);
         // one 16-byte fetch (chunk a = 4G + q of the k-block: k = 32G + 8q ..) -> four fp16 pairs in MMA fragment order at
@@ -465,7 +487,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         kbc += nkb;
         if (kbc >= kb1) {
             bool changed;
-            more = wk.next(s_pair, p, changed);
+            more = wk.next(s_pair, s_ps, p.P, changed);
             kbc = more ? wk.kb : 0;
         }
         return true;
@@ -473,7 +495,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
     // the first chunk is staged by the consumer and service warps together: one fetch latency instead of many
     GvWalk swk;
     swk.start();
-    bool s_changed, s_more = swk.next(s_pair, p, s_changed);
+    bool s_changed, s_more = swk.next(s_pair, s_ps, p.P, s_changed);
     int s_kbc = s_more ? swk.kb : 0;
     if (warp < GV_CONS + GV_SERV) {
         stage_chunk(std::integral_constant<int, 4>{}, swk, s_kbc, s_more, 0, (GV_CONS + GV_SERV) * 32, tid);
@@ -489,12 +511,12 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             Ring ring;
             bool changed, ok = true;
             int issued = 0;
-            while (ok && wk.next(s_pair, p, changed)) {
+            while (ok && wk.next(s_pair, s_ps, p.P, changed)) {
                 const int v = wk.v, n = wk.run();
-                const uint32_t stride = (uint32_t)p.ex[v].tile_stride;
-                const bool gated = FUSED && p.tiles2[v] != nullptr;
+                const uint32_t stride = (uint32_t)s_ps[v].stride;
+                const bool gated = FUSED && s_ps[v].gated;
                 const int nt = gated ? wk.nt2 : 2 * wk.nt2;
-                const bool two = gated || nt + 1 < p.NT1[v];
+                const bool two = gated || nt + 1 < s_ps[v].NT1;
                 const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * stride;
                 const uint8_t* b = gated ? p.tiles2[v] + ((size_t)nt * wk.KB + wk.kb) * stride : a + (size_t)wk.KB * stride;
                 for (int i = 0; i < n; ++i) {
@@ -599,11 +621,11 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             const ChunkDesc* d = s_desc + buf;
             if (!d->valid) break;
             const int v = d->v, nt2 = d->nt2, kbc = d->kbc, nkb = d->nkb, kb0 = d->kb0, kb1 = d->kb1;
-            const int row0 = s_off[p.rexp[v]], rows = s_off[p.rexp[v] + 1] - row0;
-            const int bits = p.ex[v].bits, group = p.ex[v].group, has_zeros = p.ex[v].has_zeros;
-            const bool gated = FUSED && p.tiles2[v] != nullptr;
+            const int row0 = s_off[s_ps[v].rexp], rows = s_off[s_ps[v].rexp + 1] - row0;
+            const int bits = s_ps[v].bits, group = s_ps[v].group, has_zeros = s_ps[v].has_zeros;
+            const bool gated = FUSED && s_ps[v].gated;
             const int nt = gated ? nt2 : 2 * nt2 + half;
-            const bool active = nt < p.NT1[v];
+            const bool active = nt < s_ps[v].NT1;
             const int n_r = nt * 128 + blob * 16 + g;
             if (kbc == kb0) {
 #pragma unroll
@@ -638,7 +660,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             if (kbc + nkb == kb1 && active) {
                 // ---- the piece is complete
                 const int NT = rows > 8 ? 2 : 1;
-                const int KB = p.KB[v], N = p.N[v];
+                const int KB = s_ps[v].KB, N = s_ps[v].N;
                 uint16_t* Y = p.Y[v];
                 const uint16_t* R = FUSED ? p.Res[v] : nullptr;
                 auto store_rows = [&]() {
@@ -685,7 +707,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                     // part of a segment: park this warp's sums, announce, and add everything up if this was the last arrival
                     // (for a gated pair the two warps of a blob share one counter and whoever is last finishes both products)
                     const long long C = *s_C, base = s_base[v];
-                    const int G = *s_G, wv = p.w[v];
+                    const int G = *s_G, wv = s_ps[v].w;
                     const int c_a = (int)(((base + (long long)(nt2 * KB) * wv) * G) / C);
                     const int c_b = (int)(((base + (long long)(nt2 * KB + KB - 1) * wv) * G) / C);
                     float* slot = p.partials + (size_t)(2 * blockIdx.x + (kb0 == 0 ? 1 : 0)) * GV_SLOT_FLOATS;
@@ -708,13 +730,23 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                         auto gather = [&](int wsrc, float (&dst)[8]) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) dst[i] = 0.f;
-                            for (int c = c_a; c <= c_b; ++c) {
-                                const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
+                            // four CTAs' sums are fetched together (one round trip), then added in CTA order
+                            for (int c0 = c_a; c0 <= c_b; c0 += 4) {
+                                float part[4][8];
 #pragma unroll
-                                for (int tb = 0; tb < 2; ++tb)
+                                for (int u = 0; u < 4; ++u) {
+                                    const int c = c0 + u;
+                                    const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
 #pragma unroll
-                                    for (int j = 0; j < 4; ++j)
-                                        if (tb < NT) dst[4 * tb + j] += __ldcg(src + ((wsrc * 2 + tb) * 4 + j) * 32 + lane);
+                                    for (int tb = 0; tb < 2; ++tb)
+#pragma unroll
+                                        for (int j = 0; j < 4; ++j)
+                                            part[u][4 * tb + j] = (c <= c_b && tb < NT) ? __ldcg(src + ((wsrc * 2 + tb) * 4 + j) * 32 + lane) : 0.f;
+                                }
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) dst[i] += part[u][i];
                             }
                         };
                         if (FUSED && gated) {
@@ -798,19 +830,22 @@ moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const m
                 return MOQE_ERR_MISMATCH;
     if (!ws || ws_bytes < decode_workspace_bytes(M)) return MOQE_ERR_WORKSPACE;
     GvParams p;
+    long long total_cost = 0;                       // with every expert touched: an upper bound of what the kernel adds up
     for (int l = 0; l < nl; ++l)
         for (int e = 0; e < E; ++e) {
             const int v = l * E + e;
             p.ex[v] = ex[v]->dev();
             p.X[v] = (const uint16_t*)X[l];
             p.Y[v] = (uint16_t*)Y[l];
-            p.N[v] = ex[v]->N;
-            p.K[v] = ex[v]->K;
-            p.KB[v] = ex[v]->Kp / 128;
-            p.NT1[v] = ex[v]->Np / 128;
-            p.rexp[v] = e;
-            p.w[v] = g_dec_cost[ex[v]->bits];
             const moqe_expert* second = ex2 ? ex2[v] : nullptr;
+            PairS& q = p.ps[v];
+            q.bits = p.ex[v].bits; q.group = p.ex[v].group; q.has_zeros = p.ex[v].has_zeros; q.stride = p.ex[v].tile_stride;
+            q.N = ex[v]->N; q.K = ex[v]->K; q.KB = ex[v]->Kp / 128; q.NT1 = ex[v]->Np / 128;
+            q.rexp = e;
+            q.w = g_dec_cost[ex[v]->bits];
+            q.gated = second ? 1 : 0;
+            q.pad = 0;
+            total_cost += (long long)(second ? q.NT1 : (q.NT1 + 1) / 2) * q.KB * q.w;
             p.tiles2[v] = second ? second->tiles : nullptr;
             p.scales_pc2[v] = second ? second->scales_pc : nullptr;
             p.zeros_pc2[v] = second ? second->zeros_pc : nullptr;
@@ -826,6 +861,7 @@ moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const m
     p.status = device_status_word();
     int grid = dec_sm_count();
     if (grid > GV_MAX_GRID) grid = GV_MAX_GRID;
+    p.small = total_cost * (grid + 1) < (1ll << 31) ? 1 : 0;
     const bool fused = ex2 != nullptr || R != nullptr;
     const int smem = fused ? GvSmem<true>::dyn_bytes : GvSmem<false>::dyn_bytes;
     auto kernel = fused ? qgemm_decode_kernel<true> : qgemm_decode_kernel<false>;
