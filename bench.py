@@ -430,6 +430,9 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
             L = Ls[0]
             moqe.moqe_routed_qgemm_sorted(L["X"], perm, offsets, L["experts"], L["Y"], L["ws"], path=args.path, _arr=L["arr"])
 
+    one_launch_routing = (not on_device_router and len({L["spec"].rows_per_sample for L in layers}) == 1
+                          and layers[0]["M"] <= 1024 and w.n_samples <= 1024)
+
     # groups of layers that share one row structure share one sort
     def hot_path(from_host: bool):
         lgd = logits
@@ -440,8 +443,14 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
         else:
             if from_host:
                 lgd.copy_(logits_h, non_blocking=True)
-            ids = moqe.moqe_route(lgd)
-        sorted_for = {}
+            if one_launch_routing:                          # a decode step: arg-max, expansion and sort in one launch
+                L0 = layers[0]
+                _, _, perm, offsets = moqe.moqe_route_permute(lgd, L0["row_off"], L0["M"])
+                sorted_for = {L0["spec"].rows_per_sample: (perm, offsets)}
+            else:
+                ids = moqe.moqe_route(lgd)
+        if not one_launch_routing:
+            sorted_for = {}
         for g in groups:
             Ls = [layers[j] for j in g]
             if from_host:

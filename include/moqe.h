@@ -150,6 +150,14 @@ MOQE_API moqe_status moqe_route(const float* logits, int S, int E, int32_t* ids,
 MOQE_API moqe_status moqe_expand_ids(const int32_t* ids, const int32_t* row_offsets, int S, int M,
                             int32_t* row_ids, void* stream);
 
+/* moqe_route, moqe_expand_ids and the index part of moqe_permute (below) in ONE launch, for small batches (a decode
+ * step): S <= 1024 samples, M <= 1024 rows (else MOQE_ERR_UNSUPPORTED, nothing launched).  logits fp32 [S][E],
+ * row_offsets int32 [S+1] as for moqe_expand_ids, or NULL for one row per sample (then M == S); written: ids int32 [S],
+ * row_ids int32 [M], perm int32 [M], offsets int32 [E+1], with exactly the values the three calls give.  All device
+ * pointers; no workspace; E <= MOQE_MAX_EXPERTS. */
+MOQE_API moqe_status moqe_route_permute(const float* logits, int S, int E, const int32_t* row_offsets, int M, int32_t* ids,
+                                        int32_t* row_ids, int32_t* perm, int32_t* offsets, void* stream);
+
 /* ---------------------------------------------------------------------------
  * Stable counting sort of rows by expert id, and the row gather / scatter.
  * (The batching glue between "one expert per sample" and a grouped GEMM; the

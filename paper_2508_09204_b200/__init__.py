@@ -24,7 +24,7 @@ PATH_AUTO, PATH_STREAM, PATH_TCGEN05, PATH_DECODE, PATH_DENSE = 0, 1, 2, 5, 6
 
 EXPORTED = (
     "moqe_quantize_rtn", "moqe_expert_export", "moqe_expert_import", "moqe_expert_info", "moqe_expert_destroy",
-    "moqe_route", "moqe_expand_ids", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
+    "moqe_route", "moqe_expand_ids", "moqe_route_permute", "moqe_permute_workspace", "moqe_permute", "moqe_permute_static", "moqe_unpermute",
     "moqe_routed_qgemm_workspace", "moqe_routed_qgemm", "moqe_routed_qgemm_path", "moqe_routed_qgemm_sorted",
     "moqe_routed_qgemm_sorted_multi", "moqe_routed_qgemm_workspace_clear", "moqe_async_status",
     "moqe_status_str", "moqe_launch_count", "moqe_tune", "moqe_selftest_timeout",
@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         L.moqe_expert_destroy.argtypes = [vp]
         L.moqe_route.argtypes = [vp, i32, i32, vp, vp]
         L.moqe_expand_ids.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.moqe_route_permute.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp, vp]
         L.moqe_permute_workspace.argtypes = [i32, i32]
         L.moqe_permute_workspace.restype = sz
         L.moqe_permute.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -243,6 +244,23 @@ def moqe_expand_ids(ids: torch.Tensor, row_offsets: torch.Tensor, M: int) -> tor
     _check(lib().moqe_expand_ids(_ptr(ids), _ptr(row_offsets), ids.numel(), int(M), _ptr(row_ids), _stream()),
            "moqe_expand_ids")
     return row_ids
+
+
+def moqe_route_permute(logits: torch.Tensor, row_offsets: Optional[torch.Tensor], M: int):
+    """moqe_route + moqe_expand_ids + moqe_permute (indices only) in one launch, for at most 1024 samples and rows.
+    -> (ids int32 [S], row_ids int32 [M], perm int32 [M], offsets int32 [E+1])."""
+    logits = _dev(logits, torch.float32, "logits")
+    S, E = logits.shape
+    dev = logits.device
+    if row_offsets is not None:
+        row_offsets = _dev(row_offsets, torch.int32, "row_offsets")
+    ids = torch.empty(S, dtype=torch.int32, device=dev)
+    row_ids = torch.empty(int(M), dtype=torch.int32, device=dev)
+    perm = torch.empty(int(M), dtype=torch.int32, device=dev)
+    offsets = torch.empty(E + 1, dtype=torch.int32, device=dev)
+    _check(lib().moqe_route_permute(_ptr(logits), S, E, _ptr(row_offsets) if row_offsets is not None else None, int(M),
+                                    _ptr(ids), _ptr(row_ids), _ptr(perm), _ptr(offsets), _stream()), "moqe_route_permute")
+    return ids, row_ids, perm, offsets
 
 
 def moqe_permute(X: Optional[torch.Tensor], row_ids: torch.Tensor, E: int):

@@ -21,18 +21,22 @@ constexpr int SORT_THREADS = 1024;
 constexpr int SORT_WARPS = SORT_THREADS / 32;
 constexpr int MAXB = MOQE_MAX_EXPERTS + 1;   // buckets incl. the invalid-id bucket
 
-__global__ void route_kernel(const float* __restrict__ logits, int S, int E, int32_t* __restrict__ ids) {
-    int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= S) return;
-    const float* l = logits + (size_t)s * E;
+// first maximum of one row of logits; NaN never wins; a row of NaNs gives 0
+__device__ __forceinline__ int first_argmax(const float* __restrict__ l, int E) {
     int best = -1;
     float bv = 0.f;
     for (int e = 0; e < E; ++e) {
         float v = l[e];
-        if (v != v) continue;                       // NaN never wins
+        if (v != v) continue;
         if (best < 0 || v > bv) { best = e; bv = v; }
     }
-    ids[s] = best < 0 ? 0 : best;
+    return best < 0 ? 0 : best;
+}
+
+__global__ void route_kernel(const float* __restrict__ logits, int S, int E, int32_t* __restrict__ ids) {
+    int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    ids[s] = first_argmax(logits + (size_t)s * E, E);
 }
 
 __global__ void expand_ids_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ row_offsets, int S, int M,
@@ -112,6 +116,66 @@ __global__ void __launch_bounds__(SORT_THREADS) sort_small_kernel(const int32_t*
         perm[s_off[br.bucket] + br.rank] = threadIdx.x;
         if (br.bucket == E && Y) zero_row(Y, N, threadIdx.x);
     }
+}
+
+// Route, expand and sort in one block for a batch of at most 1024 rows and 1024 samples: thread s < S takes the arg-max
+// of sample s, thread m < M looks up its sample and sorts as sort_small_kernel does.  Dependents may be scheduled at
+// once (they wait for this grid's results themselves).
+__global__ void __launch_bounds__(SORT_THREADS) route_sort_small_kernel(const float* __restrict__ logits, int S, int E,
+                                                                        const int32_t* __restrict__ row_offsets, int M,
+                                                                        int32_t* __restrict__ ids, int32_t* __restrict__ row_ids,
+                                                                        int32_t* __restrict__ perm, int32_t* __restrict__ offsets) {
+    __shared__ int s_warp[SORT_WARPS][MAXB];
+    __shared__ int s_tot[MAXB];
+    __shared__ int s_off[MAXB + 1];
+    __shared__ int s_ids[SORT_THREADS];
+    __shared__ int s_rows[SORT_THREADS];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int t = threadIdx.x;
+    if (t < S) {
+        const int id = first_argmax(logits + (size_t)t * E, E);
+        s_ids[t] = id;
+        ids[t] = id;
+    }
+    if (t < S) s_rows[t] = row_offsets ? row_offsets[t] : t;
+    __syncthreads();
+    const int lane = t & 31, warp = t >> 5;
+    const bool live = t < M;
+    int bucket = 0;
+    if (live) {
+        int lo = 0, hi = S;                          // largest s with row_offsets[s] <= m
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (s_rows[mid] <= t) lo = mid; else hi = mid;
+        }
+        bucket = s_ids[lo];                          // valid by construction
+        row_ids[t] = bucket;
+    }
+    for (int i = t; i < SORT_WARPS * MAXB; i += blockDim.x) (&s_warp[0][0])[i] = 0;
+    __syncthreads();
+    const unsigned live_mask = __ballot_sync(0xffffffffu, live);
+    int rank_in_warp = 0;
+    if (live) {
+        const unsigned peers = __match_any_sync(live_mask, bucket);
+        rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+        if (rank_in_warp == 0) s_warp[warp][bucket] = __popc(peers);
+    }
+    __syncthreads();
+    if (t <= E) {
+        int run = 0;
+        for (int w = 0; w < SORT_WARPS; ++w) { int c = s_warp[w][t]; s_warp[w][t] = run; run += c; }
+        s_tot[t] = run;
+    }
+    __syncthreads();
+    if (t == 0) {
+        int run = 0;
+        for (int b = 0; b <= E; ++b) { s_off[b] = run; run += s_tot[b]; }
+        s_off[E + 1] = run;
+    }
+    __syncthreads();
+    if (t <= E) offsets[t] = s_off[t];
+    if (live) perm[s_off[bucket] + rank_in_warp + s_warp[warp][bucket]] = t;
 }
 
 // M > 1024: three kernels.  (1) per-block bucket totals
@@ -341,6 +405,26 @@ extern "C" moqe_status moqe_expand_ids(const int32_t* ids, const int32_t* row_of
     if (S < 0 || M < 0 || (S == 0 && M != 0)) return MOQE_ERR_SHAPE;
     if (M == 0) return MOQE_OK;
     expand_ids_kernel<<<(M + 255) / 256, 256, 0, (cudaStream_t)stream>>>(ids, row_offsets, S, M, row_ids);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+extern "C" moqe_status moqe_route_permute(const float* logits, int S, int E, const int32_t* row_offsets, int M, int32_t* ids,
+                                          int32_t* row_ids, int32_t* perm, int32_t* offsets, void* stream) {
+    if (!offsets) return MOQE_ERR_NULL;
+    if (S < 0 || M < 0 || E <= 0 || (S == 0 && M != 0)) return MOQE_ERR_SHAPE;
+    if (!row_offsets && M != S) return MOQE_ERR_SHAPE;
+    if (E > MOQE_MAX_EXPERTS || S > SORT_THREADS || M > SORT_THREADS) return MOQE_ERR_UNSUPPORTED;
+    if (S > 0 && (!logits || !ids)) return MOQE_ERR_NULL;
+    if (M > 0 && (!row_ids || !perm)) return MOQE_ERR_NULL;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1); cfg.blockDim = dim3(SORT_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, route_sort_small_kernel, logits, S, E, row_offsets, M, ids, row_ids, perm, offsets) != cudaSuccess)
+        return MOQE_ERR_CUDA;
     count_launch();
     return cuda_ok(cudaGetLastError());
 }

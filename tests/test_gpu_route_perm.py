@@ -59,6 +59,38 @@ def test_sort_matches_oracle(M, E):
     assert moqe.moqe_async_status() == moqe.OK
 
 
+@pytest.mark.parametrize("S,E,rows", [(1, 1, None), (16, 3, None), (16, 3, "ragged"), (1024, 5, None), (100, 32, "ragged"),
+                                      (7, 4, "empty-samples")])
+def test_route_permute_in_one_launch_matches_the_three_oracle_steps(S, E, rows):
+    import paper_2508_09204_b200 as moqe
+    from gpu_helpers import dev
+    g = np.random.default_rng(S * 31 + E)
+    logits = g.standard_normal((S, E)).astype(np.float32)
+    logits[g.random((S, E)) < 0.05] = np.float32("nan")
+    logits[::5] = np.round(logits[::5])                          # ties
+    if E >= 3:
+        logits[:, 1] = -100.0                                    # an expert with no rows
+    if rows is None:
+        off, M = None, S
+    else:
+        n = g.integers(0 if rows == "empty-samples" else 1, 1024 // S + 1, size=S)
+        off = np.concatenate([[0], np.cumsum(n)]).astype(np.int32)
+        M = int(off[-1])
+    ids, row_ids, perm, offsets = moqe.moqe_route_permute(torch.from_numpy(logits).to(dev()),
+                                                          None if off is None else torch.from_numpy(off).to(dev()), M)
+    ids_ref = oracle.route(logits)
+    rid_ref = ids_ref if off is None else oracle.expand_ids(ids_ref, off)
+    _, off_ref, perm_ref, _ = oracle.permutation(rid_ref, E)
+    assert np.array_equal(ids.cpu().numpy(), ids_ref)
+    assert np.array_equal(row_ids.cpu().numpy(), rid_ref)
+    assert np.array_equal(offsets.cpu().numpy(), off_ref)
+    assert np.array_equal(perm.cpu().numpy(), perm_ref)
+    # beyond the single-block limit nothing is launched
+    big = torch.zeros((1025, 2), dtype=torch.float32, device=dev())
+    with pytest.raises(moqe.MoqeError):
+        moqe.moqe_route_permute(big, None, 1025)
+
+
 @pytest.mark.parametrize("M,C,E", [(64, 1024, 2), (333, 40, 4), (4160, 3584, 4), (5000, 8, 3)])
 def test_permute_unpermute_rows(M, C, E):
     import paper_2508_09204_b200 as moqe
