@@ -254,6 +254,7 @@ def main():
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to moqe_tune (measurement knob)")
     ap.add_argument("--repeats", type=int, default=5, help="timings of --steps steps each; the median is reported")
     ap.add_argument("--no-workloads", action="store_true", help="skip the sub-records of the other workloads")
+    ap.add_argument("--force-expert", type=int, default=None, help="route every sample to this expert (per-format timing)")
     ap.add_argument("--fused-block", action="store_true",
                     help="decode workloads: gate/up as ONE gated launch (silu(gate) * up), residual add in the o / down stores")
     args = ap.parse_args()
@@ -298,7 +299,7 @@ def main():
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
-    line = bench_workload(ctx, w, steps=args.steps, warmup=args.warmup, repeats=args.repeats, with_e2e=True)
+    line = bench_workload(ctx, w, steps=args.steps, warmup=args.warmup, repeats=args.repeats, with_e2e=True, force_expert=args.force_expert)
     line["clocks"] = sampler.stop()
 
     # ---- the other workloads of the metric, as sub-records (resident inputs, fewer steps) -------

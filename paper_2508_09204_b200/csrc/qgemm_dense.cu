@@ -6,9 +6,11 @@
 //
 //   tile      : 128 token rows of one expert x up to 256 output channels (one TMEM accumulator of up to 256 columns,
 //               two of them so that the epilogue of a tile overlaps the MMAs of the next)
-//   operands  : both by TMA (2-D tiled, 128-byte swizzle, no multicast), 64 k per stage: the token rows (boxes of 64
-//               rows, read in place from X where the sorted rows are consecutive there -- always, for per-image
-//               routing of whole 64-row runs -- else from the gathered copy), and the channel rows of the dense weights
+//   operands  : 64 k per stage.  The channel rows of the dense weights by TMA (2-D tiled, 128-byte swizzle, no
+//               multicast); the token rows in boxes of 64 rows: by TMA straight from X where the box's sorted rows are
+//               consecutive there (always, for per-image routing of whole 64-row runs), else gathered row by row
+//               through `perm` by the producer warp's 16-byte cp.async copies into the same swizzled layout -- the
+//               fused permutation, no gathered copy of X exists
 //   epilogue  : one thread per token row reads its accumulator row from TMEM, multiplies by the per-channel scale,
 //               rounds to bf16 and writes up to 512 contiguous bytes of Y at the row's ORIGINAL position (fused
 //               un-permutation).  X is read once per channel chunk and Y written once.
@@ -32,7 +34,9 @@
 namespace moqe {
 namespace {
 
-constexpr int DN_THREADS = 320;                 // warp 0: TMA producer, warp 1: MMA issuer, warps 2..9: epilogue
+constexpr int DN_THREADS = 416;                 // warp 0: producer (TMA + gather), warp 1: MMA issuer, warps 2..9: epilogue,
+                                                // warps 10..12: gather helpers
+constexpr int DN_GATHER_WARPS = 4;              // warp 0 and the helpers
 constexpr int DN_EPI_THREADS = 256;
 constexpr int DN_MAX_STAGES = 8;
 constexpr int DN_XSTAGE = 128 * 128;            // 128 token rows x 64 k bf16
@@ -55,11 +59,11 @@ struct DnSmem {
 struct DnParams {
     const int32_t* perm;
     const int32_t* offsets;
-    const int32_t* box_src;     // per 64-row box of the sorted rows: first source row in X if consecutive there, else -1
+    const uint16_t* X;          // token rows [M][K] bf16, unsorted
     const float* col_scale;     // [E][Np]
     uint16_t* Y;
     int* status;
-    int M, N, Np, Kp, E, Ksteps;   // Ksteps: 64-k stages that hold real k (columns beyond K read as zeros)
+    int M, N, K, Np, Kp, E, Ksteps;   // Ksteps: 64-k stages that hold real k (columns beyond K read as zeros)
     int Nw;                        // channel rows that take part: N rounded up to whole 64-row boxes
     unsigned split_mask;           // bit e: expert e is stored as hi + lo halves (grouped formats)
     int resident, max_steps;       // the experts' dense weights fit shared memory; 64-k steps of the largest one
@@ -92,7 +96,6 @@ __device__ __forceinline__ bool dn_tile(const int* s_off, int E, int t, DnTile& 
 }
 
 __global__ void __launch_bounds__(DN_THREADS, 1) qgemm_dense_kernel(const __grid_constant__ DnParams p,
-                                                                    const __grid_constant__ CUtensorMap tmap_xp,
                                                                     const __grid_constant__ CUtensorMap tmap_x,
                                                                     const __grid_constant__ CUtensorMap tmap_w) {
     extern __shared__ unsigned char smem_raw[];
@@ -119,7 +122,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) qgemm_dense_kernel(const __grid
     float* s_cs = reinterpret_cast<float*>(smem + L::cs_off);
 
     if (tid == 0) {
-        for (int i = 0; i < DN_MAX_STAGES; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+        for (int i = 0; i < DN_MAX_STAGES; ++i) { mbar_init(bar_full + 8 * i, 1 + 32 * DN_GATHER_WARPS); mbar_init(bar_empty + 8 * i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar_accfull + 8 * i, 1); mbar_init(bar_accempty + 8 * i, DN_EPI_THREADS); }
         mbar_init(bar_wres_full, 1);
         mbar_init(bar_wres_empty, 1);
@@ -134,68 +137,109 @@ __global__ void __launch_bounds__(DN_THREADS, 1) qgemm_dense_kernel(const __grid
     const uint32_t tmem_base = *s_tmem;
     const int nchunks = (p.Nw + DN_NC - 1) / DN_NC, kstages = p.Ksteps;
 
-    if (warp == 0) {
-        // ---------------- producer: token boxes and weight boxes, 64 k per stage ----------------
-        if (lane == 0) {
-            Ring ring;
-            DnTile ti;
-            bool ok = true;
-            int w_e = -1;
-            uint32_t w_uses = 0;
-            // (the sources of a tile's two boxes are fetched one tile ahead: a global round trip per tile would
-            // otherwise sit in front of every tile's copies)
-            DnTile nx;
-            int nsrc[2] = {-1, -1};
-            bool have = dn_tile(s_off, p.E, blockIdx.x, nx);
-            if (have) {
-                nsrc[0] = p.box_src[nx.box0];
-                nsrc[1] = nx.rows > 64 ? p.box_src[nx.box0 + 1] : -1;
+    if (warp == 0 || warp >= 10) {
+        // ---------------- producers: token boxes and weight boxes, 64 k per stage ----------------
+        // Four warps walk the tiles in step.  Lane 0 of warp 0 issues the TMA copies: the weight boxes, and every 64-row
+        // token box whose sorted rows are consecutive in X (always, for per-image routing of whole 64-row runs) straight
+        // from X.  A box whose rows are scattered in X is gathered by the 128 lanes with 16-byte cp.async copies, row by
+        // row through `perm`, into the same 128-byte-swizzled layout (warp g takes box rows 16g .. 16g + 15); a
+        // stage's full barrier takes one arrival per lane (tied to the lane's copies where it made some) on top of
+        // the transaction count.
+        const int g = warp == 0 ? 0 : warp - 9;
+        const bool tma_lane = warp == 0 && lane == 0;
+        Ring ring;
+        DnTile ti;
+        bool ok = true;
+        int w_e = -1;
+        uint32_t w_uses = 0;
+        // this lane's entries of `perm` for the tile's rows lane, lane + 32, lane + 64, lane + 96 (-1 beyond the tile),
+        // fetched one tile ahead: a global round trip per tile would otherwise sit in front of every tile's copies
+        auto fetch_rows = [&](const DnTile& t, int (&o)[4]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) o[q] = q * 32 + lane < t.rows ? p.perm[t.m0 + q * 32 + lane] : -1;
+        };
+        DnTile nx;
+        int npv[4] = {-1, -1, -1, -1};
+        bool have = dn_tile(s_off, p.E, blockIdx.x, nx);
+        if (have) fetch_rows(nx, npv);
+        const uint16_t* Xg = p.X;
+        for (int t = blockIdx.x; ok && have; t += gridDim.x) {
+            ti = nx;
+            const int pv[4] = {npv[0], npv[1], npv[2], npv[3]};
+            have = dn_tile(s_off, p.E, t + gridDim.x, nx);
+            if (have) fetch_rows(nx, npv);
+            const int nbox = (ti.rows + 63) / 64;
+            int src_row[2];                 // first row in X of a box whose rows are consecutive there, else -1
+            int xr[2][4];                   // the X row of box row 16g + 4i + lane / 8 (-1: none, zero fill)
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const int cnt = min(64, ti.rows - 64 * b);
+                const int first = __shfl_sync(0xffffffffu, pv[2 * b], 0);
+                const bool mine = (lane >= cnt || pv[2 * b] == first + lane) && (lane + 32 >= cnt || pv[2 * b + 1] == first + lane + 32);
+                src_row[b] = (b < nbox && __all_sync(0xffffffffu, mine)) ? first : -1;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    xr[b][i] = __shfl_sync(0xffffffffu, g < 2 ? pv[2 * b] : pv[2 * b + 1], (16 * g + 4 * i + (lane >> 3)) & 31);
             }
-            for (int t = blockIdx.x; ok && have; t += gridDim.x) {
-                ti = nx;
-                const int nbox = (ti.rows + 63) / 64;
-                const int src_row[2] = {nsrc[0], nsrc[1]};
-                have = dn_tile(s_off, p.E, t + gridDim.x, nx);
-                if (have) {
-                    nsrc[0] = p.box_src[nx.box0];
-                    nsrc[1] = nx.rows > 64 ? p.box_src[nx.box0 + 1] : -1;
-                }
-                const int steps = ((p.split_mask >> ti.e) & 1u) ? 2 * kstages : kstages;
-                if (p.resident && ti.e != w_e) {
-                    // a new expert: its dense weights replace the resident ones once the MMAs that read those are done
-                    if (w_uses > 0 && !(ok = mbar_wait(bar_wres_empty, (w_uses - 1) & 1u, s_abort, p.status))) break;
+            const bool gather0 = nbox > 0 && src_row[0] < 0, gather1 = nbox > 1 && src_row[1] < 0;
+            const int n_tma = (nbox > 0 && !gather0 ? 1 : 0) + (nbox > 1 && !gather1 ? 1 : 0);
+            const int steps = ((p.split_mask >> ti.e) & 1u) ? 2 * kstages : kstages;
+            if (warp == 0 && p.resident && ti.e != w_e) {
+                // a new expert: its dense weights replace the resident ones once the MMAs that read those are done
+                if (w_uses > 0 && !(ok = __all_sync(0xffffffffu, mbar_wait(bar_wres_empty, (w_uses - 1) & 1u, s_abort, p.status)))) break;
+                if (lane == 0) {
                     mbar_expect_tx(bar_wres_full, (uint32_t)(steps * (p.Nw / 64)) * 8192u);
                     for (int ks = 0; ks < steps; ++ks) {
                         const int wcol = ks < kstages ? ks * 64 : p.Kp + (ks - kstages) * 64;
                         for (int b = 0; b < p.Nw / 64; ++b)
                             tma_load_2d(wres_base + (ks * (p.Nw / 64) + b) * 8192, &tmap_w, wcol, ti.e * p.Np + b * 64, bar_wres_full);
                     }
-                    w_e = ti.e;
-                    ++w_uses;
                 }
-                for (int nc = 0; ok && nc < nchunks; ++nc) {
-                    const int wrows = min(DN_NC, p.Nw - nc * DN_NC);
-                    for (int ks = 0; ks < steps; ++ks) {
-                        if (!(ok = mbar_wait(bar_empty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status))) break;
-                        const uint32_t full = bar_full + 8 * ring.stage;
-                        mbar_expect_tx(full, (uint32_t)(nbox + (p.resident ? 0 : wrows / 64)) * 8192u);
-                        const uint32_t xd = ring_base + ring.stage * stage_bytes;
-                        const int xcol = (ks < kstages ? ks : ks - kstages) * 64;             // the second half re-reads the tokens
-                        for (int b = 0; b < nbox; ++b) {
-                            if (src_row[b] >= 0) tma_load_2d(xd + b * 8192, &tmap_x, xcol, src_row[b], full);
-                            else tma_load_2d(xd + b * 8192, &tmap_xp, xcol, ti.m0 + b * 64, full);
-                        }
+                w_e = ti.e;
+                ++w_uses;
+            }
+            for (int nc = 0; ok && nc < nchunks; ++nc) {
+                const int wrows = min(DN_NC, p.Nw - nc * DN_NC);
+                for (int ks = 0; ks < steps; ++ks) {
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * ring.stage, ring.phase ^ 1u, s_abort, p.status)))) break;
+                    const uint32_t full = bar_full + 8 * ring.stage;
+                    const uint32_t xd = ring_base + ring.stage * stage_bytes;
+                    const int xcol = (ks < kstages ? ks : ks - kstages) * 64;             // the second half re-reads the tokens
+                    if (tma_lane) {
+                        mbar_expect_tx(full, (uint32_t)(n_tma + (p.resident ? 0 : wrows / 64)) * 8192u);
+                        if (nbox > 0 && !gather0) tma_load_2d(xd, &tmap_x, xcol, src_row[0], full);
+                        if (nbox > 1 && !gather1) tma_load_2d(xd + 8192, &tmap_x, xcol, src_row[1], full);
                         if (!p.resident) {
                             const int wcol = ks < kstages ? ks * 64 : p.Kp + (ks - kstages) * 64;
                             const uint32_t wd = xd + DN_XSTAGE;
                             for (int b = 0; b < wrows / 64; ++b)
                                 tma_load_2d(wd + b * 8192, &tmap_w, wcol, ti.e * p.Np + nc * DN_NC + b * 64, full);
                         }
-                        ring.advance(nstg);
                     }
+                    if (gather0 || gather1) {
+                        const int chunk = lane & 7, kk = xcol + chunk * 8;
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            if (b == 0 ? gather0 : gather1) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int r = 16 * g + 4 * i + (lane >> 3);
+                                    const bool real = xr[b][i] >= 0 && kk < p.K;
+                                    const uint16_t* src = real ? Xg + (size_t)xr[b][i] * p.K + kk : Xg;
+                                    const uint32_t dst = xd + b * 8192 + r * 128 + ((chunk ^ (r & 7)) << 4);
+                                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(real ? 16 : 0) : "memory");
+                                }
+                            }
+                        }
+                        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
+                    } else {
+                        mbar_arrive(full);
+                    }
+                    ring.advance(nstg);
                 }
             }
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");
     } else if (warp == 1) {
         // ---------------- MMA issuer: the whole warp walks the tiles, one elected lane issues ----------------
         Ring ring;
@@ -224,6 +268,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) qgemm_dense_kernel(const __grid
                 const int steps = ((p.split_mask >> ti.e) & 1u) ? 2 * kstages : kstages;
                 for (int ks = 0; ks < steps; ++ks) {
                     if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
+                    fence_proxy_async();                 // gathered token rows were written by plain (generic-proxy) copies
                     tc_fence_after();
                     const uint32_t stage = ring_base + ring.stage * stage_bytes;
                     const uint64_t adesc = umma_desc_sw128(stage);
@@ -362,7 +407,8 @@ bool dense_supported(int M, int N, int K, const moqe_expert* const* ex, int E) {
 }
 
 size_t dense_workspace_bytes(int M, int K, int E, int Np, int Kp) {
-    return al256((size_t)M * K * 2) + gather_boxes_bytes(M, E) + al256((size_t)E * Np * Kp * 4) + al256((size_t)E * Np * 4);
+    (void)M; (void)K;
+    return al256((size_t)E * Np * Kp * 4) + al256((size_t)E * Np * 4);
 }
 
 moqe_status launch_qgemm_dense(const void* X, int M, int N, int K, const moqe_expert* const* ex, int E, void* Y,
@@ -374,21 +420,17 @@ moqe_status launch_qgemm_dense(const void* X, int M, int N, int K, const moqe_ex
     EncodeTiledFn enc = dn_encode_fn();
     if (!enc) return MOQE_ERR_CUDA;
     char* base = (char*)ws;
-    void* Xp = base;
-    int32_t* box_src = (int32_t*)(base + al256((size_t)M * K * 2));
-    uint16_t* Wd = (uint16_t*)((char*)box_src + gather_boxes_bytes(M, E));
-    float* cs = (float*)((char*)Wd + al256((size_t)E * Np * Kp * 4));
-    moqe_status s = launch_gather_boxes(X, perm, offsets, M, K, E, Xp, box_src, st);
+    uint16_t* Wd = (uint16_t*)base;
+    float* cs = (float*)(base + al256((size_t)E * Np * Kp * 4));
+    moqe_status s = launch_dense_unpack(ex, E, Wd, cs, st);
     if (s != MOQE_OK) return s;
-    s = launch_dense_unpack(ex, E, Wd, cs, st);
-    if (s != MOQE_OK) return s;
-    CUtensorMap tmap_xp, tmap_x, tmap_w;
-    if (!dn_map(enc, &tmap_xp, Xp, M, K) || !dn_map(enc, &tmap_x, X, M, K) || !dn_map(enc, &tmap_w, Wd, (size_t)E * Np, 2 * (size_t)Kp))
+    CUtensorMap tmap_x, tmap_w;
+    if (!dn_map(enc, &tmap_x, X, M, K) || !dn_map(enc, &tmap_w, Wd, (size_t)E * Np, 2 * (size_t)Kp))
         return MOQE_ERR_CUDA;
     DnParams p;
-    p.perm = perm; p.offsets = offsets; p.box_src = box_src; p.col_scale = cs; p.Y = (uint16_t*)Y;
+    p.perm = perm; p.offsets = offsets; p.X = (const uint16_t*)X; p.col_scale = cs; p.Y = (uint16_t*)Y;
     p.status = device_status_word();
-    p.M = M; p.N = N; p.Np = Np; p.Kp = Kp; p.E = E; p.Ksteps = (K + 63) / 64;
+    p.M = M; p.N = N; p.K = K; p.Np = Np; p.Kp = Kp; p.E = E; p.Ksteps = (K + 63) / 64;
     p.Nw = (N + 63) / 64 * 64;
     p.split_mask = 0;
     for (int e = 0; e < E; ++e)
@@ -402,7 +444,7 @@ moqe_status launch_qgemm_dense(const void* X, int M, int N, int K, const moqe_ex
     const int grid = (int)(tiles < sms ? tiles : sms);
     if (cudaFuncSetAttribute(qgemm_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DnSmem::dyn_bytes) != cudaSuccess)
         return MOQE_ERR_CUDA;
-    qgemm_dense_kernel<<<grid, DN_THREADS, DnSmem::dyn_bytes, st>>>(p, tmap_xp, tmap_x, tmap_w);
+    qgemm_dense_kernel<<<grid, DN_THREADS, DnSmem::dyn_bytes, st>>>(p, tmap_x, tmap_w);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }

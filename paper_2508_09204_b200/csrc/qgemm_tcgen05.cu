@@ -246,6 +246,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
             }
         } else if (warp == 1) {
             // ---------------- MMA issuer ----------------
+            // (Its waits spin on the plain try_wait: they sit on the critical path and coming round a short spin is
+            // faster than waking from the hinted sleep.)
             // The WHOLE warp walks the tiles, so that control flow stays warp-uniform, and one elected lane issues
             // straight-line MMAs whose operands were all computed beforehand.  Measured on B200: issued this way a
             // 128x256x16 MMA costs its 128 tensor-pipe cycles (and a 16-column one 24); issued from a loop that
@@ -262,15 +264,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                 const int group_k = ex.group == 0 ? p.KB * 128 : min(ex.group, 128);
                 int kcount = 0;
                 for (int ks = 0; ok && ks < 2 * p.KB; ++ks) {
-                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_xfull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
-                    if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_afull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait_short(bar_xfull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait_short(bar_afull + 8 * ring.stage, ring.phase, s_abort, p.status)))) break;
                     const uint64_t adesc = umma_desc_sw128(sbase + L::a_off + ring.stage * A_STAGE_BYTES);
                     const uint64_t bdesc = umma_desc_sw128(sbase + L::x_off + ring.stage * (TN * 128));
                     const uint32_t empty_bar = bar_empty + 8 * ring.stage;
                     if (group_k >= 64) {
                         // the stage's four MMAs feed one accumulator buffer
                         if (kcount == 0 &&
-                            !(ok = __all_sync(0xffffffffu, mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
+                            !(ok = __all_sync(0xffffffffu, mbar_wait_short(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
                         tc_fence_after();
                         const uint32_t d = tmem_base + buf * TN;
                         const bool group_ends = kcount + 64 == group_k;
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                         tc_fence_after();
                         for (int j = 0; ok && j < 4; ++j) {
                             if (kcount == 0) {
-                                if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
+                                if (!(ok = __all_sync(0xffffffffu, mbar_wait_short(bar_accempty + 8 * buf, (acc_use[buf] & 1u) ^ 1u, s_abort, p.status)))) break;
                                 tc_fence_after();
                             }
                             const bool group_ends = kcount + 16 == group_k;

@@ -260,9 +260,11 @@ def test_dense_weights_kernel(M, N, K):
     gpu, What, _ = build_experts(W, specs)
     E = len(specs)
     rs = np.random.default_rng(M + N)
-    for routing in ("runs", "scattered"):
+    for routing in ("runs", "images", "scattered"):
         if routing == "runs":                                    # whole runs of 64 rows share an expert (read in place)
             ids = np.repeat(rs.integers(0, E, size=(M + 63) // 64), 64)[:M].astype(np.int32)
+        elif routing == "images":                                # runs of 196 rows: boxes read in place next to gathered ones
+            ids = np.repeat(rs.integers(0, E, size=(M + 195) // 196), 196)[:M].astype(np.int32)
         else:
             ids = rs.integers(0, E, size=M).astype(np.int32)
         ids[ids == 1] = 0                                        # expert 1 idle
