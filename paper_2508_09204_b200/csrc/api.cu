@@ -90,76 +90,74 @@ extern "C" size_t moqe_routed_qgemm_workspace(int M, int N, int K, int E) {
     return ws_layout(M, Np, K, E).total;
 }
 
-extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
-                                              const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
-                                              size_t workspace_bytes, void* stream, int path) {
-    if (!h_experts) return MOQE_ERR_NULL;
+namespace {
+// Argument checks shared by the single-layer entry points (`ids_or_perm`: row ids, or the sort's perm).  *done: the
+// call is complete (an empty batch) when MOQE_OK comes back with it set.
+moqe_status single_layer_args(const void* X, const void* ids_or_perm, const void* offsets_or_self, int M,
+                              const moqe_expert* const* ex, int E, const void* Y, void* workspace, size_t workspace_bytes,
+                              int path, WsLayout& w, int& kernel, bool& done) {
+    done = false;
+    if (!ex) return MOQE_ERR_NULL;
     if (E <= 0 || M < 0) return MOQE_ERR_SHAPE;
     if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
     for (int e = 0; e < E; ++e)
-        if (!h_experts[e]) return MOQE_ERR_NULL;
-    const int N = h_experts[0]->N, K = h_experts[0]->K;
+        if (!ex[e]) return MOQE_ERR_NULL;
+    const int N = ex[0]->N, K = ex[0]->K;
     for (int e = 1; e < E; ++e)
-        if (h_experts[e]->N != N || h_experts[e]->K != K) return MOQE_ERR_MISMATCH;
-    if (M == 0) return MOQE_OK;
-    if (!X_bf16 || !row_ids || !Y_bf16) return MOQE_ERR_NULL;
-    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
+        if (ex[e]->N != N || ex[e]->K != K) return MOQE_ERR_MISMATCH;
+    if (M == 0) { done = true; return MOQE_OK; }
+    if (!X || !ids_or_perm || !offsets_or_self || !Y) return MOQE_ERR_NULL;
+    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X % 16 || (uintptr_t)Y % 16) return MOQE_ERR_UNSUPPORTED;
     if (path < 0 || path > LAST_PATH) return MOQE_ERR_SHAPE;
-    const int Np = h_experts[0]->Np;
-    WsLayout w = ws_layout(M, Np, K, E);
+    w = ws_layout(M, ex[0]->Np, K, E);
     if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
+    kernel = pick_kernel(path, M, ex, E);
+    if (kernel == 2 && !decode_supported_multi(M, ex, 1, E)) return MOQE_ERR_UNSUPPORTED;
+    return MOQE_OK;
+}
+
+// the grouped product on sorted rows with the kernel `pick_kernel` chose
+moqe_status run_sorted(int kernel, int path, const void* X, int M, const moqe_expert* const* ex, int E, void* Y,
+                       const int32_t* perm, const int32_t* offsets, void* body, size_t body_bytes, cudaStream_t st) {
+    const int N = ex[0]->N, K = ex[0]->K;
+    if (kernel == 2) return launch_qgemm_decode_multi(&X, M, 1, ex, E, &Y, perm, offsets, body, body_bytes, st);
+    if (kernel == 1) return launch_qgemm_stream(X, M, N, K, ex, E, Y, perm, offsets, body, body_bytes, st);
+    if (kernel == 3) return launch_qgemm_dense(X, M, N, K, ex, E, Y, perm, offsets, body, body_bytes, st);
+    tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
+    return launch_qgemm_tc(X, M, N, K, ex, E, Y, perm, offsets, body, body_bytes, st);
+}
+}  // namespace
+
+extern "C" moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* row_ids, int M,
+                                              const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
+                                              size_t workspace_bytes, void* stream, int path) {
+    WsLayout w;
+    int kernel = 0;
+    bool done = false;
+    moqe_status s = single_layer_args(X_bf16, row_ids, row_ids, M, h_experts, E, Y_bf16, workspace, workspace_bytes, path, w, kernel, done);
+    if (s != MOQE_OK || done) return s;
     cudaStream_t st = (cudaStream_t)stream;
     char* base = (char*)workspace;
     int32_t* perm = (int32_t*)(base + w.perm);
     int32_t* offsets = (int32_t*)(base + w.offsets);
-    const int kernel = pick_kernel(path, M, h_experts, E);
-    if (kernel == 2 && !decode_supported_multi(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
-    size_t zero_bytes = kernel != 0 ? body_zero_bytes(M, Np) : 0;
-    moqe_status s = launch_sort(row_ids, M, E, perm, offsets, base + w.sort, w.body - w.sort, base + w.body, zero_bytes,
-                                Y_bf16, N, st);
+    const size_t zero_bytes = kernel != 0 ? body_zero_bytes(M, h_experts[0]->Np) : 0;
+    s = launch_sort(row_ids, M, E, perm, offsets, base + w.sort, w.body - w.sort, base + w.body, zero_bytes, Y_bf16,
+                    h_experts[0]->N, st);
     if (s != MOQE_OK) return s;
-    if (kernel == 2)
-        return launch_qgemm_decode_multi(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
-    if (kernel == 1)
-        return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
-                                   w.total - w.body, st);
-    if (kernel == 3)
-        return launch_qgemm_dense(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
-    tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
-    return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+    return run_sorted(kernel, path, X_bf16, M, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
 }
 
 extern "C" moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
                                                 const moqe_expert* const* h_experts, int E, void* Y_bf16, void* workspace,
                                                 size_t workspace_bytes, void* stream, int path) {
-    if (!h_experts) return MOQE_ERR_NULL;
-    if (E <= 0 || M < 0) return MOQE_ERR_SHAPE;
-    if (E > MOQE_MAX_EXPERTS) return MOQE_ERR_UNSUPPORTED;
-    for (int e = 0; e < E; ++e)
-        if (!h_experts[e]) return MOQE_ERR_NULL;
-    const int N = h_experts[0]->N, K = h_experts[0]->K;
-    for (int e = 1; e < E; ++e)
-        if (h_experts[e]->N != N || h_experts[e]->K != K) return MOQE_ERR_MISMATCH;
-    if (M == 0) return MOQE_OK;
-    if (!X_bf16 || !perm || !offsets || !Y_bf16) return MOQE_ERR_NULL;
-    if (N % 8 != 0 || K % 8 != 0 || (uintptr_t)X_bf16 % 16 || (uintptr_t)Y_bf16 % 16) return MOQE_ERR_UNSUPPORTED;
-    if (path < 0 || path > LAST_PATH) return MOQE_ERR_SHAPE;
-    const int Np = h_experts[0]->Np;
-    WsLayout w = ws_layout(M, Np, K, E);
-    if (!workspace || workspace_bytes < w.total || (uintptr_t)workspace % 256) return MOQE_ERR_WORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
+    WsLayout w;
+    int kernel = 0;
+    bool done = false;
+    moqe_status s = single_layer_args(X_bf16, perm, offsets, M, h_experts, E, Y_bf16, workspace, workspace_bytes, path, w, kernel, done);
+    if (s != MOQE_OK || done) return s;
     char* base = (char*)workspace;
-    const int kernel = pick_kernel(path, M, h_experts, E);
-    if (kernel == 2 && !decode_supported_multi(M, h_experts, 1, E)) return MOQE_ERR_UNSUPPORTED;
-    if (kernel == 2)
-        return launch_qgemm_decode_multi(&X_bf16, M, 1, h_experts, E, &Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
-    if (kernel == 1)
-        return launch_qgemm_stream(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body,
-                                   w.total - w.body, st);
-    if (kernel == 3)
-        return launch_qgemm_dense(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
-    tc_set_tile_tokens(path == 3 ? 128 : (path == 4 ? 256 : 0));
-    return launch_qgemm_tc(X_bf16, M, N, K, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body, st);
+    return run_sorted(kernel, path, X_bf16, M, h_experts, E, Y_bf16, perm, offsets, base + w.body, w.total - w.body,
+                      (cudaStream_t)stream);
 }
 
 extern "C" moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16, const int32_t* perm, const int32_t* offsets,
