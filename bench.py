@@ -434,16 +434,33 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
     one_launch_routing = (not on_device_router and len({L["spec"].rows_per_sample for L in layers}) == 1
                           and layers[0]["M"] <= 1024 and w.n_samples <= 1024)
 
+    # Host buffers: the inputs of every call go up on one copy stream and the results come down on another, so that the
+    # copies of a call overlap the kernels of its neighbours (PCIe is full duplex); a step begins when the previous one
+    # has completely finished and ends when its last result has landed.
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
     # groups of layers that share one row structure share one sort
     def hot_path(from_host: bool):
         lgd = logits
+        ev_in = []
+        if from_host:
+            fork = torch.cuda.Event()
+            fork.record(stream)
+            s_in.wait_event(fork)
+            s_out.wait_event(fork)
+            with torch.cuda.stream(s_in):
+                if not on_device_router:
+                    lgd.copy_(logits_h, non_blocking=True)
+                for g in groups:
+                    for j in g:
+                        layers[j]["X"].copy_(layers[j]["Xh"], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(s_in)
+                    ev_in.append(ev)
+            stream.wait_event(ev_in[0])                     # (recorded after the logits and the first call's inputs)
         if on_device_router:
-            if from_host:
-                layers[0]["X"].copy_(layers[0]["Xh"], non_blocking=True)
             _, ids = moqe.moqe_router_mlp(layers[0]["X"], layers[0]["row_off"], rW1, rW2, workspace=r_ws)
         else:
-            if from_host:
-                lgd.copy_(logits_h, non_blocking=True)
             if one_launch_routing:                          # a decode step: arg-max, expansion and sort in one launch
                 L0 = layers[0]
                 _, _, perm, offsets = moqe.moqe_route_permute(lgd, L0["row_off"], L0["M"])
@@ -452,11 +469,10 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
                 ids = moqe.moqe_route(lgd)
         if not one_launch_routing:
             sorted_for = {}
-        for g in groups:
+        for gi, g in enumerate(groups):
             Ls = [layers[j] for j in g]
             if from_host:
-                for L in Ls:
-                    L["X"].copy_(L["Xh"], non_blocking=True)
+                stream.wait_event(ev_in[gi])
             key = Ls[0]["spec"].rows_per_sample
             if key not in sorted_for:
                 row_ids = moqe.moqe_expand_ids(ids, Ls[0]["row_off"], Ls[0]["M"])
@@ -465,8 +481,16 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
             perm, offsets = sorted_for[key]
             run_group(g, perm, offsets)
             if from_host:
-                for L in Ls:
-                    L["Yh"].copy_(L["Y"], non_blocking=True)
+                done = torch.cuda.Event()
+                done.record(stream)
+                s_out.wait_event(done)
+                with torch.cuda.stream(s_out):
+                    for L in Ls:
+                        L["Yh"].copy_(L["Y"], non_blocking=True)
+        if from_host:
+            join = torch.cuda.Event()
+            join.record(s_out)
+            stream.wait_event(join)
         return sorted_for
 
     def make_runner(from_host: bool):
