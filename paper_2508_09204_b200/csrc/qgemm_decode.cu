@@ -57,6 +57,7 @@ constexpr int GV_CHUNK_KB = 16;                                // k-blocks per c
 constexpr int GV_SBUF = GV_CHUNK_KB * 8 * 2 * 4;               // the chunk's sums: [k-block][token block][t][4] floats
 constexpr int GV_SLOT_FLOATS = GV_CONS * 2 * 4 * 32;           // a parked partial sum: 256 channels x 16 tokens
 constexpr int GV_MAX_GRID = 256;
+constexpr int GV_PREFETCH_TILES = 4;                           // super-tiles asked of L2 before the dependency wait
 
 // FUSED: the variant with gated pairs and residual adds (it gives 8 KB of the ring to the exchange buffer)
 template <bool FUSED>
@@ -317,22 +318,17 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // from here on the previous kernel's results are needed (sort tables, activations, workspace)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (tid >= 32 && tid <= 32 + p.R) s_off[tid - 32] = p.offsets[tid - 32];
-    if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
-
-    // ---- the work split, by warp 0: lane v works out pair v
-    if (warp == 0) {
+    // ---- the work split, by warp 0: lane v works out pair v from the offset table (read past L1: the table may be
+    // rewritten by the previous kernel between the two reads below)
+    auto work_split = [&]() {
         const int v = lane;
         long long cost = 0;
         int TT = 0, wv = 1;
-        if (v < p.P) {
-            const PairS q = p.ps[v];
-            const int rows = p.offsets[q.rexp + 1] - p.offsets[q.rexp];
+        {
+            const PairS q = p.ps[v < p.P ? v : 0];
+            const int rows = __ldcg(p.offsets + q.rexp + 1) - __ldcg(p.offsets + q.rexp);
             wv = q.w;
-            TT = rows > 0 ? ((FUSED && q.gated) ? q.NT1 : (q.NT1 + 1) >> 1) * q.KB : 0;
+            TT = (v < p.P && rows > 0) ? ((FUSED && q.gated) ? q.NT1 : (q.NT1 + 1) >> 1) * q.KB : 0;
             cost = (long long)TT * wv;
         }
         long long incl = cost;
@@ -379,6 +375,46 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             s_geom[0] = min(GV_MAX_STAGES, L::ring_bytes / stage_bytes);
             s_geom[1] = stage_bytes;
         }
+    };
+    // A guess at the split from whatever the offset table holds before the previous kernel is known to have finished
+    // (in a block's later launches it is final already), used ONLY to ask L2 for the first packed tiles this CTA would
+    // stream: a CTA that starts while the previous kernel's last CTAs are still running spends the wait pulling its
+    // weights out of HBM.  A wrong guess costs some prefetched lines; every address lies inside the pair's tile array.
+    int guess_off = 0, guess_last = 0;
+    if (warp == 0) {
+        guess_off = lane <= p.R ? __ldcg(p.offsets + lane) : 0;
+        guess_last = p.R >= 32 ? __ldcg(p.offsets + p.R) : 0;
+        work_split();
+        __syncwarp();
+        if (lane == 0) {
+            GvWalk wk;
+            wk.start();
+            bool changed;
+            int left = GV_PREFETCH_TILES;
+            while (left > 0 && wk.next(s_pair, p.ps, p.P, changed)) {
+                const int v = wk.v, n = min(wk.run(), left);
+                const PairS q = p.ps[v];
+                const bool gated = FUSED && q.gated;
+                const int nt = gated ? wk.nt2 : 2 * wk.nt2;
+                const uint8_t* a = p.ex[v].tiles + ((size_t)nt * wk.KB + wk.kb) * q.stride;
+                const uint8_t* b2 = gated ? p.tiles2[v] + ((size_t)nt * wk.KB + wk.kb) * q.stride
+                                          : (nt + 1 < q.NT1 ? a + (size_t)wk.KB * q.stride : nullptr);
+                // the run's tiles are contiguous: one request per 128-channel tile row
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"(n * q.stride) : "memory");
+                if (b2) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(b2), "r"(n * q.stride) : "memory");
+                left -= n;
+            }
+        }
+    }
+    // from here on the previous kernel's results are needed (sort tables, activations, workspace)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (tid >= 32 && tid <= 32 + p.R) s_off[tid - 32] = __ldcg(p.offsets + tid - 32);
+    if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+    if (warp == 0) {
+        const int my_off = lane <= p.R ? __ldcg(p.offsets + lane) : 0;
+        const int my_last = p.R >= 32 ? __ldcg(p.offsets + p.R) : 0;
+        if (!__all_sync(0xffffffffu, my_off == guess_off && my_last == guess_last)) work_split();   // (else the guess was the split)
     }
     __syncthreads();
     const int nstg = s_geom[0], stage_bytes = s_geom[1];
