@@ -756,13 +756,12 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                     unsigned* counter = p.counters + c_a * GV_CONS + (gated ? blob : warp);
                     const unsigned last = (unsigned)(gated ? 2 * (c_b - c_a) + 1 : c_b - c_a);
                     unsigned arrived = 0;
-                    if (lane == 0) {
-                        __threadfence();
-                        arrived = atomicAdd(counter, 1u);
-                    }
+                    // one acquire-release increment: the release side publishes the warp's parked sums (ordered before it
+                    // by the warp barrier above), the acquire side lets the last arriver read everybody else's
+                    if (lane == 0) asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(counter) : "memory");
                     arrived = __shfl_sync(0xffffffffu, arrived, 0);
                     if (arrived == last) {
-                        __threadfence();
+                        __syncwarp();
                         auto gather = [&](int wsrc, float (&dst)[8]) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) dst[i] = 0.f;
@@ -819,8 +818,9 @@ int dec_sm_count() {
     return n > 0 ? n : 148;
 }
 
-// relative cost of one super-tile in the work split, by code width
-int g_dec_cost[9] = {0, 0, 0, 10, 10, 0, 0, 0, 10};
+// relative cost of one super-tile in the work split, by code width (measured: a 3-bit super-tile takes the consumers
+// about a tenth longer than a 4-bit one, an 8-bit one lies between -- its copies are twice as large)
+int g_dec_cost[9] = {0, 0, 0, 22, 20, 0, 0, 0, 21};
 
 bool dec_formats_ok(const moqe_expert* const* ex, int n) {
     for (int v = 0; v < n; ++v) {
