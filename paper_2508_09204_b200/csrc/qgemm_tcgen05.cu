@@ -381,8 +381,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                         uint32_t v[32];
                         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * TN + col0 + c * 32, v);
                         tmem_ld_wait();
+                        // acc += s * v, two columns per instruction (each half rounds as a scalar fma does)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(s, __uint_as_float(v[i]), acc[c * 32 + i]);
+                        for (int i = 0; i < 32; i += 2)
+                            asm("{\n\t.reg .b64 a, x, s2;\n\tmov.b64 a, {%0, %1};\n\tmov.b64 x, {%3, %4};\n\tmov.b64 s2, {%2, %2};\n\t"
+                                "fma.rn.f32x2 a, s2, x, a;\n\tmov.b64 {%0, %1}, a;\n\t}"
+                                : "+f"(acc[c * 32 + i]), "+f"(acc[c * 32 + i + 1]) : "f"(s), "r"(v[i]), "r"(v[i + 1]));
                     }
                 }
                 tc_fence_before();
