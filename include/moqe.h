@@ -50,7 +50,7 @@ typedef enum {
     MOQE_OK = 0,
     MOQE_ERR_NULL = 1,         /* a required pointer is NULL */
     MOQE_ERR_SHAPE = 2,        /* a size is negative, zero where it may not be, or inconsistent */
-    MOQE_ERR_UNSUPPORTED = 3,  /* bits not in {3,4,8}; group not 0, 32, 64 or a multiple of 128;
+    MOQE_ERR_UNSUPPORTED = 3,  /* bits not in {2,3,4,8}; group not 0, 32, 64 or a multiple of 128;
                                   K % 8 != 0; E > MOQE_MAX_EXPERTS; misaligned pointer */
     MOQE_ERR_ALLOC = 4,        /* device allocation failed */
     MOQE_ERR_WORKSPACE = 5,    /* workspace NULL or smaller than the *_workspace() figure */
@@ -78,7 +78,7 @@ typedef struct moqe_expert moqe_expert;
  *   asymmetric: lo = min(0,min w), hi = max(0,max w), s = fp16((hi-lo)/(2^b-1)),
  *               z = clamp(rint(-lo/s), 0, 2^b-1), c = clamp(rint(w/s)+z, 0, 2^b-1)
  *   s == 0 or non-finite after the fp16 rounding -> s = 1;   dequant = s*(c-z).
- * W: device fp32 [N][K], finite.  bits in {3,4,8}; group 0, 32, 64 or a multiple
+ * W: device fp32 [N][K], finite.  bits in {2,3,4,8}; group 0, 32, 64 or a multiple
  * of 128, dividing K.  On success *out owns new device buffers (cudaMalloc'ed by
  * this call; it is therefore not capturable in a CUDA graph) and must be
  * released with moqe_expert_destroy.  The kernels run on `stream`.

@@ -15,6 +15,7 @@ template <int BITS> struct PieceWords;
 template <> struct PieceWords<4> { static constexpr int n = 4; };
 template <> struct PieceWords<8> { static constexpr int n = 8; };
 template <> struct PieceWords<3> { static constexpr int n = 3; };
+template <> struct PieceWords<2> { static constexpr int n = 2; };
 
 __device__ __forceinline__ uint32_t hsub2_bf16(uint32_t a, uint32_t b) {
     __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a), y = *reinterpret_cast<__nv_bfloat162*>(&b);
@@ -35,6 +36,12 @@ __device__ __forceinline__ void unpack_chunk(const uint32_t (&w)[PieceWords<BITS
         const uint32_t v = w[G];
 #pragma unroll
         for (int i = 0; i < 4; ++i) out[i] = hsub2_bf16(((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u, zz);
+    } else if constexpr (BITS == 2) {
+        // word G / 2 holds chunks G & ~1 and G | 1: pair i of chunk G is field 4 * (G & 1) + i of both halfwords
+        const uint32_t zz = pack_bf16x2(128.f + z, 128.f + z);
+        const uint32_t v = w[G >> 1] >> (8 * (G & 1));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = hsub2_bf16(((v >> (2 * i)) & 0x00030003u) | 0x43004300u, zz);
     } else if constexpr (BITS == 3) {
         const uint32_t zz = pack_bf16x2(128.f + z, 128.f + z);
 #pragma unroll
@@ -71,11 +78,15 @@ constexpr float W8_PRESCALE = 8192.f;
 // The caller removes (128 + z) * sum_k X with the help of a second MMA against an all-ones operand.
 template <int BITS, int G>
 __device__ __forceinline__ void unpack_chunk_biased(const uint32_t (&w)[PieceWords<BITS>::n], uint32_t (&out)[4]) {
-    static_assert(BITS == 4 || BITS == 3, "biased form exists for 4- and 3-bit codes");
+    static_assert(BITS == 4 || BITS == 3 || BITS == 2, "biased form exists for 4-, 3- and 2-bit codes");
     if constexpr (BITS == 4) {
         const uint32_t v = w[G];
 #pragma unroll
         for (int i = 0; i < 4; ++i) out[i] = ((v >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+    } else if constexpr (BITS == 2) {
+        const uint32_t v = w[G >> 1] >> (8 * (G & 1));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = ((v >> (2 * i)) & 0x00030003u) | 0x43004300u;
     } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -99,6 +110,9 @@ __device__ __forceinline__ void load_piece_smem(const unsigned char* blob, int h
         uint4 v = *reinterpret_cast<const uint4*>(blob + half * 1024 + slot * 16);
         uint4 u = *reinterpret_cast<const uint4*>(blob + half * 1024 + 512 + slot * 16);
         w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w; w[4] = u.x; w[5] = u.y; w[6] = u.z; w[7] = u.w;
+    } else if constexpr (BITS == 2) {
+        uint2 v = *reinterpret_cast<const uint2*>(blob + slot * 16 + half * 8);
+        w[0] = v.x; w[1] = v.y;
     } else {
         if (half == 0) {
             uint4 v = *reinterpret_cast<const uint4*>(blob + slot * 16);

@@ -101,6 +101,12 @@ __device__ __forceinline__ void load_chunk_smem(LaneBlob<BITS>& b, const unsigne
     if constexpr (BITS == 4) {
         b.lo[G] = *reinterpret_cast<const uint32_t*>(blob + slot * 16 + 4 * G);
         b.hi[G] = *reinterpret_cast<const uint32_t*>(blob + 512 + slot * 16 + 4 * G);
+    } else if constexpr (BITS == 2) {
+        if constexpr (G == 0) {          // one 16-byte slot holds the pieces of both rows
+            const uint4 x = *reinterpret_cast<const uint4*>(blob + slot * 16);
+            b.lo[0] = x.x; b.lo[1] = x.y;
+            b.hi[0] = x.z; b.hi[1] = x.w;
+        }
     } else if constexpr (BITS == 8) {
         const uint2 l = *reinterpret_cast<const uint2*>(blob + (G >> 1) * 512 + slot * 16 + 8 * (G & 1));
         const uint2 h = *reinterpret_cast<const uint2*>(blob + 1024 + (G >> 1) * 512 + slot * 16 + 8 * (G & 1));
@@ -531,6 +537,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) qgemm_stream_kernel(const _
     } while (0)
                 if (ex.bits == 4) MOQE_MAIN_NT(4);
                 else if (ex.bits == 8) MOQE_MAIN_NT(8);
+                else if (ex.bits == 2) MOQE_MAIN_NT(2);
                 else MOQE_MAIN_NT(3);
 #undef MOQE_MAIN_NT
 #undef MOQE_MAIN
@@ -620,7 +627,7 @@ int sm_count() {                              // of the current device (asked ev
 
 // relative cost of one packed tile in the work split.  Measured: a tile costs about the same time whatever its
 // width (the per-tile latency of a consumer warp, not its bytes, sets the pace), hence equal costs.
-int g_tile_cost[9] = {0, 0, 0, 8, 8, 0, 0, 0, 8};
+int g_tile_cost[9] = {0, 0, 8, 8, 8, 0, 0, 0, 8};
 
 }  // namespace
 

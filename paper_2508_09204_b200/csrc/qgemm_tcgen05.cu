@@ -334,6 +334,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                     ok = dequant_kblock<4>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 else if (ex.bits == 8)
                     ok = dequant_kblock<8>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                else if (ex.bits == 2)
+                    ok = dequant_kblock<2>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 else
                     ok = dequant_kblock<3>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 wring.advance(NWS);

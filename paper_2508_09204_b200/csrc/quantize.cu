@@ -32,6 +32,13 @@ __device__ __forceinline__ void encode_piece(const uint32_t (&c)[32], uint32_t (
             }
             w[G] = v;
         }
+    } else if constexpr (BITS == 2) {
+        w[0] = w[1] = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int G = i >> 3, t = i & 7;
+            w[G >> 1] |= (c[i] & 3u) << (2 * (4 * (G & 1) + (t >> 1)) + 16 * (t & 1));
+        }
     } else if constexpr (BITS == 8) {
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -62,6 +69,12 @@ __device__ __forceinline__ void decode_piece(const uint32_t (&w)[PieceWords<BITS
                 int nib = (t & 1) ? 4 + (t >> 1) : (t >> 1);
                 c[8 * G + t] = (w[G] >> (4 * nib)) & 0xFu;
             }
+    } else if constexpr (BITS == 2) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int G = i >> 3, t = i & 7;
+            c[i] = (w[G >> 1] >> (2 * (4 * (G & 1) + (t >> 1)) + 16 * (t & 1))) & 3u;
+        }
     } else if constexpr (BITS == 8) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) c[i] = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
@@ -85,6 +98,8 @@ template <int BITS>
 __device__ __forceinline__ void store_piece(uint8_t* blob, int half, int slot, const uint32_t (&w)[PieceWords<BITS>::n]) {
     if constexpr (BITS == 4) {
         *reinterpret_cast<uint4*>(blob + half * 512 + slot * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else if constexpr (BITS == 2) {
+        *reinterpret_cast<uint2*>(blob + slot * 16 + half * 8) = make_uint2(w[0], w[1]);
     } else if constexpr (BITS == 8) {
         *reinterpret_cast<uint4*>(blob + half * 1024 + slot * 16) = make_uint4(w[0], w[1], w[2], w[3]);
         *reinterpret_cast<uint4*>(blob + half * 1024 + 512 + slot * 16) = make_uint4(w[4], w[5], w[6], w[7]);
@@ -101,6 +116,9 @@ __device__ __forceinline__ void load_piece(const uint8_t* blob, int half, int sl
     if constexpr (BITS == 4) {
         uint4 v = *reinterpret_cast<const uint4*>(blob + half * 512 + slot * 16);
         w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else if constexpr (BITS == 2) {
+        uint2 v = *reinterpret_cast<const uint2*>(blob + slot * 16 + half * 8);
+        w[0] = v.x; w[1] = v.y;
     } else if constexpr (BITS == 8) {
         uint4 v = *reinterpret_cast<const uint4*>(blob + half * 1024 + slot * 16);
         uint4 u = *reinterpret_cast<const uint4*>(blob + half * 1024 + 512 + slot * 16);
@@ -302,7 +320,7 @@ __global__ void meta_import_kernel(const uint16_t* __restrict__ scales_in, const
 
 moqe_status check_format(int N, int K, int bits, int group) {
     if (N <= 0 || K <= 0) return MOQE_ERR_SHAPE;
-    if (bits != 3 && bits != 4 && bits != 8) return MOQE_ERR_UNSUPPORTED;
+    if (bits != 2 && bits != 3 && bits != 4 && bits != 8) return MOQE_ERR_UNSUPPORTED;
     if (K % 8 != 0) return MOQE_ERR_UNSUPPORTED;
     if (group < 0) return MOQE_ERR_SHAPE;
     if (group != 0) {
@@ -352,6 +370,7 @@ moqe_status launch_encode(const moqe_expert* e, const float* W, const uint8_t* c
                                                               e->scales_pc, e->zeros_pc, npieces)
     if (e->bits == 4) MOQE_ENC(4);
     else if (e->bits == 8) MOQE_ENC(8);
+    else if (e->bits == 2) MOQE_ENC(2);
     else MOQE_ENC(3);
 #undef MOQE_ENC
     count_launch();
@@ -420,6 +439,7 @@ extern "C" moqe_status moqe_expert_export(const moqe_expert* e, uint8_t* codes, 
         const int stride = moqe_tile_stride(e->bits, e->group, !e->sym);
         if (e->bits == 4) unpack_kernel<4><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
         else if (e->bits == 8) unpack_kernel<8><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
+        else if (e->bits == 2) unpack_kernel<2><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
         else unpack_kernel<3><<<blocks, 128, 0, st>>>(e->tiles, e->N, e->K, KB, stride, codes, npieces);
         count_launch();
     }
@@ -521,6 +541,7 @@ __global__ void dense_unpack_kernel(const __grid_constant__ DenseSrc src, int N,
     float* cs = col_scale + (size_t)e * Np;
     if (src.bits[e] == 4) dense_unpack_piece<4>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
     else if (src.bits[e] == 8) dense_unpack_piece<8>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
+    else if (src.bits[e] == 2) dense_unpack_piece<2>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
     else dense_unpack_piece<3>(src.tiles[e], src.scales_pc[e], src.zeros_pc[e], N, K, Kp, KB, src.group[e], src.sym[e], wd, cs, pid);
 }
 }  // namespace

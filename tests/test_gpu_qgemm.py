@@ -13,7 +13,7 @@ import moqe_workloads as wl
 pytestmark = pytest.mark.gpu
 
 ALL_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True), (3, 64, False), (4, 0, False),
-               (4, 32, False), (8, 128, False), (3, 32, True), (4, 256, False)]
+               (4, 32, False), (8, 128, False), (3, 32, True), (4, 256, False), (2, 128, False), (2, 64, True)]
 
 
 def _run(X, ids, gpu, path=0):
@@ -254,7 +254,7 @@ def test_dense_weights_kernel(M, N, K):
     per-image-like runs of rows and scattered rows, ragged tiles, ragged N and K, an idle expert; every element."""
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, assert_close
-    specs = [f for f in [(8, 0, True), (4, 0, False), (4, 32, False), (3, 64, False), (8, 128, False)] if f[1] == 0 or K % f[1] == 0]
+    specs = [f for f in [(8, 0, True), (4, 0, False), (4, 32, False), (3, 64, False), (8, 128, False), (2, 0, False), (2, 64, False)] if f[1] == 0 or K % f[1] == 0]
     W = wl.weights_f32(f"dn/{N}/{K}", N, K)
     X = wl.activations_bf16(f"dn/{M}/{K}", M, K, relu=True)
     gpu, What, _ = build_experts(W, specs)

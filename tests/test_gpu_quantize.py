@@ -11,7 +11,8 @@ import moqe_workloads as wl
 pytestmark = pytest.mark.gpu
 
 CASES = [(8, 0, True), (8, 128, False), (8, 0, False), (4, 128, False), (4, 128, True), (4, 0, False),
-         (4, 32, False), (4, 64, True), (3, 128, False), (3, 64, False), (3, 32, True), (3, 0, False), (4, 256, False)]
+         (4, 32, False), (4, 64, True), (3, 128, False), (3, 64, False), (3, 32, True), (3, 0, False), (4, 256, False),
+         (2, 128, False), (2, 0, True), (2, 32, False), (2, 64, True)]
 
 
 @pytest.mark.parametrize("bits,group,sym", CASES)
@@ -73,7 +74,7 @@ def test_storage_ratios_match_the_papers_table():
         assert abs(float(int4) / float(fp16) - e4.code_bytes / fp16_bytes) < 0.02
     # what is really allocated (and what a parked expert's image holds): codes + scales / zero-points, nothing else when
     # N and K are multiples of 128 -- for every format, true 3.0 bits per weight included
-    for bits, group, sym in [(8, 0, True), (4, 0, True), (4, 128, False), (3, 128, False), (3, 0, False), (4, 32, False), (8, 128, True)]:
+    for bits, group, sym in [(8, 0, True), (4, 0, True), (4, 128, False), (3, 128, False), (3, 0, False), (4, 32, False), (8, 128, True), (2, 128, False), (2, 0, True)]:
         e = moqe.moqe_quantize_rtn(W, bits, group, sym)
         assert e.code_bytes == 256 * 512 * bits // 8
         assert e.meta_bytes == 256 * (1 if group == 0 else 512 // group) * 2 * (1 if sym else 2)

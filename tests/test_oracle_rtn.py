@@ -176,7 +176,7 @@ def test_special_cases():
         oracle.quantize_rtn(W, 4, 100, False)
 
 
-@pytest.mark.parametrize("bits,sym", [(3, False), (4, False), (4, True), (8, True), (8, False)])
+@pytest.mark.parametrize("bits,sym", [(2, False), (2, True), (3, False), (4, False), (4, True), (8, True), (8, False)])
 def test_brute_force_nearest_code(bits, sym):
     """4x8 tiles: the returned code is the grid point nearest to w (exact arithmetic)."""
     rs = np.random.default_rng(100 + bits + int(sym))
