@@ -16,7 +16,7 @@
 //                           work split without walking it themselves.
 //
 //   Unpacking costs 5 integer instructions per 8 four-bit codes (1 per 2 eight-bit codes, 23 per 32 three-bit
-//   codes): a masked code dropped into the mantissa of the fp16 number 1024 becomes 1024 + c, or 1024 + 16c
+//   codes, 10 per 16 two-bit codes): a masked code dropped into the mantissa of the fp16 number 1024 becomes 1024 + c, or 1024 + 16c
 //   for a code that sits four bits higher -- no shift, no subtraction.  The tensor core multiplies by token
 //   values that were pre-scaled by 1/16 at exactly those k, and what the constants 1024 and the zero-point
 //   contribute is removed in fp32 with per-(token, k-block) sums of the token values:
@@ -164,17 +164,26 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 // Constants of the unpacking, held in registers the compiler cannot see through: (v & mask) | 0x64006400 is ONE
 // three-input logic instruction when mask and constant are registers, two when they are immediates.
 struct GvConst {
-    uint32_t base, m4lo, m4hi, m3a, m3b, m3c, m3s0, m3s1, m3s2;
+    uint32_t base, m4lo, m4hi, m3a, m3b, m3c, m3s0, m3s1, m3s2, m2a, m2b, m2c;
+    // only the constants of one code width are set (and live) at a time
+    template <int BITS>
     __device__ __forceinline__ void init() {
         asm volatile("mov.u32 %0, 0x64006400;" : "=r"(base));
-        asm volatile("mov.u32 %0, 0x000F000F;" : "=r"(m4lo));
-        asm volatile("mov.u32 %0, 0x00F000F0;" : "=r"(m4hi));
-        asm volatile("mov.u32 %0, 0x00070007;" : "=r"(m3a));
-        asm volatile("mov.u32 %0, 0x00380038;" : "=r"(m3b));
-        asm volatile("mov.u32 %0, 0x01C001C0;" : "=r"(m3c));
-        asm volatile("mov.u32 %0, 0x00400040;" : "=r"(m3s0));
-        asm volatile("mov.u32 %0, 0x00800080;" : "=r"(m3s1));
-        asm volatile("mov.u32 %0, 0x01000100;" : "=r"(m3s2));
+        if constexpr (BITS == 4) {
+            asm volatile("mov.u32 %0, 0x000F000F;" : "=r"(m4lo));
+            asm volatile("mov.u32 %0, 0x00F000F0;" : "=r"(m4hi));
+        } else if constexpr (BITS == 3) {
+            asm volatile("mov.u32 %0, 0x00070007;" : "=r"(m3a));
+            asm volatile("mov.u32 %0, 0x00380038;" : "=r"(m3b));
+            asm volatile("mov.u32 %0, 0x01C001C0;" : "=r"(m3c));
+            asm volatile("mov.u32 %0, 0x00400040;" : "=r"(m3s0));
+            asm volatile("mov.u32 %0, 0x00800080;" : "=r"(m3s1));
+            asm volatile("mov.u32 %0, 0x01000100;" : "=r"(m3s2));
+        } else if constexpr (BITS == 2) {
+            asm volatile("mov.u32 %0, 0x00030003;" : "=r"(m2a));
+            asm volatile("mov.u32 %0, 0x000C000C;" : "=r"(m2b));
+            asm volatile("mov.u32 %0, 0x00300030;" : "=r"(m2c));
+        }
     }
 };
 // (v & mask) | c: the fp16 numbers 1024 + (field value) in both halves, for a field inside the mantissa
@@ -191,6 +200,20 @@ __device__ __forceinline__ void unpack_w4(const GvConst& k, uint32_t v, uint32_t
     const uint32_t u = v >> 8;
     o[2] = and_or(u, k.m4lo, k.base);
     o[3] = and_or(u, k.m4hi, k.base);
+}
+// the 8 pairs of one 2-bit word (two chunks; pair f is field f of both halfwords, at bits 2f): 1024 + {1, 4, 16} * c --
+// fields 0..2 straight from the word, 3..5 after a shift by 6, 6..7 after a shift by 12
+__device__ __forceinline__ void unpack_w2(const GvConst& k, uint32_t v, uint32_t (&o)[8]) {
+    o[0] = and_or(v, k.m2a, k.base);
+    o[1] = and_or(v, k.m2b, k.base);
+    o[2] = and_or(v, k.m2c, k.base);
+    const uint32_t u = v >> 6;
+    o[3] = and_or(u, k.m2a, k.base);
+    o[4] = and_or(u, k.m2b, k.base);
+    o[5] = and_or(u, k.m2c, k.base);
+    const uint32_t t = v >> 12;
+    o[6] = and_or(t, k.m2a, k.base);
+    o[7] = and_or(t, k.m2b, k.base);
 }
 // pairs 0..3 of an 8-bit chunk held in two words: 1024 + c
 __device__ __forceinline__ void unpack_w8(uint32_t w0, uint32_t w1, uint32_t (&o)[4]) {
@@ -223,6 +246,7 @@ __device__ __forceinline__ void unpack_w3(const GvConst& k, uint32_t A, uint32_t
 __device__ __forceinline__ int sigma_shift(int bits, int p) {
     if (bits == 8) return 0;
     if (bits == 4) return (p & 1) ? 4 : 0;
+    if (bits == 2) return (p & 7) < 6 ? 2 * ((p & 7) % 3) : 2 * ((p & 7) - 6);
     return p == 15 ? 6 : 3 * ((p % 5) % 3);
 }
 
@@ -253,6 +277,24 @@ __device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int s
             for (int tb = 0; tb < NT; ++tb) {
                 mma_f16(acc[tb], ar[0], a8[0], ar[1], a8[1], b[tb][G].x, b[tb][G].y);
                 mma_f16(acc[tb], ar[2], a8[2], ar[3], a8[3], b[tb][G].z, b[tb][G].w);
+            }
+        }
+    } else if constexpr (BITS == 2) {
+        // one 16-byte slot: {row g: chunks 0,1 | chunks 2,3 | row g + 8: chunks 0,1 | chunks 2,3}
+        const uint4 w = lds128(blob + slot16);
+        const uint32_t a0[2] = {w.x, w.y}, a1[2] = {w.z, w.w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t ar[8], a8[8];
+            unpack_w2(kc, a0[h], ar);
+            unpack_w2(kc, a1[h], a8);
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg) {
+#pragma unroll
+                for (int tb = 0; tb < NT; ++tb) {
+                    mma_f16(acc[tb], ar[4 * gg], a8[4 * gg], ar[4 * gg + 1], a8[4 * gg + 1], b[tb][2 * h + gg].x, b[tb][2 * h + gg].y);
+                    mma_f16(acc[tb], ar[4 * gg + 2], a8[4 * gg + 2], ar[4 * gg + 3], a8[4 * gg + 3], b[tb][2 * h + gg].z, b[tb][2 * h + gg].w);
+                }
             }
         }
     } else if constexpr (BITS == 8) {
@@ -443,82 +485,92 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         const float fold = s_ps[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
         const uint32_t xbuf = sbase + L::x_off + buf * GV_XBUF;
         float* sbuf = reinterpret_cast<float*>(smem + L::s_off + buf * GV_SBUF);
-        // one 16-byte fetch (chunk a = 4G + q of the k-block: k = 32G + 8q ..) -> four fp16 pairs in MMA fragment order at
-        // [slab][G][lane = 4 mm + q]; the pair sums go into the group's partial sums
-        auto convert = [&](const uint4& dat, int a, uint32_t xdst, float& S0, float& S1) {
-            const int G = a >> 2, q = a & 3;
-            const uint32_t w[4] = {dat.x, dat.y, dat.z, dat.w};
-            uint32_t o[4];
+        // (the format's scale exponents are compile-time constants: one instantiation of the loop per code width)
+        auto stage_units = [&](auto bits_tag) {
+            // one 16-byte fetch (chunk a = 4G + q of the k-block: k = 32G + 8q ..) -> four fp16 pairs in MMA fragment order at
+            // [slab][G][lane = 4 mm + q]; the pair sums go into the group's partial sums
+            auto convert = [&](const uint4& dat, int a, uint32_t xdst, float& S0, float& S1) {
+                const int G = a >> 2, q = a & 3;
+                const uint32_t w[4] = {dat.x, dat.y, dat.z, dat.w};
+                uint32_t o[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
-                const int e = sigma_shift(bits, 4 * G + j);
-                const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
-                const float sum = lo + hi;
-                S0 += sum;
-                S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
-                __half2 hh = __floats2half2_rn(lo, hi);
-                const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
-                hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
-                o[j] = *reinterpret_cast<uint32_t*>(&hh);
-            }
-            sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
-        };
-        // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block.  The sums of a row tile are
-        // (g0 + g1) + (g2 + g3) over its four 32-value groups, whoever stages it.
-        const int units = nkb * NT * 8 * PARTS;
-        for (int u0 = st & ~31; u0 < units; u0 += nthr) {
-            const int unit = u0 + (st & 31);
-            const bool live = unit < units;
-            const int rt = unit / PARTS, part = unit % PARTS;
-            const int slab = rt >> 3, mm = rt & 7;
-            const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
-            const int k0 = (kbc + kbl) * 128;
-            const uint16_t* src = live && m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
-            const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
-            float S0, S1;
-            if constexpr (PARTS == 4) {
-                uint4 data[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int a = 4 * part + i;
-                    data[i] = make_uint4(0, 0, 0, 0);
-                    if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
+                for (int j = 0; j < 4; ++j) {
+                    // pair p = 4G + j of the piece: scaled by sigma = 2^-e, e fixed by the format
+                    constexpr int BITS = decltype(bits_tag)::value;
+                    const int e = sigma_shift(BITS, 4 * G + j);
+                    const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xFFFF0000u);
+                    const float sum = lo + hi;
+                    S0 += sum;
+                    S1 = fmaf(__int_as_float((127 - e) << 23), sum, S1);
+                    __half2 hh = __floats2half2_rn(lo, hi);
+                    const uint32_t sg = (uint32_t)((15 - e) << 10) * 0x00010001u;
+                    hh = __hmul2(hh, *reinterpret_cast<const __half2*>(&sg));
+                    o[j] = *reinterpret_cast<uint32_t*>(&hh);
                 }
-                S0 = 0.f; S1 = 0.f;
-                if (live) {
+                sts128(xdst + (G << 9) + (q << 4), o[0], o[1], o[2], o[3]);
+            };
+            // row tiles of the chunk: rt = slab * 8 + mm, slab = k-block * NT + token block.  The sums of a row tile are
+            // (g0 + g1) + (g2 + g3) over its four 32-value groups, whoever stages it.
+            const int units = nkb * NT * 8 * PARTS;
+            for (int u0 = st & ~31; u0 < units; u0 += nthr) {
+                const int unit = u0 + (st & 31);
+                const bool live = unit < units;
+                const int rt = unit / PARTS, part = unit % PARTS;
+                const int slab = rt >> 3, mm = rt & 7;
+                const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
+                const int k0 = (kbc + kbl) * 128;
+                const uint16_t* src = live && m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
+                const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
+                float S0, S1;
+                if constexpr (PARTS == 4) {
+                    uint4 data[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) convert(data[i], 4 * part + i, xdst, S0, S1);
-                }
-                S0 += __shfl_xor_sync(0xffffffffu, S0, 1);
-                S1 += __shfl_xor_sync(0xffffffffu, S1, 1);
-                S0 += __shfl_xor_sync(0xffffffffu, S0, 2);
-                S1 += __shfl_xor_sync(0xffffffffu, S1, 2);
-            } else {
-                float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint4 data[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int a = 8 * h + i;
+                    for (int i = 0; i < 4; ++i) {
+                        const int a = 4 * part + i;
                         data[i] = make_uint4(0, 0, 0, 0);
                         if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
                     }
+                    S0 = 0.f; S1 = 0.f;
                     if (live) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) convert(data[i], 8 * h + i, xdst, g0[2 * h + (i >> 2)], g1[2 * h + (i >> 2)]);
+                        for (int i = 0; i < 4; ++i) convert(data[i], 4 * part + i, xdst, S0, S1);
                     }
+                    S0 += __shfl_xor_sync(0xffffffffu, S0, 1);
+                    S1 += __shfl_xor_sync(0xffffffffu, S1, 1);
+                    S0 += __shfl_xor_sync(0xffffffffu, S0, 2);
+                    S1 += __shfl_xor_sync(0xffffffffu, S1, 2);
+                } else {
+                    float g0[4] = {0.f, 0.f, 0.f, 0.f}, g1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint4 data[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int a = 8 * h + i;
+                            data[i] = make_uint4(0, 0, 0, 0);
+                            if (src != nullptr && k0 + a * 8 < K) data[i] = __ldg(reinterpret_cast<const uint4*>(src + a * 8));
+                        }
+                        if (live) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) convert(data[i], 8 * h + i, xdst, g0[2 * h + (i >> 2)], g1[2 * h + (i >> 2)]);
+                        }
+                    }
+                    S0 = (g0[0] + g0[1]) + (g0[2] + g0[3]);
+                    S1 = (g1[0] + g1[1]) + (g1[2] + g1[3]);
                 }
-                S0 = (g0[0] + g0[1]) + (g0[2] + g0[3]);
-                S1 = (g1[0] + g1[1]) + (g1[2] + g1[3]);
+                // sums at [slab][t = mm / 2][4]
+                if (live && part == 0) {
+                    float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
+                    S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
+                    S[2] = S0;
+                }
             }
-            // sums at [slab][t = mm / 2][4]
-            if (live && part == 0) {
-                float* S = sbuf + slab * 16 + (mm >> 1) * 4 + (mm & 1);
-                S[0] = fmaf(-1024.f, S1, -fold * S0);              // what the accumulator starts from
-                S[2] = S0;
-            }
+        };
+        switch (bits) {
+            case 8: stage_units(std::integral_constant<int, 8>{}); break;
+            case 4: stage_units(std::integral_constant<int, 4>{}); break;
+            case 3: stage_units(std::integral_constant<int, 3>{}); break;
+            default: stage_units(std::integral_constant<int, 2>{}); break;
         }
         kbc += nkb;
         if (kbc >= kb1) {
@@ -588,8 +640,6 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         const int slot16 = (t * 8 + (g ^ (2 * t))) * 16;          // this lane's 16-byte slot inside a 512-byte half blob
         const uint32_t tile_base = sbase + L::ring_off + half * (stage_bytes >> 1);
         Ring ring;
-        GvConst kc;
-        kc.init();
         float fin[8];                                     // the running sums of the current piece: [token block][4]
 #pragma unroll
         for (int i = 0; i < 8; ++i) fin[i] = 0.f;
@@ -600,6 +650,8 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         auto run_chunk = [&](auto tag, int nkb, int buf, bool active) {
             constexpr int BITS = decltype(tag)::bits, NT = decltype(tag)::nt;
             constexpr bool GROUPED = decltype(tag)::grouped, ASYM = decltype(tag)::asym;
+            GvConst kc;
+            kc.template init<BITS>();
             const uint32_t xb0 = sbase + L::x_off + buf * GV_XBUF + lane * 16;
             const float4* sS = reinterpret_cast<const float4*>(smem + L::s_off + buf * GV_SBUF) + t;
             const uint32_t blob_off = blob * (BITS * 256);
@@ -678,7 +730,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                 }
             }
             // dispatch on the format (uniform over the CTA)
-            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : 2)) * 8 + (rows > 8 ? 4 : 0) + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
+            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : (bits == 3 ? 2 : 3))) * 8 + (rows > 8 ? 4 : 0) + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
             switch (fmt) {
 #define GV_CASE(B, BI, NTV, GR, AS) \
                 case BI * 8 + (NTV - 1) * 4 + GR * 2 + AS: run_chunk(GvTag<B, NTV, GR != 0, AS != 0>{}, nkb, buf, active); break;
@@ -687,6 +739,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                 GV_CASES(4, 0)
                 GV_CASES(8, 1)
                 GV_CASES(3, 2)
+                GV_CASES(2, 3)
 #undef GV_CASES
 #undef GV_CASE
                 default: break;
@@ -820,11 +873,11 @@ int dec_sm_count() {
 
 // relative cost of one super-tile in the work split, by code width (measured: a 3-bit super-tile takes the consumers
 // about a tenth longer than a 4-bit one, an 8-bit one lies between -- its copies are twice as large)
-int g_dec_cost[9] = {0, 0, 0, 22, 20, 0, 0, 0, 21};
+int g_dec_cost[9] = {0, 0, 20, 22, 20, 0, 0, 0, 21};
 
 bool dec_formats_ok(const moqe_expert* const* ex, int n) {
     for (int v = 0; v < n; ++v) {
-        if (ex[v]->bits != 3 && ex[v]->bits != 4 && ex[v]->bits != 8) return false;
+        if (ex[v]->bits != 2 && ex[v]->bits != 3 && ex[v]->bits != 4 && ex[v]->bits != 8) return false;
         if (ex[v]->group != 0 && (ex[v]->group < 128 || ex[v]->group % 128 != 0)) return false;
     }
     return true;

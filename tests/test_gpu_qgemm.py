@@ -70,7 +70,7 @@ def test_all_formats_small_shapes(path, M, N, K):
     assert_close(Y, oracle.routed_gemm(X, ids, What), f"M{M} N{N} K{K}")
 
 
-DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True), (4, 0, False), (8, 128, False),
+DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True), (4, 0, False), (8, 128, False), (2, 128, False), (2, 0, True), (2, 256, False),
                   (4, 256, False), (3, 0, True), (8, 0, False), (3, 256, True)]
 
 
