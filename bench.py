@@ -255,6 +255,8 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="timings of --steps steps each; the median is reported")
     ap.add_argument("--no-workloads", action="store_true", help="skip the sub-records of the other workloads")
     ap.add_argument("--force-expert", type=int, default=None, help="route every sample to this expert (per-format timing)")
+    ap.add_argument("--experts", default=None, help="replace the workload's expert formats: 'bits,group,sym;...' (same count), "
+                                                    "e.g. '8,0,1;2,128,0;3,128,0' (measurement of other formats on the same shapes)")
     ap.add_argument("--fused-block", action="store_true",
                     help="decode workloads: gate/up as ONE gated launch (silu(gate) * up), residual add in the o / down stores")
     args = ap.parse_args()
@@ -299,6 +301,13 @@ def main():
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
+    if args.experts:
+        import dataclasses
+        sp = tuple(wl.ExpertSpec(int(b), int(g), bool(int(y))) for b, g, y in (t.split(",") for t in args.experts.split(";")))
+        if len(sp) != len(w.experts):
+            raise SystemExit(f"--experts: workload {w.name} has {len(w.experts)} experts")
+        w = dataclasses.replace(w, experts=sp)
+        args.no_workloads = True
     line = bench_workload(ctx, w, steps=args.steps, warmup=args.warmup, repeats=args.repeats, with_e2e=True, force_expert=args.force_expert)
     line["clocks"] = sampler.stop()
 
@@ -605,7 +614,7 @@ def bench_workload(ctx, w, steps, warmup, repeats, with_e2e, force_expert=None):
     iso_ms = sum(layer_ms)
     tot_ms = block_ms
     n_launch = len(groups)
-    ratio = traffic_ratio(w.name) if args.path == 0 and not args.tune and force_expert is None else None
+    ratio = traffic_ratio(w.name) if args.path == 0 and not args.tune and force_expert is None and not args.experts else None
     traffic = None if ratio is None else ratio * sum(alg_bytes) / n_launch
     hbm_time = sum(alg_bytes) / (peaks["hbm_gbs"] * 1e9)
     tensor_time = sum(flops) / (peaks["bf16_tflops"] * 1e12)

@@ -23,6 +23,10 @@
 //                     i = 8*G + t is the low (t even) / high (t odd) half of pair p = i/2:
 //                     p < 15: word p/5, bits 3*(p%5) + 16*(i&1) .. +2
 //                     p = 15: bit b of the code is bit 15 + 16*(i&1) of word b.
+//   W2  blob  512 B : [slot] 16 B = {word 0, word 1 of half 0, word 0, word 1 of half 1}: one 16-byte load brings
+//                     a lane the pieces of channel rows r and r + 8.  A piece is two words; word j holds chunks 2j
+//                     and 2j+1; code i = 8*G + t is the low (t even) / high (t odd) half of field 4*(G&1) + t/2,
+//                     bits 2*field .. +1 of its halfword, so that ((w >> 2f) & 0x00030003) yields a pair.
 //
 // This piece/k assignment serves both GEMM kernels: a lane of an mma.sync
 // m16n8k16 fragment owns 4 k of every MMA (chunk halves), and every unpacked
