@@ -165,7 +165,9 @@ __device__ __forceinline__ bool dequant_kblock(const ExpertDev& ex, int nt, unsi
 }
 
 // ---------------------------------------------------------------------------- the kernel
-template <int TN, bool REGSPLIT>
+// W2: the instantiation that also takes 2-bit experts (kept apart: the extra unpack path costs the dequant warps of
+// the common instantiation 14 % through register allocation alone)
+template <int TN, bool REGSPLIT, bool W2>
 __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_constant__ TcParams p,
                                                                 const __grid_constant__ CUtensorMap tmap,
                                                                 const __grid_constant__ CUtensorMap tmap_x) {
@@ -334,9 +336,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) qgemm_tc_kernel(const __grid_co
                     ok = dequant_kblock<4>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 else if (ex.bits == 8)
                     ok = dequant_kblock<8>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
-                else if (ex.bits == 2)
-                    ok = dequant_kblock<2>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
-                else
+                else if (W2 && ex.bits == 2) {
+                    if constexpr (W2)
+                        ok = dequant_kblock<2>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
+                } else
                     ok = dequant_kblock<3>(ex, ti.nt, sw, smem + L::a_off, wf, we, wring.phase, bar_empty, bar_afull, ring, s_abort, p.status);
                 wring.advance(NWS);
             }
@@ -489,16 +492,20 @@ moqe_status launch_qgemm_tc(const void* X, int M, int N, int K, const moqe_exper
     long long max_tiles = ((long long)(M + tn - 1) / tn + E) * p.n_tiles;
     int grid = (int)(max_tiles < sms ? max_tiles : sms);
     cudaError_t err;
-    if (tn == 256) {
-        // (set at every launch: the attribute belongs to the current device, and the call is cheap)
-        if (cudaFuncSetAttribute(qgemm_tc_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<256>::dyn_bytes) != cudaSuccess)
-            return MOQE_ERR_CUDA;
-        qgemm_tc_kernel<256, true><<<grid, TC_THREADS, Smem<256>::dyn_bytes, st>>>(p, tmap, tmap_x);
-    } else {
-        if (cudaFuncSetAttribute(qgemm_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::dyn_bytes) != cudaSuccess)
-            return MOQE_ERR_CUDA;
-        qgemm_tc_kernel<128, false><<<grid, TC_THREADS, Smem<128>::dyn_bytes, st>>>(p, tmap, tmap_x);
-    }
+    bool any_w2 = false;
+    for (int e = 0; e < E; ++e) any_w2 = any_w2 || ex[e]->bits == 2;
+    // (the attribute is set at every launch: it belongs to the current device, and the call is cheap)
+    auto launch = [&](auto kernel, int smem) -> bool {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+        kernel<<<grid, TC_THREADS, smem, st>>>(p, tmap, tmap_x);
+        return true;
+    };
+    bool launched;
+    if (tn == 256)
+        launched = any_w2 ? launch(qgemm_tc_kernel<256, true, true>, Smem<256>::dyn_bytes) : launch(qgemm_tc_kernel<256, true, false>, Smem<256>::dyn_bytes);
+    else
+        launched = any_w2 ? launch(qgemm_tc_kernel<128, false, true>, Smem<128>::dyn_bytes) : launch(qgemm_tc_kernel<128, false, false>, Smem<128>::dyn_bytes);
+    if (!launched) return MOQE_ERR_CUDA;
     err = cudaGetLastError();
     count_launch();
     return cuda_ok(err);
