@@ -270,7 +270,9 @@ MOQE_API moqe_status moqe_routed_qgemm_path(const void* X_bf16, const int32_t* r
  * since a sample keeps its expert through the whole model (Section 3.1).
  * The split-K arrival counters at the head of the workspace body must be zero on
  * entry -- clear them once with moqe_routed_qgemm_workspace_clear after
- * allocating the workspace (same M, N, K, E) -- and every call leaves them zero.
+ * allocating the workspace (same M, N, K, E) -- and every call leaves them zero,
+ * except a call that ended in MOQE_ERR_TIMEOUT (moqe_async_status): clear the
+ * workspace again before it is reused after that.
  * `path` as for moqe_routed_qgemm_path. */
 MOQE_API moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t* perm, const int32_t* offsets, int M,
                                               const moqe_expert* const* h_experts, int E, void* Y_bf16,
