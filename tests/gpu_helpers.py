@@ -58,9 +58,23 @@ def compare_outputs(got_bits: np.ndarray, ref_bits: np.ndarray):
     return float(rel.max()) if ref.size else 0.0, float(d.mean()) if ref.size else 0.0
 
 
+def _where_off(got_bits, ref_bits) -> str:
+    """Which elements are outside the relative bar (for the failure message)."""
+    got = wl.bf16_bits_to_f32(got_bits).astype(np.float64)
+    ref = wl.bf16_bits_to_f32(ref_bits).astype(np.float64)
+    rho = np.sqrt(np.mean(ref ** 2)) if ref.size else 1.0
+    bad = np.abs(got - ref) / np.maximum(np.abs(ref), max(rho, 1e-30)) > MAX_REL_ERR
+    r, c = np.nonzero(bad.reshape(bad.shape[0], -1))
+    if r.size == 0:
+        return "no element off"
+    return (f"{r.size} elements off, rows {r.min()}..{r.max()} ({np.unique(r).size} rows: {np.unique(r)[:16].tolist()}), "
+            f"columns {c.min()}..{c.max()} ({np.unique(c).size} columns), first got {got.reshape(bad.shape[0], -1)[r[0], c[0]]:.6g} "
+            f"ref {ref.reshape(bad.shape[0], -1)[r[0], c[0]]:.6g}, zeros among them {(got.reshape(bad.shape[0], -1)[r, c] == 0).sum()}")
+
+
 def assert_close(got_bits, ref_bits, what=""):
     mx, mean = compare_outputs(got_bits, ref_bits)
-    assert mx <= MAX_REL_ERR, f"{what}: max relative error {mx:.3e} > {MAX_REL_ERR}"
+    assert mx <= MAX_REL_ERR, f"{what}: max relative error {mx:.3e} > {MAX_REL_ERR}; {_where_off(got_bits, ref_bits)}"
     assert mean <= MEAN_ABS_ERR, f"{what}: mean abs error {mean:.3e} > {MEAN_ABS_ERR}"
     return mx, mean
 
