@@ -241,7 +241,7 @@ MOQE_API moqe_status moqe_router_load_report(const float* logits, const int32_t*
  * invalid id are written as zeros).  M == 0 is valid.  workspace:
  * moqe_routed_qgemm_workspace(M, N, K, E) bytes, contents irrelevant on entry;
  * calls that share a workspace must not overlap on the device.
- * Decode batches (at most 16 rows, experts per-channel or with groups of 128 k or more) stream each touched
+ * Decode batches (at most 32 rows, experts per-channel or with groups of 128 k or more) stream each touched
  * expert's packed weights once through the decode kernel (bulk-copy ring, warp-level MMAs on fp16 operands,
  * stream-K split that follows the routing: experts without rows cost nothing).  That kernel converts the bf16
  * activations to fp16: values with |x| > 65504 are outside its domain (they become infinities); every other
@@ -256,7 +256,7 @@ MOQE_API moqe_status moqe_routed_qgemm(const void* X_bf16, const int32_t* row_id
 /* Same, with the kernel chosen by the caller (testing / measurement):
  * path 0 = automatic, 1 = split-K dequant-MMA streaming kernel, 2 = tcgen05 grouped GEMM (automatic
  * token tile), 3 / 4 = tcgen05 grouped GEMM with 128- / 256-token tiles, 5 = decode kernel
- * (MOQE_ERR_UNSUPPORTED if the batch has more than 16 rows or an expert has groups narrower than 128 k),
+ * (MOQE_ERR_UNSUPPORTED if the batch has more than 32 rows or an expert has groups narrower than 128 k),
  * 6 = dense-weights tcgen05 GEMM for large batches on small layers (more than 128 rows, K <= 1024, at most 1024
  * output channels; the automatic choice there: the layer is bound by its activations, so each expert's weights
  * are expanded to bf16 once per call and X / Y are streamed; MOQE_ERR_UNSUPPORTED otherwise). */
@@ -283,7 +283,7 @@ MOQE_API moqe_status moqe_routed_qgemm_sorted(const void* X_bf16, const int32_t*
  * host arrays of device pointers to layer l's input [M][K_l] and output [M][N_l]; h_experts[l * E + e] is expert
  * e of layer l (the E experts of a layer agree on N and K; layers may differ).  Same workspace rules as
  * moqe_routed_qgemm_sorted, sized for layer 0 (moqe_routed_qgemm_workspace(M, N_0, K_0, E)).
- * Only what the decode kernel takes: M <= 16, experts per-channel or with groups of 128 k or more,
+ * Only what the decode kernel takes: M <= 32, experts per-channel or with groups of 128 k or more,
  * n_layers * E <= MOQE_MAX_EXPERTS; otherwise MOQE_ERR_UNSUPPORTED and nothing is launched (call
  * moqe_routed_qgemm_sorted per layer instead). */
 MOQE_API moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16, const int32_t* perm, const int32_t* offsets,
@@ -292,7 +292,7 @@ MOQE_API moqe_status moqe_routed_qgemm_sorted_multi(const void* const* h_X_bf16,
                                                     void* stream);
 /* Two steps of an expert's forward pass fused into the routed product of a DECODE batch (Section 4.4 times whole
  * expert forwards, so what sits between two linear layers counts).  Same `perm` / `offsets` / workspace rules as
- * moqe_routed_qgemm_sorted; only what the decode kernel takes (M <= 16, experts per-channel or with groups of
+ * moqe_routed_qgemm_sorted; only batches of at most 16 rows of what the decode kernel takes (experts per-channel or with groups of
  * 128 k or more), otherwise MOQE_ERR_UNSUPPORTED and nothing is launched.
  *   _gated    : Y[m][n] = bf16( silu(a) * b ),  a = (X . Wgate_e^T)[m][n],  b = (X . Wup_e^T)[m][n],  e = the row's
  *               expert, silu(a) = a / (1 + exp(-a)); a and b are the fp32 sums, rounded once at the end.  h_gate[e] and

@@ -121,7 +121,7 @@ void stream_set_tile_cost(int bits, int cost);   // relative cost of one packed 
 
 // qgemm_decode.cu: decode shapes -- at most DECODE_MAX_ROWS rows, experts per-channel or with groups of >= 128 k;
 // nl layers that share the routing go down as one launch (ex[l * E + e] = expert e of layer l)
-constexpr int DECODE_MAX_ROWS = 16;
+constexpr int DECODE_MAX_ROWS = 32;
 bool decode_supported_multi(int M, const moqe_expert* const* ex, int nl, int E);
 size_t decode_workspace_bytes(int M);
 size_t decode_zero_bytes(int M);

@@ -1,4 +1,4 @@
-// Routed dequant-GEMM for decode shapes (a GEMV-like, HBM-bound path) (at most 16 token rows in the batch): every touched
+// Routed dequant-GEMM for decode shapes (a GEMV-like, HBM-bound path) (at most 32 token rows in the batch): every touched
 // expert's packed weights are streamed from HBM exactly once.
 //
 //   producer (1 thread)   : one bulk copy per packed 128x128-code tile (codes + the tile's scales / zero-points,
@@ -55,7 +55,8 @@ constexpr int GV_XCHG_BYTES = 8 * 8 * 32 * 4;                  // gated pairs: [
 constexpr int GV_XBUF = 32 * 1024;                             // one chunk of staged token rows
 constexpr int GV_CHUNK_KB = 16;                                // k-blocks per chunk for one token block (8 for two)
 constexpr int GV_SBUF = GV_CHUNK_KB * 8 * 2 * 4;               // the chunk's sums: [k-block][token block][t][4] floats
-constexpr int GV_SLOT_FLOATS = GV_CONS * 2 * 4 * 32;           // a parked partial sum: 256 channels x 16 tokens
+// a parked partial sum: 256 channels x 8 * NTMAX tokens
+__host__ __device__ constexpr int gv_slot_floats(int ntmax) { return GV_CONS * ntmax * 4 * 32; }
 constexpr int GV_MAX_GRID = 256;
 constexpr int GV_PREFETCH_TILES = 4;                           // super-tiles asked of L2 before the dependency wait
 
@@ -71,7 +72,7 @@ struct GvSmem {
     static constexpr int bar_off = desc_off + 2 * 32;                     // wfull[12] wempty[12] xfull[2] xempty[2]
     static constexpr int off_off = bar_off + (2 * GV_MAX_STAGES + 4) * 8;
     static constexpr int perm_off = off_off + (MOQE_MAX_EXPERTS + 2) * 4;
-    static constexpr int pair_off = perm_off + 16 * 4;                    // {tb, te} per pair
+    static constexpr int pair_off = perm_off + DECODE_MAX_ROWS * 4;       // {tb, te} per pair
     static constexpr int base_off = pair_off + MOQE_MAX_EXPERTS * 8;     // cost before each pair (long long)
     static constexpr int misc_off = base_off + MOQE_MAX_EXPERTS * 8;     // C (long long), G, stages, stage bytes, abort
     static constexpr int ps_off = misc_off + 32;                         // the pairs' scalars (a copy of GvParams::ps)
@@ -104,7 +105,7 @@ struct GvParams {
     const uint16_t* Res[MOQE_MAX_EXPERTS];  // residual added to the product before the rounding, or nullptr
     const int32_t* perm;
     const int32_t* offsets;
-    float* partials;                        // [CTA][2][GV_SLOT_FLOATS]
+    float* partials;                        // [CTA][2][gv_slot_floats(NTMAX)]
     uint32_t* counters;                     // [CTA][warp]: arrivals for the segment whose head that CTA holds; zero on entry, left zero
     int* status;
     int M, R, P;                            // rows of the batch, routing experts, pairs
@@ -258,8 +259,72 @@ struct GvTag {
 
 // The MMAs of one tile for one lane: `blob` is the shared-memory address of the warp's blob, `xb` that of the
 // lane's token fragments of this k-block.
+// The same for more than two token blocks: the token fragments are fetched where they are used (holding them all
+// would take 16 registers per block).
+template <int BITS, int NT>
+__device__ __forceinline__ void tile_mma_wide(const GvConst& kc, uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
+    auto step = [&](int G, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) {
+        // one 32-k group of both channel rows against every token block: a* = row g pairs 0..3, c* = row g + 8
+#pragma unroll
+        for (int tb = 0; tb < NT; ++tb) {
+            const uint4 b = lds128(xb + ((tb * 4 + G) << 9));
+            mma_f16(acc[tb], a0, c0, a1, c1, b.x, b.y);
+            mma_f16(acc[tb], a2, c2, a3, c3, b.z, b.w);
+        }
+    };
+    if constexpr (BITS == 4) {
+        const uint4 w0 = lds128(blob + slot16), w1 = lds128(blob + 512 + slot16);
+        const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+        for (int G = 0; G < 4; ++G) {
+            uint32_t ar[4], a8[4];
+            unpack_w4(kc, a0[G], ar);
+            unpack_w4(kc, a1[G], a8);
+            step(G, ar[0], ar[1], ar[2], ar[3], a8[0], a8[1], a8[2], a8[3]);
+        }
+    } else if constexpr (BITS == 2) {
+        const uint4 w = lds128(blob + slot16);
+        const uint32_t a0[2] = {w.x, w.y}, a1[2] = {w.z, w.w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t ar[8], a8[8];
+            unpack_w2(kc, a0[h], ar);
+            unpack_w2(kc, a1[h], a8);
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg)
+                step(2 * h + gg, ar[4 * gg], ar[4 * gg + 1], ar[4 * gg + 2], ar[4 * gg + 3], a8[4 * gg], a8[4 * gg + 1], a8[4 * gg + 2], a8[4 * gg + 3]);
+        }
+    } else if constexpr (BITS == 8) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint4 w0 = lds128(blob + u * 512 + slot16), w1 = lds128(blob + 1024 + u * 512 + slot16);
+            const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg) {
+                uint32_t ar[4], a8[4];
+                unpack_w8(a0[2 * gg], a0[2 * gg + 1], ar);
+                unpack_w8(a1[2 * gg], a1[2 * gg + 1], a8);
+                step(2 * u + gg, ar[0], ar[1], ar[2], ar[3], a8[0], a8[1], a8[2], a8[3]);
+            }
+        }
+    } else {
+        const uint4 w0 = lds128(blob + slot16);
+        const uint2 w1 = lds64(blob + 512 + (slot16 >> 1));
+        uint32_t ar[16], a8[16];
+        unpack_w3(kc, w0.x, w0.y, w0.z, ar);
+        unpack_w3(kc, w0.w, w1.x, w1.y, a8);
+#pragma unroll
+        for (int G = 0; G < 4; ++G)
+            step(G, ar[4 * G], ar[4 * G + 1], ar[4 * G + 2], ar[4 * G + 3], a8[4 * G], a8[4 * G + 1], a8[4 * G + 2], a8[4 * G + 3]);
+    }
+}
+
 template <int BITS, int NT>
 __device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int slot16, uint32_t xb, float (&acc)[NT][4]) {
+    if constexpr (NT > 2) {
+        tile_mma_wide<BITS, NT>(kc, blob, slot16, xb, acc);
+        return;
+    }
     uint4 b[NT][4];
 #pragma unroll
     for (int G = 0; G < 4; ++G)
@@ -333,9 +398,13 @@ __device__ __forceinline__ void tile_mma(const GvConst& kc, uint32_t blob, int s
 }
 
 // ---------------------------------------------------------------------------- the kernel
-template <bool FUSED>
+// NTMAX: token blocks of 8 rows an expert may get: 2 (batches of at most 16 rows), or 4 (at most 32 rows; its own
+// instantiation, so that the common one keeps its registers)
+template <bool FUSED, int NTMAX>
 __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __grid_constant__ GvParams p) {
     using L = GvSmem<FUSED>;
+    static_assert(NTMAX == 2 || (NTMAX == 4 && !FUSED), "gated pairs and residuals exist for batches of at most 16 rows");
+    constexpr int SLOT_FLOATS = gv_slot_floats(NTMAX);
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
@@ -452,7 +521,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid >= 32 && tid <= 32 + p.R) s_off[tid - 32] = __ldcg(p.offsets + tid - 32);
-    if (tid >= 64 && tid < 80) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
+    if (tid >= 64 && tid < 64 + 8 * NTMAX) s_perm[tid - 64] = tid - 64 < p.M ? p.perm[tid - 64] : 0;
     if (warp == 0) {
         const int my_off = lane <= p.R ? __ldcg(p.offsets + lane) : 0;
         const int my_last = p.R >= 32 ? __ldcg(p.offsets + p.R) : 0;
@@ -477,9 +546,9 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         }
         const int v = wk.v;
         const int row0 = s_off[s_ps[v].rexp], rows = s_off[s_ps[v].rexp + 1] - row0;
-        const int NT = rows > 8 ? 2 : 1;
+        const int ntl = (NTMAX > 2 && rows > 16) ? 2 : (rows > 8 ? 1 : 0), NT = 1 << ntl;      // token blocks: 1, 2 or 4
         const int kb1 = wk.kb + wk.run();
-        const int nkb = min(NT == 2 ? GV_CHUNK_KB / 2 : GV_CHUNK_KB, kb1 - kbc);
+        const int nkb = min(GV_CHUNK_KB >> ntl, kb1 - kbc);
         if (st == 0) { d->v = v; d->nt2 = wk.nt2; d->kbc = kbc; d->nkb = nkb; d->kb0 = wk.kb; d->kb1 = kb1; d->valid = 1; }
         const int bits = s_ps[v].bits, K = s_ps[v].K;
         const float fold = s_ps[v].has_zeros ? 0.f : (float)(1 << (bits - 1));   // a constant zero-point goes into the sums
@@ -517,7 +586,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                 const bool live = unit < units;
                 const int rt = unit / PARTS, part = unit % PARTS;
                 const int slab = rt >> 3, mm = rt & 7;
-                const int kbl = NT == 2 ? slab >> 1 : slab, m = (NT == 2 ? (slab & 1) * 8 : 0) + mm;
+                const int kbl = slab >> ntl, m = (slab & (NT - 1)) * 8 + mm;
                 const int k0 = (kbc + kbl) * 128;
                 const uint16_t* src = live && m < rows ? p.X[v] + (size_t)s_perm[row0 + m] * K + k0 : nullptr;
                 const uint32_t xdst = xbuf + (slab << 11) + (mm << 6);
@@ -640,9 +709,9 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
         const int slot16 = (t * 8 + (g ^ (2 * t))) * 16;          // this lane's 16-byte slot inside a 512-byte half blob
         const uint32_t tile_base = sbase + L::ring_off + half * (stage_bytes >> 1);
         Ring ring;
-        float fin[8];                                     // the running sums of the current piece: [token block][4]
+        float fin[4 * NTMAX];                             // the running sums of the current piece: [token block][4]
 #pragma unroll
-        for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+        for (int i = 0; i < 4 * NTMAX; ++i) fin[i] = 0.f;
         float sc_r = 0.f, sc_r8 = 0.f, z_r = 0.f, z_r8 = 0.f;     // per-channel experts: scale / zero-point of rows g, g + 8
         bool ok = true;
 
@@ -717,7 +786,7 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
             const int n_r = nt * 128 + blob * 16 + g;
             if (kbc == kb0) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) fin[i] = 0.f;
+                for (int i = 0; i < 4 * NTMAX; ++i) fin[i] = 0.f;
                 if (group == 0 && active) {
                     const __half* sp = gated && half ? p.scales_pc2[v] : p.ex[v].scales_pc;
                     sc_r = __half2float(sp[n_r]);
@@ -730,11 +799,15 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                 }
             }
             // dispatch on the format (uniform over the CTA)
-            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : (bits == 3 ? 2 : 3))) * 8 + (rows > 8 ? 4 : 0) + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
+            const int nti = (NTMAX > 2 && rows > 16) ? 2 : (rows > 8 ? 1 : 0);                  // 1, 2 or 4 token blocks
+            const int fmt = (bits == 4 ? 0 : (bits == 8 ? 1 : (bits == 3 ? 2 : 3))) * 12 + nti * 4 + (group != 0 ? 2 : 0) + (has_zeros ? 1 : 0);
             switch (fmt) {
-#define GV_CASE(B, BI, NTV, GR, AS) \
-                case BI * 8 + (NTV - 1) * 4 + GR * 2 + AS: run_chunk(GvTag<B, NTV, GR != 0, AS != 0>{}, nkb, buf, active); break;
-#define GV_CASES(B, BI) GV_CASE(B, BI, 1, 0, 0) GV_CASE(B, BI, 1, 0, 1) GV_CASE(B, BI, 1, 1, 0) GV_CASE(B, BI, 1, 1, 1) \
+#define GV_CASE(B, BI, NTI, GR, AS) \
+                case BI * 12 + NTI * 4 + GR * 2 + AS: \
+                    if constexpr ((1 << NTI) <= NTMAX) run_chunk(GvTag<B, (1 << NTI), GR != 0, AS != 0>{}, nkb, buf, active); \
+                    break;
+#define GV_CASES(B, BI) GV_CASE(B, BI, 0, 0, 0) GV_CASE(B, BI, 0, 0, 1) GV_CASE(B, BI, 0, 1, 0) GV_CASE(B, BI, 0, 1, 1) \
+                        GV_CASE(B, BI, 1, 0, 0) GV_CASE(B, BI, 1, 0, 1) GV_CASE(B, BI, 1, 1, 0) GV_CASE(B, BI, 1, 1, 1) \
                         GV_CASE(B, BI, 2, 0, 0) GV_CASE(B, BI, 2, 0, 1) GV_CASE(B, BI, 2, 1, 0) GV_CASE(B, BI, 2, 1, 1)
                 GV_CASES(4, 0)
                 GV_CASES(8, 1)
@@ -748,13 +821,13 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
 
             if (kbc + nkb == kb1 && active) {
                 // ---- the piece is complete
-                const int NT = rows > 8 ? 2 : 1;
+                const int NT = 1 << nti;
                 const int KB = s_ps[v].KB, N = s_ps[v].N;
                 uint16_t* Y = p.Y[v];
                 const uint16_t* R = FUSED ? p.Res[v] : nullptr;
                 auto store_rows = [&]() {
 #pragma unroll
-                    for (int tb = 0; tb < 2; ++tb) {
+                    for (int tb = 0; tb < NTMAX; ++tb) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const int m = 8 * tb + 2 * t + (j & 1), nn = n_r + (j >> 1) * 8;
@@ -768,9 +841,9 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                     }
                 };
                 // gated pair: fin <- silu(fin) * other, the second expert's product of the same channels and rows
-                auto gate_with = [&](const float (&other)[8]) {
+                auto gate_with = [&](const float (&other)[4 * NTMAX]) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) fin[i] = fin[i] / (1.f + expf(-fin[i])) * other[i];
+                    for (int i = 0; i < 4 * NTMAX; ++i) fin[i] = fin[i] / (1.f + expf(-fin[i])) * other[i];
                 };
                 float* xchg = reinterpret_cast<float*>(smem + L::xchg_off) + blob * 256 + lane;
                 if (kb0 == 0 && kb1 == KB) {
@@ -778,13 +851,13 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                         // warps w and w + 8 hold the two products of the same channels: hand the second to the first
                         if (half == 1) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) xchg[i * 32] = fin[i];
+                            for (int i = 0; i < 4 * NTMAX; ++i) xchg[i * 32] = fin[i];
                         }
                         asm volatile("bar.sync %0, 64;" ::"r"(2 + blob) : "memory");
                         if (half == 0) {
-                            float other[8];
+                            float other[4 * NTMAX];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) other[i] = xchg[i * 32];
+                            for (int i = 0; i < 4 * NTMAX; ++i) other[i] = xchg[i * 32];
                             gate_with(other);
                             store_rows();
                         }
@@ -799,12 +872,12 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                     const int G = *s_G, wv = s_ps[v].w;
                     const int c_a = (int)(((base + (long long)(nt2 * KB) * wv) * G) / C);
                     const int c_b = (int)(((base + (long long)(nt2 * KB + KB - 1) * wv) * G) / C);
-                    float* slot = p.partials + (size_t)(2 * blockIdx.x + (kb0 == 0 ? 1 : 0)) * GV_SLOT_FLOATS;
+                    float* slot = p.partials + (size_t)(2 * blockIdx.x + (kb0 == 0 ? 1 : 0)) * SLOT_FLOATS;
 #pragma unroll
-                    for (int tb = 0; tb < 2; ++tb)
+                    for (int tb = 0; tb < NTMAX; ++tb)
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
-                            if (tb < NT) __stcg(slot + ((warp * 2 + tb) * 4 + j) * 32 + lane, fin[4 * tb + j]);
+                            if (tb < NT) __stcg(slot + ((warp * NTMAX + tb) * 4 + j) * 32 + lane, fin[4 * tb + j]);
                     __syncwarp();
                     unsigned* counter = p.counters + c_a * GV_CONS + (gated ? blob : warp);
                     const unsigned last = (unsigned)(gated ? 2 * (c_b - c_a) + 1 : c_b - c_a);
@@ -815,30 +888,31 @@ __global__ void __launch_bounds__(GV_THREADS, 1) qgemm_decode_kernel(const __gri
                     arrived = __shfl_sync(0xffffffffu, arrived, 0);
                     if (arrived == last) {
                         __syncwarp();
-                        auto gather = [&](int wsrc, float (&dst)[8]) {
+                        auto gather = [&](int wsrc, float (&dst)[4 * NTMAX]) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) dst[i] = 0.f;
-                            // four CTAs' sums are fetched together (one round trip), then added in CTA order
-                            for (int c0 = c_a; c0 <= c_b; c0 += 4) {
-                                float part[4][8];
+                            for (int i = 0; i < 4 * NTMAX; ++i) dst[i] = 0.f;
+                            // several CTAs' sums are fetched together (one round trip), then added in CTA order
+                            constexpr int GB = NTMAX == 2 ? 4 : 2;
+                            for (int c0 = c_a; c0 <= c_b; c0 += GB) {
+                                float part[GB][4 * NTMAX];
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) {
+                                for (int u = 0; u < GB; ++u) {
                                     const int c = c0 + u;
-                                    const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * GV_SLOT_FLOATS;
+                                    const float* src = p.partials + (size_t)(2 * c + (c == c_a ? 1 : 0)) * SLOT_FLOATS;
 #pragma unroll
-                                    for (int tb = 0; tb < 2; ++tb)
+                                    for (int tb = 0; tb < NTMAX; ++tb)
 #pragma unroll
                                         for (int j = 0; j < 4; ++j)
-                                            part[u][4 * tb + j] = (c <= c_b && tb < NT) ? __ldcg(src + ((wsrc * 2 + tb) * 4 + j) * 32 + lane) : 0.f;
+                                            part[u][4 * tb + j] = (c <= c_b && tb < NT) ? __ldcg(src + ((wsrc * NTMAX + tb) * 4 + j) * 32 + lane) : 0.f;
                                 }
 #pragma unroll
-                                for (int u = 0; u < 4; ++u)
+                                for (int u = 0; u < GB; ++u)
 #pragma unroll
-                                    for (int i = 0; i < 8; ++i) dst[i] += part[u][i];
+                                    for (int i = 0; i < 4 * NTMAX; ++i) dst[i] += part[u][i];
                             }
                         };
                         if (FUSED && gated) {
-                            float other[8];
+                            float other[4 * NTMAX];
                             gather(blob, fin);
                             gather(blob + 8, other);
                             gate_with(other);
@@ -895,7 +969,7 @@ size_t decode_zero_bytes(int M) { return M > DECODE_MAX_ROWS ? 0 : (size_t)GV_MA
 
 size_t decode_workspace_bytes(int M) {
     if (M > DECODE_MAX_ROWS) return 0;
-    return (decode_zero_bytes(M) + 255) / 256 * 256 + (size_t)GV_MAX_GRID * 2 * GV_SLOT_FLOATS * sizeof(float);
+    return (decode_zero_bytes(M) + 255) / 256 * 256 + (size_t)GV_MAX_GRID * 2 * gv_slot_floats(M > 16 ? 4 : 2) * sizeof(float);
 }
 
 // nl layers that share the routing; ex[l * E + e] = expert e of layer l; X[l] / Y[l] the layer's input / output
@@ -952,8 +1026,9 @@ moqe_status launch_qgemm_decode_ext(const void* const* X, int M, int nl, const m
     if (grid > GV_MAX_GRID) grid = GV_MAX_GRID;
     p.small = total_cost * (grid + 1) < (1ll << 31) ? 1 : 0;
     const bool fused = ex2 != nullptr || R != nullptr;
+    if (fused && M > 16) return MOQE_ERR_UNSUPPORTED;     // gated pairs and residual adds: batches of at most 16 rows
     const int smem = fused ? GvSmem<true>::dyn_bytes : GvSmem<false>::dyn_bytes;
-    auto kernel = fused ? qgemm_decode_kernel<true> : qgemm_decode_kernel<false>;
+    auto kernel = fused ? qgemm_decode_kernel<true, 2> : (M > 16 ? qgemm_decode_kernel<false, 4> : qgemm_decode_kernel<false, 2>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};

@@ -78,9 +78,10 @@ DECODE_FORMATS = [(8, 0, True), (4, 128, False), (3, 128, False), (4, 128, True)
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 128), (5, 200, 320), (16, 384, 1280), (13, 136, 2304), (16, 1000, 640),
-                                   (7, 4096, 1024), (16, 512, 11008), (9, 128, 32768)])
+                                   (7, 4096, 1024), (16, 512, 11008), (9, 128, 32768), (17, 200, 320), (32, 384, 1280),
+                                   (29, 1000, 640), (32, 512, 11008), (24, 128, 32768)])
 def test_decode_kernel_all_formats(M, N, K):
-    """The decode kernel (path 5: at most 16 rows, per-channel experts or groups of >= 128 k): every such
+    """The decode kernel (path 5: at most 32 rows; above 16 its instantiation with four token blocks per expert, per-channel experts or groups of >= 128 k): every such
     format as its own expert, ragged N, K not a multiple of 128, split K with several contributors per segment
     (dozens in the last, one-tile-wide case, where most CTAs hold nothing but the middle of a segment), an expert
     that gets no rows."""
@@ -179,11 +180,11 @@ def test_exact_integer_case_on_gpu(path):
 @pytest.mark.parametrize("path", [1, 3, 4, 5])
 def test_degenerate_batches(path):
     """All rows to one expert, a shuffled batch, M = 0, ids outside [0, E) -- on every kernel; the decode kernel
-    (path 5) takes batches of at most 16 rows."""
+    (path 5) takes batches of at most 32 rows."""
     import paper_2508_09204_b200 as moqe
     from gpu_helpers import build_experts, assert_close, dev, bf16_to_torch
     N, K = 256, 512
-    Mb = 16 if path == 5 else 40
+    Mb = 32 if path == 5 else 40
     W = wl.weights_f32("deg", N, K)
     specs = [(8, 0, True), (4, 128, False), (3, 128, False)]
     gpu, What, _ = build_experts(W, specs)
